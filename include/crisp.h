@@ -1,0 +1,141 @@
+/*
+ * crisp.h — C ABI of the B200 (sm_100a) implementation of CRISP's sparse-prefill attention path.
+ *
+ * One attention layer, all heads, one GPU.  The path is Algorithm 1 of the paper:
+ *   crisp_route          proxy attention of the last query block + C_struct router + block scores
+ *                        (Algorithm 2; Eq. 2; Algorithm 3 lines 3-5)
+ *   crisp_select         sink-aware noise-floor selection (Algorithm 3 lines 6-12, Eq. 3-4), the
+ *                        cumulative-gamma comparison rule (Algorithm 6), pooled estimation for PE heads
+ *                        (Algorithm 4), and the expansion into per-query-block key-block lists
+ *   crisp_sparse_prefill exact softmax attention over the listed blocks, causal (Eq. 1)
+ *   crisp_dense_prefill  the same kernel over every causal block (the dense baseline)
+ *
+ * Conventions shared by every entry point
+ *   - Tensors are contiguous, row major, bf16: Q and O are [seq_len, n_q_heads, 128]; K and V are
+ *     [seq_len, n_kv_heads, 128].  Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - All data pointers are DEVICE pointers owned by the caller.  The library never allocates or frees
+ *     device memory; scratch memory is passed in as a workspace whose size crisp_workspace_bytes gives.
+ *     Q, K, V, O and workspaces must be 16-byte aligned (256-byte recommended).
+ *   - `cuda_stream` is a cudaStream_t (NULL = legacy default stream).  Calls only enqueue work on that
+ *     stream and return; they never synchronise, except crisp_poll_device_status.
+ *   - The return value is a crisp_status.  Host-side argument errors are reported immediately and
+ *     nothing is launched.  Device-side conditions (capacity overflow, a bounded wait that gave up) are
+ *     recorded in the first word of the workspace and read back with crisp_poll_device_status.
+ *   - Nothing throws, exits, traps or spins without a bound.
+ *   - The library needs a CUDA device of compute capability 10.0; there is no CPU fallback.
+ */
+#ifndef CRISP_H_
+#define CRISP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum crisp_status {
+  CRISP_OK = 0,
+  CRISP_ERR_INVALID_ARG = -1,    /* null pointer, non-positive size, inconsistent head counts, ...   */
+  CRISP_ERR_UNSUPPORTED = -2,    /* head_dim != 128, block != 128, seq_len not a multiple of block, ... */
+  CRISP_ERR_WORKSPACE = -3,      /* workspace too small or misaligned                                */
+  CRISP_ERR_CAPACITY = -4,       /* col_idx capacity too small for the selected blocks               */
+  CRISP_ERR_CUDA = -5,           /* a CUDA runtime / driver call failed (see crisp_last_cuda_error)  */
+  CRISP_ERR_DEVICE_TIMEOUT = -6  /* a bounded device-side wait gave up                               */
+} crisp_status;
+
+/* Pattern labels written by crisp_route (Algorithm 2). */
+#define CRISP_PATTERN_PE 0
+#define CRISP_PATTERN_VS 1
+
+/* Problem description: the inputs of Algorithm 1 plus the constants of Sections 3.2 and 4.3. */
+typedef struct crisp_params {
+  int32_t struct_size;   /* = sizeof(crisp_params); ABI guard                                        */
+  int32_t seq_len;       /* n; a multiple of `block`, at least 2 * block                             */
+  int32_t n_q_heads;     /* H_q                                                                      */
+  int32_t n_kv_heads;    /* H_kv; H_q % H_kv == 0 and H_q / H_kv <= 16                               */
+  int32_t head_dim;      /* 128 only                                                                 */
+  int32_t block;         /* B = 128 only (Section 4.3)                                               */
+  int32_t sink_tokens;   /* w_sink: anchor keys j < w_sink (Eq. 2; paper value 128), 1..seq_len      */
+  int32_t local_tokens;  /* w_local: anchor keys j >= n - w_local (Eq. 2; paper value 128)           */
+  int32_t k_min_blocks;  /* minimum budget per direction in blocks (paper: 1024 tokens = 8), >= 0    */
+  int32_t selector;      /* 0 = noise floor alpha (Algorithm 3); 1 = cumulative gamma (Algorithm 6)  */
+  int32_t force_pattern; /* 0 = route by C_struct; 1 = every head VS; 2 = every head PE              */
+  float tau;             /* tau_proxy: VS iff C_struct >= tau (paper 0.2)                            */
+  float alpha;           /* noise-floor multiplier (paper 1.0 / 1.25), >= 0                          */
+  float gamma;           /* cumulative-mass target: PE heads always, VS heads when selector == 1     */
+  float softmax_scale;   /* 0 => 1 / sqrt(head_dim)                                                  */
+} crisp_params;
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int crisp_version(void);
+
+/* Static string for a status code. */
+const char* crisp_status_string(int status);
+
+/* Text of the last CUDA error seen by this thread inside the library ("" if none). */
+const char* crisp_last_cuda_error(void);
+
+/*
+ * Minimum workspace sizes in bytes for the three stages (any output pointer may be NULL).
+ * The first 256 bytes of every workspace are a header whose first int32 is the device status word;
+ * crisp_route / crisp_select / crisp_*_prefill clear it on entry (on the stream); before the first
+ * such call on a workspace the word holds whatever the caller's allocation held.
+ */
+int crisp_workspace_bytes(const crisp_params* p, size_t* route_ws, size_t* select_ws, size_t* prefill_ws);
+
+/*
+ * Stage 1-3a (Algorithm 2; Algorithm 3 lines 3-5).  For every query head: the causal proxy attention
+ * A_hat of the last `block` queries against all keys (never written to memory), then
+ *   c_struct[h] = (1/block) sum_i sum_{j in anchors} A_hat[i, j]                              (Eq. 2)
+ *   pattern[h]  = VS if c_struct[h] >= tau else PE (or the forced pattern)
+ *   p_v[h, J]   = mass of key block J;  p_s[h, s] = mass of the diagonal band of block offset s,
+ * both normalised to sum to 1.  Outputs: c_struct [H_q] f32, pattern [H_q] i32, p_v, p_s [H_q, N_b] f32.
+ */
+int crisp_route(const crisp_params* p, const void* q, const void* k, void* ws, size_t ws_bytes,
+                float* c_struct, int32_t* pattern, float* p_v, float* p_s, void* cuda_stream);
+
+/*
+ * Stage 3b-3c.  VS heads: per direction d in {v, s}, mu_d = (sum of the middle blocks of p_d)/(N_b - 2),
+ * k_d = clip(#{p_d > alpha * mu_d}, k_min, N_b) (selector 0) or the smallest k whose top-k mass reaches
+ * gamma (selector 1), S_d = top-k_d with ties to the lower index (Algorithm 3 / Algorithm 6).
+ * PE heads: block means of Q and K, causal row softmax of their product, normalised by the total,
+ * smallest prefix of the descending order whose mass reaches gamma (Algorithm 4).
+ * Expansion: query block m of a VS head gets {0, m} u {J in S_v, J <= m} u {m-s, m-s-1 : s in S_s};
+ * of a PE head {0, m} u {J : (m, J) selected}.
+ *
+ * Output is CSR over (head, query block): row_ptr [H_q, N_b + 1] int64 with global offsets into col_idx
+ * (row_ptr[h][N_b] == row_ptr[h+1][0]); columns ascending, unique, all <= m, always containing 0 and m.
+ * *nnz_needed (device int64) receives the total number of entries.  If it exceeds `capacity`, col_idx is
+ * left untouched, the status word becomes CRISP_ERR_CAPACITY, and the lists must not be used.
+ * q, k are read only for PE heads.
+ */
+int crisp_select(const crisp_params* p, const void* q, const void* k, const int32_t* pattern,
+                 const float* p_v, const float* p_s, void* ws, size_t ws_bytes, int64_t* row_ptr,
+                 int32_t* col_idx, int64_t capacity, int64_t* nnz_needed, void* cuda_stream);
+
+/*
+ * Stage 4 (Eq. 1).  O[t, h, :] = sum_j softmax_j(Q[t,h] . K[j,kv(h)] * scale) V[j,kv(h)] over the keys j <= t
+ * of the key blocks listed for query block t / block.  Exact softmax over the kept keys; bf16 inputs,
+ * fp32 accumulation, bf16 output.  lse (optional, [H_q, seq_len] f32) receives the natural-log
+ * sum-exp of the kept scaled logits.  row_ptr / col_idx as produced by crisp_select (every row must
+ * contain its diagonal block).
+ */
+int crisp_sparse_prefill(const crisp_params* p, const void* q, const void* k, const void* v,
+                         const int64_t* row_ptr, const int32_t* col_idx, void* ws, size_t ws_bytes, void* o,
+                         float* lse, void* cuda_stream);
+
+/* Dense causal attention: crisp_sparse_prefill with every causal block listed (the baseline of Section 5). */
+int crisp_dense_prefill(const crisp_params* p, const void* q, const void* k, const void* v, void* ws,
+                        size_t ws_bytes, void* o, float* lse, void* cuda_stream);
+
+/*
+ * Synchronises `cuda_stream`, reads the status word at the start of `ws`, clears it and returns it
+ * (CRISP_OK, CRISP_ERR_CAPACITY or CRISP_ERR_DEVICE_TIMEOUT), or CRISP_ERR_CUDA if the stream failed.
+ */
+int crisp_poll_device_status(void* ws, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CRISP_H_ */

@@ -1,0 +1,63 @@
+// Shared host/device declarations of the CRISP library internals (not part of the public ABI).
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include "../../include/crisp.h"
+
+namespace crisp {
+
+constexpr int kBlock = 128;       // B: tokens per block (Section 4.3)
+constexpr int kHeadDim = 128;     // d
+constexpr int kMaxGroup = 16;     // H_q / H_kv
+constexpr size_t kWsHeader = 256; // bytes reserved at the start of every workspace (status word first)
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Validated, derived problem sizes passed to kernels by value.
+struct Dims {
+  int n;          // seq_len
+  int nb;         // N_b = n / B
+  int hq, hkv, group;
+  int w_sink, w_local;
+  int n_sink_tiles;    // key tiles intersecting [0, w_sink)
+  int first_local_tile; // first key tile (>= n_sink_tiles) intersecting [n - w_local, n)
+  int n_anchor_slots;  // n_sink_tiles + (nb - first_local_tile)
+  int k_min, selector, force_pattern;
+  float tau, alpha, gamma;
+  float scale;      // softmax scale
+  float scale_log2; // scale * log2(e)
+};
+
+int validate(const crisp_params* p, Dims* d);
+void set_cuda_error(cudaError_t e, const char* where);
+void set_cu_error(const char* msg);
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Tensor map of a [n, H, 128] bf16 tensor with a {64, 1, 128} box and 128-byte swizzle.
+int make_tmap_bf16_nhd(CUtensorMap* out, const void* base, int n, int heads, int box_rows = 128);
+
+#define CRISP_CUDA_TRY(expr, where)              \
+  do {                                           \
+    cudaError_t e__ = (expr);                    \
+    if (e__ != cudaSuccess) {                    \
+      ::crisp::set_cuda_error(e__, where);       \
+      return CRISP_ERR_CUDA;                     \
+    }                                            \
+  } while (0)
+
+// stage launchers (each enqueues on `stream` and returns a crisp_status)
+int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c_struct, int32_t* pattern,
+                 float* p_v, float* p_s, cudaStream_t stream);
+size_t route_ws_bytes(const Dims& d);
+int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pattern, const float* p_v,
+                  const float* p_s, void* ws, int64_t* row_ptr, int32_t* col_idx, int64_t capacity,
+                  int64_t* nnz_needed, cudaStream_t stream);
+size_t select_ws_bytes(const Dims& d);
+int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, const int64_t* row_ptr,
+                   const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream);
+size_t prefill_ws_bytes(const Dims& d);
+
+}  // namespace crisp

@@ -1,0 +1,515 @@
+// Stage 4: block-sparse (and dense) causal attention (Eq. 1) on tcgen05 tensor cores.
+//
+// One CTA processes work items; an item is one query head and a PAIR of adjacent query blocks
+// (two 128-row tiles).  Both tiles share every K/V block that TMA brings into shared memory, which
+// halves the L2 -> shared-memory traffic per flop.  The key blocks of the pair are the sorted union
+// of the two blocks' lists; each entry carries two flags saying which tile uses it.
+//
+// Warp roles (384 threads):
+//   warps 0-3  softmax of tile 0 (one thread per query row; TMEM lanes 0-127)
+//   warps 4-7  softmax of tile 1
+//   warp  8    TMA producer: Q once per item, K and V blocks through two-stage rings
+//   warp  9    MMA issuer: S_t = Q_t K^T (SS) and O_t += P_t V (P read from TMEM)
+// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each; P_t (bf16) overwrites the first
+// 64 columns of S_t.  The issuer interleaves the two tiles so that the tensor pipe works on one
+// tile while the other tile's softmax runs.  The online softmax rescales O lazily, only when the
+// running maximum grows by more than 2^8, and does it in place in TMEM.
+// Every mbarrier wait is bounded; a wait that gives up sets a flag that ends all roles, and the
+// status word reports CRISP_ERR_DEVICE_TIMEOUT.
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace crisp {
+using namespace sm100;
+
+namespace {
+
+constexpr uint32_t kFlag0 = 1u << 30, kFlag1 = 1u << 31, kColMask = kFlag0 - 1u;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+struct PrefillArgs {
+  const int32_t* merged;   // per item: union list, entry = key block | flags (sparse only)
+  const int64_t* row_ptr;  // [hq][nb+1]
+  const int* item_len;     // [hq][n_pairs] number of union entries (sparse only)
+  __nv_bfloat16* o;        // [n][hq][128]
+  float* lse;              // [hq][n] or null
+  int* status;
+  int n_pairs;
+  int n_items;
+};
+
+struct PrefillSmem {
+  alignas(1024) uint8_t q[2][2][16384];  // [tile][half]
+  alignas(1024) uint8_t k[2][2][16384];  // [stage][half]
+  alignas(1024) uint8_t v[2][2][16384];  // [stage][half]
+  uint64_t q_full, q_free;
+  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
+  uint64_t s_full[2], p_ready[2], o_done[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct Item {
+  int h, kvh, m0, m1;
+  bool tile1;
+  int n_entries;
+  long long base;  // offset of the item's union list
+};
+
+template <bool kDense>
+__device__ __forceinline__ Item decode_item(int idx, const Dims& d, const PrefillArgs& a) {
+  Item it;
+  it.h = idx % d.hq;
+  const int u = a.n_pairs - 1 - idx / d.hq;  // long rows first
+  it.kvh = it.h / d.group;
+  it.m0 = 2 * u;
+  it.m1 = 2 * u + 1;
+  it.tile1 = it.m1 < d.nb;
+  if (kDense) {
+    it.n_entries = it.tile1 ? it.m1 + 1 : it.m0 + 1;
+    it.base = 0;
+  } else {
+    it.n_entries = a.item_len[it.h * a.n_pairs + u];
+    it.base = a.row_ptr[static_cast<size_t>(it.h) * (d.nb + 1) + it.m0];
+  }
+  return it;
+}
+
+// Entry e of an item: key block and per-tile flags.  Sparse lists are fetched 32 entries at a time,
+// one per lane, and broadcast with a shuffle; all 32 lanes of the warp must call this together.
+template <bool kDense>
+struct EntryReader {
+  const int32_t* list;
+  uint32_t chunk;
+  int m0;
+  bool tile1;
+  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& a) {
+    list = kDense ? nullptr : a.merged + it.base;
+    m0 = it.m0;
+    tile1 = it.tile1;
+    chunk = 0;
+  }
+  __device__ __forceinline__ uint32_t get(int e, int n_entries, int lane) {
+    if (kDense) {
+      uint32_t x = static_cast<uint32_t>(e);
+      if (e <= m0) x |= kFlag0;
+      if (tile1) x |= kFlag1;
+      return x;
+    }
+    if ((e & 31) == 0) chunk = (e + lane < n_entries) ? static_cast<uint32_t>(list[e + lane]) : 0u;
+    return __shfl_sync(0xffffffffu, chunk, e & 31);
+  }
+};
+
+template <bool kDense>
+__global__ void __launch_bounds__(384, 1)
+prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+               const __grid_constant__ CUtensorMap tmap_v, const Dims d, const PrefillArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  PrefillSmem& s = *reinterpret_cast<PrefillSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    s.abort_flag = 0;
+    mbar_init(&s.q_full, 1);
+    mbar_init(&s.q_free, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s.k_full[i], 1);
+      mbar_init(&s.k_empty[i], 1);
+      mbar_init(&s.v_full[i], 1);
+      mbar_init(&s.v_empty[i], 1);
+      mbar_init(&s.s_full[i], 1);
+      mbar_init(&s.p_ready[i], 128);
+      mbar_init(&s.o_done[i], 1);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 8) {
+    tmem_alloc(&s.tmem_base, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tm = s.tmem_base;
+  volatile int* abort_flag = &s.abort_flag;
+
+  if (warp == 8) {
+    // =============================================================== TMA producer
+    if (lane == 0) {
+      prefetch_tmap(&tmap_q);
+      prefetch_tmap(&tmap_k);
+      prefetch_tmap(&tmap_v);
+    }
+    uint32_t ecount = 0;
+    int it_count = 0;
+    bool ok = true;
+    for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
+      const Item it = decode_item<kDense>(idx, d, a);
+      EntryReader<kDense> rd;
+      rd.init(it, a);
+      if (it_count > 0) ok = mbar_wait_warp(&s.q_free, (it_count - 1) & 1, abort_flag);
+      if (!ok) break;
+      if (lane == 0) {
+        mbar_arrive_expect_tx(&s.q_full, it.tile1 ? 65536u : 32768u);
+        tma_load_3d(s.q[0][0], &tmap_q, &s.q_full, 0, it.h, it.m0 * kBlock);
+        tma_load_3d(s.q[0][1], &tmap_q, &s.q_full, 64, it.h, it.m0 * kBlock);
+        if (it.tile1) {
+          tma_load_3d(s.q[1][0], &tmap_q, &s.q_full, 0, it.h, it.m1 * kBlock);
+          tma_load_3d(s.q[1][1], &tmap_q, &s.q_full, 64, it.h, it.m1 * kBlock);
+        }
+      }
+      for (int e = 0; e < it.n_entries; ++e, ++ecount) {
+        const uint32_t ent = rd.get(e, it.n_entries, lane);
+        const int J = static_cast<int>(ent & kColMask);
+        const int st = ecount & 1;
+        const uint32_t use = ecount >> 1;
+        if (use > 0) ok = mbar_wait_warp(&s.k_empty[st], (use - 1) & 1, abort_flag);
+        if (!ok) break;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(&s.k_full[st], 32768u);
+          tma_load_3d(s.k[st][0], &tmap_k, &s.k_full[st], 0, it.kvh, J * kBlock);
+          tma_load_3d(s.k[st][1], &tmap_k, &s.k_full[st], 64, it.kvh, J * kBlock);
+        }
+        if (use > 0) ok = mbar_wait_warp(&s.v_empty[st], (use - 1) & 1, abort_flag);
+        if (!ok) break;
+        if (lane == 0) {
+          mbar_arrive_expect_tx(&s.v_full[st], 32768u);
+          tma_load_3d(s.v[st][0], &tmap_v, &s.v_full[st], 0, it.kvh, J * kBlock);
+          tma_load_3d(s.v[st][1], &tmap_v, &s.v_full[st], 64, it.kvh, J * kBlock);
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // =============================================================== MMA issuer
+    constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 128, false, false);
+    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, false, true);
+    uint32_t ecount_base = 0;
+    uint32_t pv_count[2] = {0, 0};  // P-ready phases consumed per tile
+    int it_count = 0;
+    bool ok = true;
+
+    auto issue_qk = [&](int t, uint32_t ecount, bool last_use, bool last_of_item) {
+      const int st = ecount & 1;
+      ok = ok && mbar_wait_warp(&s.k_full[st], (ecount >> 1) & 1, abort_flag);
+      if (!ok) return;
+      tc_fence_after_sync();
+      if (lane == 0) {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t ad = umma_desc_sw128(smem_u32(s.q[t][kk >> 2]) + (kk & 3) * 32, 0, 1024);
+          const uint64_t bd = umma_desc_sw128(smem_u32(s.k[st][kk >> 2]) + (kk & 3) * 32, 0, 1024);
+          umma_ss(tm + t * 128, ad, bd, idesc_qk, kk > 0);
+        }
+        umma_commit(&s.s_full[t]);
+        if (last_use) umma_commit(&s.k_empty[st]);
+        if (last_of_item) umma_commit(&s.q_free);
+      }
+      __syncwarp();
+    };
+    auto issue_pv = [&](int t, uint32_t ecount, bool last_use, bool first_of_tile) {
+      const int st = ecount & 1;
+      ok = ok && mbar_wait_warp(&s.p_ready[t], pv_count[t] & 1, abort_flag);
+      ok = ok && mbar_wait_warp(&s.v_full[st], (ecount >> 1) & 1, abort_flag);
+      if (!ok) return;
+      ++pv_count[t];
+      tc_fence_after_sync();
+      if (lane == 0) {
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          // V block as the MN-major B operand: 16 keys per step = two groups of 8 key rows
+          const uint64_t bd = umma_desc_sw128(smem_u32(s.v[st][0]) + kk * 2048, 16384, 1024);
+          umma_ts(tm + 256 + t * 128, tm + t * 128 + kk * 8, bd, idesc_pv, (kk > 0 || !first_of_tile) ? 1u : 0u);
+        }
+        umma_commit(&s.o_done[t]);
+        if (last_use) umma_commit(&s.v_empty[st]);
+      }
+      __syncwarp();
+    };
+
+    for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
+      const Item it = decode_item<kDense>(idx, d, a);
+      EntryReader<kDense> rd;
+      rd.init(it, a);
+      ok = mbar_wait_warp(&s.q_full, it_count & 1, abort_flag);
+      if (!ok) break;
+      // pending step whose P*V has not been issued yet
+      bool have_prev = false;
+      int prev_t = 0;
+      uint32_t prev_ec = 0;
+      bool prev_last_use = false, prev_first = false;
+      bool seen[2] = {false, false};
+      for (int e = 0; e < it.n_entries && ok; ++e) {
+        const uint32_t ent = rd.get(e, it.n_entries, lane);
+        const bool f0 = (ent & kFlag0) != 0, f1 = (ent & kFlag1) != 0;
+        const uint32_t ec = ecount_base + e;
+        for (int t = 0; t < 2; ++t) {
+          if (!(t == 0 ? f0 : f1)) continue;
+          const bool last_use = (t == 1) || !f1;
+          // the last step of an item is the diagonal block of its last tile
+          const bool last_of_item = (e == it.n_entries - 1) && last_use;
+          if (have_prev && prev_t != t) {
+            issue_qk(t, ec, last_use, last_of_item);
+            issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
+          } else if (have_prev) {
+            issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
+            issue_qk(t, ec, last_use, last_of_item);
+          } else {
+            issue_qk(t, ec, last_use, last_of_item);
+          }
+          have_prev = true;
+          prev_t = t;
+          prev_ec = ec;
+          prev_last_use = last_use;
+          prev_first = !seen[t];
+          seen[t] = true;
+        }
+      }
+      if (have_prev && ok) issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
+      ecount_base += it.n_entries;
+    }
+  } else if (warp < 8) {
+    // =============================================================== softmax / epilogue, one row per thread
+    const int t = warp >> 2;                     // tile
+    const int r = tid & 127;                     // row within the tile
+    const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t s_addr = tm + lane_addr + t * 128;
+    const uint32_t o_addr = tm + lane_addr + 256 + t * 128;
+    uint32_t step_count = 0;  // steps of this tile so far (all items): phase of s_full / o_done
+    bool ok = true;
+    for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+      const Item it = decode_item<kDense>(idx, d, a);
+      if (t == 1 && !it.tile1) continue;
+      EntryReader<kDense> rd;
+      rd.init(it, a);
+      const int m_t = t == 0 ? it.m0 : it.m1;
+      float m_used = 0.f, l_run = 0.f;
+      bool first = true;
+      for (int e = 0; e < it.n_entries && ok; ++e) {
+        const uint32_t ent = rd.get(e, it.n_entries, lane);
+        if (!(ent & (t == 0 ? kFlag0 : kFlag1))) continue;
+        const int J = static_cast<int>(ent & kColMask);
+        ok = mbar_wait_warp(&s.s_full[t], step_count & 1, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t x[4][32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld_x32(s_addr + c * 32, x[c]);
+        tmem_ld_wait();
+        const bool diag = (J == m_t);
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float val = __uint_as_float(x[c][i]);
+            if (!diag || (c * 32 + i) <= r) mx = fmaxf(mx, val);
+          }
+        mx *= d.scale_log2;
+        if (first) {
+          m_used = mx;
+        } else if (mx > m_used + kRescaleThreshold) {
+          // rescale the accumulator in place once every earlier P*V of this tile has completed
+          ok = mbar_wait_warp(&s.o_done[t], (step_count - 1) & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const float f = ex2(m_used - mx);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint32_t ov[32];
+            tmem_ld_x32(o_addr + c * 32, ov);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
+            tmem_st_x32(o_addr + c * 32, ov);
+          }
+          l_run *= f;
+          m_used = mx;
+        }
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0 = ex2(fmaf(__uint_as_float(x[c][2 * i]), d.scale_log2, -m_used));
+            float p1 = ex2(fmaf(__uint_as_float(x[c][2 * i + 1]), d.scale_log2, -m_used));
+            if (diag) {
+              if (c * 32 + 2 * i > r) p0 = 0.f;
+              if (c * 32 + 2 * i + 1 > r) p1 = 0.f;
+            }
+            sum += p0 + p1;
+            pk[i] = pack_bf16(p0, p1);
+          }
+          tmem_st_x16(s_addr + c * 16, pk);
+        }
+        l_run += sum;
+        tmem_st_wait();
+        tc_fence_before_sync();
+        mbar_arrive(&s.p_ready[t]);
+        first = false;
+        ++step_count;
+      }
+      if (!ok) break;
+      // ---- epilogue: wait for the last P*V of this tile, normalise, store
+      ok = mbar_wait_warp(&s.o_done[t], (step_count - 1) & 1, abort_flag);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const float inv = 1.0f / l_run;
+      const size_t token = static_cast<size_t>(m_t) * kBlock + r;
+      __nv_bfloat16* orow = a.o + (token * d.hq + it.h) * kHeadDim;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t ov[32];
+        tmem_ld_x32(o_addr + c * 32, ov);
+        tmem_ld_wait();
+        uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          uint4 val;
+          val.x = pack_bf16(__uint_as_float(ov[8 * g + 0]) * inv, __uint_as_float(ov[8 * g + 1]) * inv);
+          val.y = pack_bf16(__uint_as_float(ov[8 * g + 2]) * inv, __uint_as_float(ov[8 * g + 3]) * inv);
+          val.z = pack_bf16(__uint_as_float(ov[8 * g + 4]) * inv, __uint_as_float(ov[8 * g + 5]) * inv);
+          val.w = pack_bf16(__uint_as_float(ov[8 * g + 6]) * inv, __uint_as_float(ov[8 * g + 7]) * inv);
+          dst[g] = val;
+        }
+      }
+      if (a.lse) a.lse[static_cast<size_t>(it.h) * d.n + token] = m_used * 0.6931471805599453f + logf(l_run);
+      tc_fence_before_sync();
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && s.abort_flag) atomicExch(a.status, CRISP_ERR_DEVICE_TIMEOUT);
+  if (warp == 8) tmem_dealloc(tm, 512);
+}
+
+// Union of the lists of query blocks (2u, 2u+1) of one head, with per-tile flags.  One warp per pair;
+// the two lists become bitmaps in shared memory, the union is emitted in ascending order.
+__global__ void __launch_bounds__(128)
+merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                   int32_t* __restrict__ merged, int* __restrict__ item_len, int n_pairs) {
+  extern __shared__ uint32_t bm[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
+  const int words = (d.nb + 31) / 32;
+  uint32_t* b0 = bm + static_cast<size_t>(warp) * 2 * words;
+  uint32_t* b1 = b0 + words;
+  if (u >= n_pairs) return;
+  const int m0 = 2 * u, m1 = 2 * u + 1;
+  for (int i = lane; i < 2 * words; i += 32) b0[i] = 0u;
+  __syncwarp();
+  const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
+  const int64_t s0 = rp[m0], e0 = rp[m0 + 1];
+  for (int64_t i = s0 + lane; i < e0; i += 32) {
+    const int c = col_idx[i];
+    atomicOr(&b0[c >> 5], 1u << (c & 31));
+  }
+  int64_t e1 = e0;
+  if (m1 < d.nb) {
+    e1 = rp[m1 + 1];
+    for (int64_t i = e0 + lane; i < e1; i += 32) {
+      const int c = col_idx[i];
+      atomicOr(&b1[c >> 5], 1u << (c & 31));
+    }
+  }
+  __syncwarp();
+  int32_t* out = merged + s0;
+  int written = 0;
+  for (int w0 = 0; w0 < words; w0 += 32) {
+    const int wd = w0 + lane;
+    const uint32_t x0 = wd < words ? b0[wd] : 0u, x1 = wd < words ? b1[wd] : 0u;
+    uint32_t un = x0 | x1;
+    const int c = __popc(un);
+    int incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int tmp = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += tmp;
+    }
+    int pos = written + incl - c;
+    while (un) {
+      const int b = __ffs(un) - 1;
+      un &= un - 1;
+      uint32_t ent = static_cast<uint32_t>(wd * 32 + b);
+      if ((x0 >> b) & 1u) ent |= kFlag0;
+      if ((x1 >> b) & 1u) ent |= kFlag1;
+      out[pos++] = static_cast<int32_t>(ent);
+    }
+    written += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (lane == 0) item_len[h * n_pairs + u] = written;
+}
+
+struct PrefillWs {
+  int* item_len;
+  int32_t* merged;
+};
+
+PrefillWs carve(const Dims& d, void* ws, size_t* total) {
+  PrefillWs w;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  size_t off = kWsHeader;
+  const int n_pairs = (d.nb + 1) / 2;
+  w.item_len = reinterpret_cast<int*>(base + off);
+  off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
+  w.merged = reinterpret_cast<int32_t*>(base + off);
+  off += align_up(sizeof(int32_t) * static_cast<size_t>(d.hq) * d.nb * (static_cast<size_t>(d.nb) + 1) / 2, 256);
+  *total = off;
+  return w;
+}
+
+}  // namespace
+
+size_t prefill_ws_bytes(const Dims& d) {
+  size_t total;
+  carve(d, nullptr, &total);
+  return total;
+}
+
+int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, const int64_t* row_ptr,
+                   const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream) {
+  const bool dense = (row_ptr == nullptr);
+  size_t total;
+  PrefillWs w = carve(d, ws, &total);
+  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "prefill: clear status");
+  CUtensorMap tq, tk, tv;
+  int rc = make_tmap_bf16_nhd(&tq, q, d.n, d.hq);
+  if (rc == CRISP_OK) rc = make_tmap_bf16_nhd(&tk, k, d.n, d.hkv);
+  if (rc == CRISP_OK) rc = make_tmap_bf16_nhd(&tv, v, d.n, d.hkv);
+  if (rc != CRISP_OK) return rc;
+
+  PrefillArgs a;
+  a.n_pairs = (d.nb + 1) / 2;
+  a.n_items = a.n_pairs * d.hq;
+  a.merged = w.merged;
+  a.row_ptr = row_ptr;
+  a.item_len = w.item_len;
+  a.o = static_cast<__nv_bfloat16*>(o);
+  a.lse = lse;
+  a.status = static_cast<int*>(ws);
+
+  int dev = 0, n_sm = 0;
+  CRISP_CUDA_TRY(cudaGetDevice(&dev), "prefill: device");
+  CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "prefill: SM count");
+  const int grid = a.n_items < n_sm ? a.n_items : n_sm;
+  const size_t smem = sizeof(PrefillSmem) + 1024;
+  if (dense) {
+    CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(smem)),
+                   "prefill: smem attribute");
+    prefill_kernel<true><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a);
+  } else {
+    const int words = (d.nb + 31) / 32;
+    merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
+        d, row_ptr, col_idx, w.merged, w.item_len, a.n_pairs);
+    CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(smem)),
+                   "prefill: smem attribute");
+    prefill_kernel<false><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a);
+  }
+  CRISP_CUDA_TRY(cudaGetLastError(), "prefill: launch");
+  return CRISP_OK;
+}
+
+}  // namespace crisp

@@ -1,0 +1,331 @@
+// Stage 1-3a: proxy attention of the last query block, C_struct router and block scores
+// (Algorithm 2; Eq. 2; Algorithm 3 lines 3-5).
+//
+// A_hat (128 x n per head) is never written to memory.  `proxy_partials_kernel` computes one
+// 128 x 128 tile of logits per (KV head, key tile, query head of the group) with tcgen05 MMAs into
+// TMEM and reduces it, one thread per proxy row, to four numbers per (row, tile): the tile-local max
+// and the sums of exp(logit - max) over the entries on/below the tile diagonal, above it, and on the
+// anchor keys.  Entries on/below the diagonal of key tile J belong to the diagonal band of block
+// offset N_b-1-J, entries above it to offset N_b-2-J, so these sums are all the later steps need.
+// The small kernels after it merge the partials: per-row global max and sum (`row_stats`,
+// `row_final`), per-tile masses across rows with warp-shuffle reductions (`tile_sums`) and the final
+// p_v, p_s, C_struct and routing label (`finalize`).  All reductions run in a fixed order.
+#include "common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace crisp {
+using namespace sm100;
+
+namespace {
+
+constexpr int kChunk = 16;  // key tiles per CTA in the merge kernels
+
+struct RoutePtrs {
+  float* pm;       // [hq][nb][128] tile-local max of the scaled logits (base-2 units)
+  float* plo;      // [hq][nb][128] sum of 2^(x - max) over entries with key offset <= row
+  float* pup;      // [hq][nb][128] ... over entries with key offset > row
+  float* panc;     // [hq][slots][128] ... over anchor keys of the tile
+  float* cm;       // [hq][n_chunks][128] chunk max
+  float* cl;       // [hq][n_chunks][128] chunk sum relative to chunk max
+  float* row_m;    // [hq][128] global row max
+  float* row_invl; // [hq][128] 1 / global row sum
+  float* slo;      // [hq][nb] mass (over rows) on/below the tile diagonal
+  float* sup;      // [hq][nb] mass above the tile diagonal
+  int n_chunks;
+};
+
+struct ProxySmem {
+  alignas(1024) uint8_t k[2][16384];      // key tile, two 64-column halves, 128-byte swizzle
+  alignas(1024) uint8_t q[2][2][16384];   // [buffer][half] proxy queries of one head
+  uint64_t bar_k;
+  uint64_t bar_q[2];
+  uint64_t bar_s_full[2];
+  uint64_t bar_s_free[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(160)
+proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
+                      const Dims d, const RoutePtrs w, int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  ProxySmem& s = *reinterpret_cast<ProxySmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int J = blockIdx.x, kvh = blockIdx.y;
+  const int G = d.group;
+
+  if (tid == 0) {
+    s.abort_flag = 0;
+    mbar_init(&s.bar_k, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&s.bar_q[b], 1);
+      mbar_init(&s.bar_s_full[b], 1);
+      mbar_init(&s.bar_s_free[b], 4);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(&s.tmem_base, 256);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tm = s.tmem_base;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      // ---- producer + MMA issuer
+      prefetch_tmap(&tmap_q);
+      prefetch_tmap(&tmap_k);
+      mbar_arrive_expect_tx(&s.bar_k, 32768);
+      tma_load_3d(s.k[0], &tmap_k, &s.bar_k, 0, kvh, J * kBlock);
+      tma_load_3d(s.k[1], &tmap_k, &s.bar_k, 64, kvh, J * kBlock);
+      for (int g = 0; g < G && g < 2; ++g) {
+        mbar_arrive_expect_tx(&s.bar_q[g], 32768);
+        tma_load_3d(s.q[g][0], &tmap_q, &s.bar_q[g], 0, kvh * G + g, d.n - kBlock);
+        tma_load_3d(s.q[g][1], &tmap_q, &s.bar_q[g], 64, kvh * G + g, d.n - kBlock);
+      }
+      bool ok = mbar_wait(&s.bar_k, 0, &s.abort_flag);
+      constexpr uint32_t idesc = umma_idesc_bf16(128, 128, false, false);
+      for (int g = 0; g < G && ok; ++g) {
+        const int b = g & 1, use = g >> 1;
+        ok = ok && mbar_wait(&s.bar_q[b], use & 1, &s.abort_flag);
+        if (use > 0) ok = ok && mbar_wait(&s.bar_s_free[b], (use - 1) & 1, &s.abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t ad = umma_desc_sw128(smem_u32(s.q[b][kk >> 2]) + (kk & 3) * 32, 0, 1024);
+          const uint64_t bd = umma_desc_sw128(smem_u32(s.k[kk >> 2]) + (kk & 3) * 32, 0, 1024);
+          umma_ss(tm + b * 128, ad, bd, idesc, kk > 0);
+        }
+        umma_commit(&s.bar_s_full[b]);
+        if (g + 2 < G) {
+          // the query buffer is free again once this MMA has read it
+          ok = ok && mbar_wait(&s.bar_s_full[b], use & 1, &s.abort_flag);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&s.bar_q[b], 32768);
+          tma_load_3d(s.q[b][0], &tmap_q, &s.bar_q[b], 0, kvh * G + g + 2, d.n - kBlock);
+          tma_load_3d(s.q[b][1], &tmap_q, &s.bar_q[b], 64, kvh * G + g + 2, d.n - kBlock);
+        }
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---- one thread per proxy row
+    const int i = tid;
+    const bool last_tile = (J == d.nb - 1);
+    const int js = min(max(d.w_sink - J * kBlock, 0), kBlock);            // anchor: local key < js
+    const int jl = min(max(d.n - d.w_local - J * kBlock, 0), kBlock);     // anchor: local key >= jl
+    const bool has_slot = (J < d.n_sink_tiles) || (J >= d.first_local_tile);
+    const int slot = (J < d.n_sink_tiles) ? J : d.n_sink_tiles + (J - d.first_local_tile);
+    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+    for (int g = 0; g < G; ++g) {
+      const int b = g & 1, use = g >> 1;
+      if (!mbar_wait(&s.bar_s_full[b], use & 1, &s.abort_flag)) break;
+      tc_fence_after_sync();
+      uint32_t r[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld_x32(tm + lane_addr + b * 128 + c * 32, r[c]);
+      tmem_ld_wait();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s.bar_s_free[b]);
+
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int t = 0; t < 32; ++t) {
+          const int j = c * 32 + t;
+          const float x = __uint_as_float(r[c][t]) * d.scale_log2;
+          r[c][t] = __float_as_uint(x);
+          if (!last_tile || j <= i) mx = fmaxf(mx, x);
+        }
+      float lo = 0.f, up = 0.f, anc = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int t = 0; t < 32; ++t) {
+          const int j = c * 32 + t;
+          const float e = ex2(__uint_as_float(r[c][t]) - mx);
+          const bool below = (j <= i);
+          const bool valid = below || !last_tile;
+          lo += below ? e : 0.f;
+          up += (valid && !below) ? e : 0.f;
+          anc += (valid && (j < js || j >= jl)) ? e : 0.f;
+        }
+      const int h = kvh * G + g;
+      const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
+      w.pm[off] = mx;
+      w.plo[off] = lo;
+      w.pup[off] = up;
+      if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
+  if (warp == 4) tmem_dealloc(tm, 256);
+}
+
+// Per (head, chunk of tiles): running max and sum of every proxy row over the chunk's tiles.
+__global__ void __launch_bounds__(128) row_stats_kernel(const Dims d, const RoutePtrs w) {
+  const int h = blockIdx.y, chunk = blockIdx.x, i = threadIdx.x;
+  const int j0 = chunk * kChunk, j1 = min(j0 + kChunk, d.nb);
+  float M = -INFINITY, L = 0.f;
+  const size_t base = static_cast<size_t>(h) * d.nb * kBlock + i;
+#pragma unroll 4
+  for (int J = j0; J < j1; ++J) {
+    const size_t off = base + static_cast<size_t>(J) * kBlock;
+    const float m = w.pm[off];
+    const float sum = w.plo[off] + w.pup[off];
+    const float nm = fmaxf(M, m);
+    L = L * ex2(M - nm) + sum * ex2(m - nm);
+    M = nm;
+  }
+  const size_t o = (static_cast<size_t>(h) * w.n_chunks + chunk) * kBlock + i;
+  w.cm[o] = M;
+  w.cl[o] = L;
+}
+
+// Per head: merge the chunk statistics into the global row max and 1 / row sum.
+__global__ void __launch_bounds__(128) row_final_kernel(const Dims d, const RoutePtrs w) {
+  const int h = blockIdx.x, i = threadIdx.x;
+  float M = -INFINITY, L = 0.f;
+  for (int c = 0; c < w.n_chunks; ++c) {
+    const size_t o = (static_cast<size_t>(h) * w.n_chunks + c) * kBlock + i;
+    const float m = w.cm[o], l = w.cl[o];
+    const float nm = fmaxf(M, m);
+    L = L * ex2(M - nm) + l * ex2(m - nm);
+    M = nm;
+  }
+  w.row_m[h * kBlock + i] = M;
+  w.row_invl[h * kBlock + i] = 1.0f / L;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Per (head, chunk): one warp per key tile sums the normalised masses over the 128 proxy rows.
+__global__ void __launch_bounds__(128) tile_sums_kernel(const Dims d, const RoutePtrs w, float* __restrict__ p_v) {
+  const int h = blockIdx.y, chunk = blockIdx.x;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  float M[4], invl[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    M[r] = w.row_m[h * kBlock + lane + 32 * r];
+    invl[r] = w.row_invl[h * kBlock + lane + 32 * r] * (1.0f / kBlock);
+  }
+  const int j0 = chunk * kChunk, j1 = min(j0 + kChunk, d.nb);
+  for (int J = j0 + warp; J < j1; J += 4) {
+    const size_t base = (static_cast<size_t>(h) * d.nb + J) * kBlock + lane;
+    float lo = 0.f, up = 0.f;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+      const float wgt = ex2(w.pm[base + 32 * r] - M[r]) * invl[r];
+      lo += wgt * w.plo[base + 32 * r];
+      up += wgt * w.pup[base + 32 * r];
+    }
+    lo = warp_sum(lo);
+    up = warp_sum(up);
+    if (lane == 0) {
+      w.slo[static_cast<size_t>(h) * d.nb + J] = lo;
+      w.sup[static_cast<size_t>(h) * d.nb + J] = up;
+      p_v[static_cast<size_t>(h) * d.nb + J] = lo + up;
+    }
+  }
+}
+
+// Per head: slash scores from the two triangle sums, C_struct from the anchor partials, routing label.
+__global__ void __launch_bounds__(256) finalize_kernel(const Dims d, const RoutePtrs w, float* __restrict__ p_s,
+                                                       float* __restrict__ c_struct, int32_t* __restrict__ pattern) {
+  const int h = blockIdx.x, tid = threadIdx.x;
+  const float* slo = w.slo + static_cast<size_t>(h) * d.nb;
+  const float* sup = w.sup + static_cast<size_t>(h) * d.nb;
+  for (int sidx = tid; sidx < d.nb; sidx += blockDim.x) {
+    const int jlo = d.nb - 1 - sidx, jup = d.nb - 2 - sidx;
+    p_s[static_cast<size_t>(h) * d.nb + sidx] = slo[jlo] + (jup >= 0 ? sup[jup] : 0.f);
+  }
+  __shared__ float red[4];
+  float acc = 0.f;
+  if (tid < kBlock) {
+    const float M = w.row_m[h * kBlock + tid];
+    const float invl = w.row_invl[h * kBlock + tid] * (1.0f / kBlock);
+    for (int slot = 0; slot < d.n_anchor_slots; ++slot) {
+      const int J = slot < d.n_sink_tiles ? slot : d.first_local_tile + (slot - d.n_sink_tiles);
+      const float m = w.pm[(static_cast<size_t>(h) * d.nb + J) * kBlock + tid];
+      acc += ex2(m - M) * invl * w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + tid];
+    }
+    acc = warp_sum(acc);
+    if ((tid & 31) == 0) red[tid >> 5] = acc;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const float c = (red[0] + red[1]) + (red[2] + red[3]);
+    c_struct[h] = c;
+    int pat = (c >= d.tau) ? CRISP_PATTERN_VS : CRISP_PATTERN_PE;
+    if (d.force_pattern == 1) pat = CRISP_PATTERN_VS;
+    if (d.force_pattern == 2) pat = CRISP_PATTERN_PE;
+    pattern[h] = pat;
+  }
+}
+
+RoutePtrs carve(const Dims& d, void* ws) {
+  RoutePtrs w;
+  uint8_t* p = static_cast<uint8_t*>(ws) + kWsHeader;
+  auto take = [&](size_t n_floats) {
+    float* r = reinterpret_cast<float*>(p);
+    p += align_up(n_floats * sizeof(float), 256);
+    return r;
+  };
+  w.n_chunks = (d.nb + kChunk - 1) / kChunk;
+  const size_t part = static_cast<size_t>(d.hq) * d.nb * kBlock;
+  w.pm = take(part);
+  w.plo = take(part);
+  w.pup = take(part);
+  w.panc = take(static_cast<size_t>(d.hq) * d.n_anchor_slots * kBlock);
+  w.cm = take(static_cast<size_t>(d.hq) * w.n_chunks * kBlock);
+  w.cl = take(static_cast<size_t>(d.hq) * w.n_chunks * kBlock);
+  w.row_m = take(static_cast<size_t>(d.hq) * kBlock);
+  w.row_invl = take(static_cast<size_t>(d.hq) * kBlock);
+  w.slo = take(static_cast<size_t>(d.hq) * d.nb);
+  w.sup = take(static_cast<size_t>(d.hq) * d.nb);
+  return w;
+}
+
+}  // namespace
+
+size_t route_ws_bytes(const Dims& d) {
+  RoutePtrs w = carve(d, nullptr);
+  return reinterpret_cast<size_t>(w.sup) + align_up(static_cast<size_t>(d.hq) * d.nb * sizeof(float), 256);
+}
+
+int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c_struct, int32_t* pattern,
+                 float* p_v, float* p_s, cudaStream_t stream) {
+  RoutePtrs w = carve(d, ws);
+  int* status = static_cast<int*>(ws);
+  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "route: clear status");
+  CUtensorMap tq, tk;
+  int rc = make_tmap_bf16_nhd(&tq, q, d.n, d.hq);
+  if (rc != CRISP_OK) return rc;
+  rc = make_tmap_bf16_nhd(&tk, k, d.n, d.hkv);
+  if (rc != CRISP_OK) return rc;
+  const size_t smem = sizeof(ProxySmem) + 1024;
+  CRISP_CUDA_TRY(cudaFuncSetAttribute(proxy_partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(smem)),
+                 "route: smem attribute");
+  proxy_partials_kernel<<<dim3(d.nb, d.hkv), 160, smem, stream>>>(tq, tk, d, w, status);
+  row_stats_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w);
+  row_final_kernel<<<d.hq, 128, 0, stream>>>(d, w);
+  tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v);
+  finalize_kernel<<<d.hq, 256, 0, stream>>>(d, w, p_s, c_struct, pattern);
+  CRISP_CUDA_TRY(cudaGetLastError(), "route: launch");
+  return CRISP_OK;
+}
+
+}  // namespace crisp

@@ -1,0 +1,641 @@
+// Stage 3b-3c: block selection and expansion into per-query-block key-block lists.
+//
+//   VS heads  (Algorithm 3 lines 6-12 / Eq. 3-4, or Algorithm 6 when selector == 1):
+//     `select_vs_kernel`, one CTA per (head, direction), keeps p_d in shared memory, computes the
+//     noise floor, the budget k_d and the top-k_d set (ties to the lower index) as a bitmap.
+//   PE heads  (Algorithm 4): block means of Q and K (`pool_kernel`), pooled logits (`pe_logits_kernel`),
+//     causal row softmax normalised by the total (`pe_normalise_kernel`), then the gamma cut WITHOUT a
+//     sort: a three-level radix histogram over the fp32 bit patterns (`pe_hist_kernel`,
+//     `pe_cut_kernel`) finds the value at the cut and how many entries tied with it are taken
+//     (ties in row-major order).
+//   Expansion + compaction: per (head, query block) a bitmap over key blocks is formed from the
+//     vertical bitmap, the shifted slash bitmap and the forced blocks {0, m}; popcounts give the row
+//     lengths (`count_vs_kernel`), one scan gives row_ptr (`scan_rows_kernel`), a second pass writes the
+//     ascending column lists (`fill_kernel`).  No atomics touch the lists, so they are reproducible.
+#include "common.cuh"
+
+namespace crisp {
+
+namespace {
+
+constexpr int kL0Bins = 2048, kL1Bins = 2048, kL2Bins = 512;  // key bits 30..20, 19..9, 8..0
+constexpr int kHistStride = kL0Bins + kL1Bins + kL2Bins;
+
+struct CutState {      // per head, device memory
+  unsigned int prefix; // key bits fixed so far
+  unsigned int cutkey; // final: fp32 bit pattern of the value at the cut
+  double mass_above;   // mass of entries strictly above the current prefix range
+  long long take;      // number of entries equal to cutkey that are selected
+};
+
+struct SelectPtrs {
+  uint32_t* selv;   // [hq][words] vertical bitmap
+  uint32_t* selsr;  // [hq][words + 2] reversed slash bitmap: bit x = S_s contains N_b-1-x
+  float* kbar;      // [hkv][nb][128]
+  float* qbar;      // [hq][nb][128]
+  float* amat;      // [hq][nb][nb] pooled map (row m uses columns 0..m)
+  unsigned int* hcount;  // [hq][kHistStride]
+  double* hmass;         // [hq][kHistStride]
+  CutState* cut;         // [hq]
+  int* n_gt;        // [hq][nb]
+  int* n_eq;        // [hq][nb]
+  int* flags;       // [hq][nb] bit0: a[m][0] > cut, bit1: == cut, bit2: a[m][m] > cut, bit3: == cut
+  int* take;        // [hq][nb] ties of row m that are selected
+  int* counts;      // [hq][nb] row lengths
+  int words;
+};
+
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_sum_i(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Block-wide sum in a fixed order (warp shuffles, then the warp totals in warp order).
+template <typename T>
+__device__ T block_sum(T v, T* scratch /* >= 32 */) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  __syncthreads();
+  if (lane == 0) scratch[warp] = v;
+  __syncthreads();
+  T total = 0;
+  for (int wdx = 0; wdx < nw; ++wdx) total += scratch[wdx];
+  return total;
+}
+
+// ------------------------------------------------------------------------------------------------
+// VS heads: budget and top-k per direction
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+select_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const float* __restrict__ p_v,
+                 const float* __restrict__ p_s, const SelectPtrs w) {
+  extern __shared__ uint8_t sm_raw[];
+  const int nb = d.nb;
+  double* sorted = reinterpret_cast<double*>(sm_raw);  // [nb] values in descending order (gamma rule)
+  float* p = reinterpret_cast<float*>(sorted + nb);    // [nb]
+  int* ranks = reinterpret_cast<int*>(p + nb);         // [nb]
+  uint8_t* sel = reinterpret_cast<uint8_t*>(ranks + nb);  // [nb]
+  __shared__ float fscratch[32];
+  __shared__ int iscratch[32];
+  __shared__ int s_k;
+  const int h = blockIdx.x, dir = blockIdx.y, tid = threadIdx.x;
+  uint32_t* out = dir == 0 ? w.selv + static_cast<size_t>(h) * w.words
+                           : w.selsr + static_cast<size_t>(h) * (w.words + 2);
+  const int out_words = dir == 0 ? w.words : w.words + 2;
+  if (pattern[h] != CRISP_PATTERN_VS) {
+    for (int i = tid; i < out_words; i += blockDim.x) out[i] = 0u;
+    return;
+  }
+  const float* src = (dir == 0 ? p_v : p_s) + static_cast<size_t>(h) * nb;
+  for (int i = tid; i < nb; i += blockDim.x) p[i] = src[i];
+  __syncthreads();
+
+  bool need_rank = false;
+  int k = nb;
+  float thr = -1.f;  // N_b <= 2: every block is kept
+  if (nb > 2) {
+    // noise floor over the blocks that are not always retained (Eq. 3), as the sum of the middle blocks
+    float part = 0.f;
+    for (int i = 1 + tid; i < nb - 1; i += blockDim.x) part += p[i];
+    const float r = block_sum<float>(part, fscratch);
+    const float mu = r / static_cast<float>(nb - 2);
+    thr = d.alpha * mu;
+    if (d.selector == 0) {
+      int c = 0;
+      for (int i = tid; i < nb; i += blockDim.x) c += (p[i] > thr) ? 1 : 0;
+      const int cnt = block_sum<int>(c, iscratch);
+      if (cnt >= d.k_min) {
+        k = cnt;  // the top-cnt set is exactly {p > thr} (Eq. 4)
+      } else {
+        k = min(d.k_min, nb);
+        need_rank = true;
+      }
+    } else {
+      need_rank = true;
+    }
+  }
+  if (!need_rank) {
+    for (int i = tid; i < nb; i += blockDim.x) sel[i] = p[i] > thr;
+  } else {
+    // rank in the stable descending order: larger value first, then lower index
+    for (int e = tid; e < nb; e += blockDim.x) {
+      const float pe = p[e];
+      int rank = 0;
+      for (int j = 0; j < nb; ++j) {
+        const float pj = p[j];
+        rank += (pj > pe || (pj == pe && j < e)) ? 1 : 0;
+      }
+      ranks[e] = rank;
+      sorted[rank] = static_cast<double>(pe);
+    }
+    __syncthreads();
+    if (d.selector == 1) {
+      // smallest k whose running sum (in sorted order) reaches gamma (Algorithm 6); all if never
+      if (tid == 0) {
+        double c = 0.0;
+        int found = nb;
+        for (int i = 0; i < nb; ++i) {
+          c += sorted[i];
+          if (c >= static_cast<double>(d.gamma)) {
+            found = i + 1;
+            break;
+          }
+        }
+        s_k = min(max(found, d.k_min), nb);
+      }
+      __syncthreads();
+      k = s_k;
+    }
+    for (int e = tid; e < nb; e += blockDim.x) sel[e] = ranks[e] < k;
+  }
+  __syncthreads();
+  // bitmaps: vertical as is; slash reversed (bit x <-> offset nb-1-x) and zero padded
+  for (int wd = tid; wd < out_words; wd += blockDim.x) {
+    uint32_t bits = 0;
+    for (int b = 0; b < 32; ++b) {
+      const int x = wd * 32 + b;
+      if (x < nb) {
+        const int e = dir == 0 ? x : nb - 1 - x;
+        bits |= static_cast<uint32_t>(sel[e] != 0) << b;
+      }
+    }
+    out[wd] = bits;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// PE heads: pooling, pooled logits, row softmax
+// ------------------------------------------------------------------------------------------------
+// Block means of one [128 tokens, 128 dims] tile per CTA.  x is [n, heads, 128] bf16.
+__global__ void __launch_bounds__(128)
+pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is_query,
+            const int32_t* __restrict__ pattern, float* __restrict__ out) {
+  const int J = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+  if (is_query) {
+    if (pattern[h] != CRISP_PATTERN_PE) return;
+  } else {
+    bool any = false;
+    for (int g = 0; g < d.group; ++g) any = any || (pattern[h * d.group + g] == CRISP_PATTERN_PE);
+    if (!any) return;
+  }
+  const int pair = tid & 63, half = tid >> 6;
+  const __nv_bfloat162* base = reinterpret_cast<const __nv_bfloat162*>(
+      x + (static_cast<size_t>(J) * kBlock + half * 64) * heads * kHeadDim + static_cast<size_t>(h) * kHeadDim);
+  float a0 = 0.f, a1 = 0.f;
+#pragma unroll 8
+  for (int t = 0; t < 64; ++t) {
+    const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
+    a0 += v.x;
+    a1 += v.y;
+  }
+  __shared__ float2 other[64];
+  if (half == 1) other[pair] = make_float2(a0, a1);
+  __syncthreads();
+  if (half == 0) {
+    float* o = out + (static_cast<size_t>(h) * d.nb + J) * kHeadDim;
+    o[2 * pair] = (a0 + other[pair].x) * (1.0f / kBlock);
+    o[2 * pair + 1] = (a1 + other[pair].y) * (1.0f / kBlock);
+  }
+}
+
+// Pooled logits Z[m, J] = qbar[m] . kbar[J] * scale_log2 for a 64 x 64 tile (fp32 FMA, no tensor
+// cores: the selection compares these values, so they keep full fp32 precision).
+__global__ void __launch_bounds__(256)
+pe_logits_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  const int jt = blockIdx.x, mt = blockIdx.y, h = blockIdx.z;
+  if (jt > mt || pattern[h] != CRISP_PATTERN_PE) return;
+  __shared__ float qs[64][33];
+  __shared__ float ks[64][33];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const float* qb = w.qbar + (static_cast<size_t>(h) * d.nb + mt * 64) * kHeadDim;
+  const float* kb = w.kbar + (static_cast<size_t>(h / d.group) * d.nb + jt * 64) * kHeadDim;
+  const int mrows = min(64, d.nb - mt * 64), jrows = min(64, d.nb - jt * 64);
+  float acc[4][4] = {};
+  for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
+    for (int idx = tid; idx < 64 * 32; idx += 256) {
+      const int r = idx >> 5, c = idx & 31;
+      qs[r][c] = r < mrows ? qb[static_cast<size_t>(r) * kHeadDim + c0 + c] : 0.f;
+      ks[r][c] = r < jrows ? kb[static_cast<size_t>(r) * kHeadDim + c0 + c] : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 8
+    for (int c = 0; c < 32; ++c) {
+      float a[4], b[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) a[i] = qs[ty + 16 * i][c];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = ks[tx + 16 * j][c];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+  float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int m = mt * 64 + ty + 16 * i;
+    if (m >= d.nb) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int J = jt * 64 + tx + 16 * j;
+      if (J <= m) am[static_cast<size_t>(m) * d.nb + J] = acc[i][j] * d.scale_log2;
+    }
+  }
+}
+
+// Row softmax over J <= m, divided by N_b (= the total of the pooled map).
+__global__ void __launch_bounds__(256)
+pe_normalise_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  const int m = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
+  float* row = w.amat + (static_cast<size_t>(h) * d.nb + m) * d.nb;
+  __shared__ float red[32];
+  __shared__ float fscratch[32];
+  float mx = -INFINITY;
+  for (int J = tid; J <= m; J += 256) mx = fmaxf(mx, row[J]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if ((tid & 31) == 0) red[tid >> 5] = mx;
+  __syncthreads();
+  mx = red[0];
+  for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
+  float sum = 0.f;
+  for (int J = tid; J <= m; J += 256) sum += exp2f(row[J] - mx);
+  const float total = block_sum<float>(sum, fscratch);
+  const float inv = 1.0f / (total * static_cast<float>(d.nb));
+  for (int J = tid; J <= m; J += 256) row[J] = exp2f(row[J] - mx) * inv;
+}
+
+// ------------------------------------------------------------------------------------------------
+// PE heads: gamma cut by radix histogram over the value bits
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ bool key_in_level(unsigned int key, unsigned int prefix, int level, int* bin) {
+  if (level == 0) {
+    *bin = static_cast<int>(key >> 20);
+    return true;
+  }
+  if (level == 1) {
+    *bin = static_cast<int>((key >> 9) & 2047u);
+    return (key >> 20) == (prefix >> 20);
+  }
+  *bin = static_cast<int>(key & 511u);
+  return (key >> 9) == (prefix >> 9);
+}
+
+__global__ void __launch_bounds__(256)
+pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int level) {
+  const int h = blockIdx.y, tid = threadIdx.x;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
+  __shared__ unsigned int cnt[2048];
+  __shared__ double mass[2048];
+  const int nbins = level == 2 ? kL2Bins : 2048;
+  for (int i = tid; i < nbins; i += 256) {
+    cnt[i] = 0u;
+    mass[i] = 0.0;
+  }
+  __syncthreads();
+  const unsigned int prefix = w.cut[h].prefix;
+  const float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
+  for (int m = blockIdx.x; m < d.nb; m += gridDim.x) {
+    const float* row = am + static_cast<size_t>(m) * d.nb;
+    for (int J = tid; J <= m; J += 256) {
+      const float v = row[J];
+      int bin;
+      if (key_in_level(__float_as_uint(v), prefix, level, &bin)) {
+        atomicAdd(&cnt[bin], 1u);
+        atomicAdd(&mass[bin], static_cast<double>(v));
+      }
+    }
+  }
+  __syncthreads();
+  const int off = level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins);
+  unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + off;
+  double* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
+  for (int i = tid; i < nbins; i += 256)
+    if (cnt[i]) {
+      atomicAdd(&gc[i], cnt[i]);
+      atomicAdd(&gm[i], mass[i]);
+    }
+}
+
+// One thread per head walks the bins from the largest values down until the mass reaches gamma.
+__global__ void pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int level) {
+  const int h = blockIdx.x * blockDim.x + threadIdx.x;
+  if (h >= d.hq || pattern[h] != CRISP_PATTERN_PE) return;
+  const int nbins = level == 2 ? kL2Bins : 2048;
+  const int off = level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins);
+  const unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + off;
+  const double* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
+  CutState c = w.cut[h];
+  if (level == 0) {
+    c.prefix = 0u;
+    c.mass_above = 0.0;
+    c.cutkey = 0u;
+    c.take = 0x7fffffffffffffffLL;
+  } else if (c.take == -1) {  // gamma was never reached at an earlier level: everything is kept
+    return;
+  }
+  const double gamma = static_cast<double>(d.gamma);
+  int found = -1;
+  double above = c.mass_above;
+  for (int b = nbins - 1; b >= 0; --b) {
+    if (gc[b] == 0u) continue;
+    if (above + gm[b] >= gamma) {
+      found = b;
+      break;
+    }
+    above += gm[b];
+  }
+  if (found < 0) {
+    // the target exceeds the total mass (gamma >= 1 or rounding): keep every causal entry
+    c.cutkey = 0u;
+    c.take = -1;
+    c.mass_above = above;
+    w.cut[h] = c;
+    return;
+  }
+  c.mass_above = above;
+  const int shift = level == 0 ? 20 : (level == 1 ? 9 : 0);
+  c.prefix |= static_cast<unsigned int>(found) << shift;
+  if (level == 2) {
+    c.cutkey = c.prefix;
+    const double v = static_cast<double>(__uint_as_float(c.cutkey));
+    long long t = static_cast<long long>(ceil((gamma - above) / v));
+    // guard the division against rounding: t is the smallest count whose mass reaches gamma
+    while (t > 1 && above + static_cast<double>(t - 1) * v >= gamma) --t;
+    while (above + static_cast<double>(t) * v < gamma && t < static_cast<long long>(gc[found])) ++t;
+    if (t < 1) t = 1;
+    if (t > static_cast<long long>(gc[found])) t = static_cast<long long>(gc[found]);
+    c.take = t;
+  }
+  w.cut[h] = c;
+}
+
+// Per row of a PE head: how many entries lie above the cut, how many tie with it, and how the two
+// forced entries (column 0 and the diagonal) compare.
+__global__ void __launch_bounds__(256)
+pe_row_stats_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  const int m = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
+  __shared__ int iscratch[32];
+  const CutState c = w.cut[h];
+  const float* row = w.amat + (static_cast<size_t>(h) * d.nb + m) * d.nb;
+  int gt = 0, eq = 0;
+  for (int J = tid; J <= m; J += 256) {
+    const unsigned int key = __float_as_uint(row[J]);
+    gt += key > c.cutkey;
+    eq += key == c.cutkey;
+  }
+  gt = block_sum<int>(gt, iscratch);
+  eq = block_sum<int>(eq, iscratch);
+  if (tid == 0) {
+    const unsigned int k0 = __float_as_uint(row[0]), km = __float_as_uint(row[m]);
+    const int f = (k0 > c.cutkey ? 1 : 0) | (k0 == c.cutkey ? 2 : 0) | (km > c.cutkey ? 4 : 0) |
+                  (km == c.cutkey ? 8 : 0);
+    const size_t o = static_cast<size_t>(h) * d.nb + m;
+    w.n_gt[o] = gt;
+    w.n_eq[o] = eq;
+    w.flags[o] = f;
+  }
+}
+
+// Per PE head: ties are taken in row-major order, so row m takes clamp(T - (ties in rows < m), 0, ties_m).
+__global__ void __launch_bounds__(1024)
+pe_take_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  const int h = blockIdx.x, tid = threadIdx.x;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
+  __shared__ long long seg_tot[1024];
+  const int seg = (d.nb + 1023) / 1024;
+  const int b0 = min(tid * seg, d.nb), b1 = min(b0 + seg, d.nb);
+  const size_t base = static_cast<size_t>(h) * d.nb;
+  long long local = 0;
+  for (int m = b0; m < b1; ++m) local += w.n_eq[base + m];
+  seg_tot[tid] = local;
+  __syncthreads();
+  long long before = 0;
+  for (int t = 0; t < tid; ++t) before += seg_tot[t];
+  const CutState c = w.cut[h];
+  for (int m = b0; m < b1; ++m) {
+    const int eq = w.n_eq[base + m];
+    int take;
+    if (c.take < 0) {
+      take = eq;
+    } else {
+      const long long left = c.take - before;
+      take = static_cast<int>(left <= 0 ? 0 : (left >= eq ? eq : left));
+    }
+    before += eq;
+    const int f = w.flags[base + m];
+    const bool sel0 = (f & 1) || ((f & 2) && take >= 1);
+    const bool selm = (f & 4) || ((f & 8) && take >= eq);
+    int count = w.n_gt[base + m] + take + (sel0 ? 0 : 1);
+    if (m > 0) count += selm ? 0 : 1;
+    w.take[base + m] = take;
+    w.counts[base + m] = count;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Expansion of VS heads, row lengths, scan, fill
+// ------------------------------------------------------------------------------------------------
+// Word `wd` (key blocks 32*wd .. 32*wd+31) of the keep bitmap of query block m of a VS head.
+__device__ __forceinline__ uint32_t vs_keep_word(const uint32_t* __restrict__ selv, const uint32_t* __restrict__ selsr,
+                                                 int nb, int m, int wd) {
+  const int sh = nb - 1 - m;              // slash offset s = m - J  <->  reversed bit J + sh
+  const int pos0 = wd * 32 + sh, pos1 = pos0 + 1;
+  const uint32_t a = __funnelshift_r(selsr[pos0 >> 5], selsr[(pos0 >> 5) + 1], pos0 & 31);
+  const uint32_t b = __funnelshift_r(selsr[pos1 >> 5], selsr[(pos1 >> 5) + 1], pos1 & 31);
+  uint32_t bits = selv[wd] | a | b;
+  if (wd == 0) bits |= 1u;
+  if (wd == (m >> 5)) {
+    bits |= 1u << (m & 31);
+    const int top = m & 31;
+    bits &= (top == 31) ? 0xffffffffu : ((2u << top) - 1u);
+  }
+  return bits;
+}
+
+__global__ void __launch_bounds__(256)
+count_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = blockIdx.x * 8 + warp, h = blockIdx.y;
+  if (m >= d.nb || pattern[h] != CRISP_PATTERN_VS) return;
+  const uint32_t* selv = w.selv + static_cast<size_t>(h) * w.words;
+  const uint32_t* selsr = w.selsr + static_cast<size_t>(h) * (w.words + 2);
+  int c = 0;
+  for (int wd = lane; wd <= (m >> 5); wd += 32) c += __popc(vs_keep_word(selv, selsr, d.nb, m, wd));
+  c = warp_sum_i(c);
+  if (lane == 0) w.counts[static_cast<size_t>(h) * d.nb + m] = c;
+}
+
+// Exclusive scan of all row lengths (head-major) into row_ptr; total into *nnz_needed; capacity check.
+__global__ void __launch_bounds__(1024)
+scan_rows_kernel(const Dims d, const SelectPtrs w, int64_t* __restrict__ row_ptr, int64_t capacity,
+                 int64_t* __restrict__ nnz_needed, int* status) {
+  const int tid = threadIdx.x;
+  const long long total_rows = static_cast<long long>(d.hq) * d.nb;
+  const long long seg = (total_rows + 1023) / 1024;
+  const long long b0 = min(tid * seg, total_rows), b1 = min(b0 + seg, total_rows);
+  __shared__ long long seg_tot[1024];
+  long long local = 0;
+  for (long long r = b0; r < b1; ++r) local += w.counts[r];
+  seg_tot[tid] = local;
+  __syncthreads();
+  long long run = 0;
+  for (int t = 0; t < tid; ++t) run += seg_tot[t];
+  for (long long r = b0; r < b1; ++r) {
+    const int h = static_cast<int>(r / d.nb), m = static_cast<int>(r % d.nb);
+    row_ptr[static_cast<size_t>(h) * (d.nb + 1) + m] = run;
+    run += w.counts[r];
+    if (m == d.nb - 1) row_ptr[static_cast<size_t>(h) * (d.nb + 1) + d.nb] = run;
+  }
+  if (tid == 1023) {
+    *nnz_needed = run;
+    if (run > capacity) atomicExch(status, CRISP_ERR_CAPACITY);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w,
+            const int64_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx, int64_t capacity,
+            const int64_t* __restrict__ nnz_needed) {
+  if (*nnz_needed > capacity) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m = blockIdx.x * 8 + warp, h = blockIdx.y;
+  if (m >= d.nb) return;
+  int32_t* out = col_idx + row_ptr[static_cast<size_t>(h) * (d.nb + 1) + m];
+  int written = 0;
+  if (pattern[h] == CRISP_PATTERN_VS) {
+    const uint32_t* selv = w.selv + static_cast<size_t>(h) * w.words;
+    const uint32_t* selsr = w.selsr + static_cast<size_t>(h) * (w.words + 2);
+    const int nwords = (m >> 5) + 1;
+    for (int w0 = 0; w0 < nwords; w0 += 32) {
+      const int wd = w0 + lane;
+      uint32_t bits = wd < nwords ? vs_keep_word(selv, selsr, d.nb, m, wd) : 0u;
+      const int c = __popc(bits);
+      int incl = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+      }
+      int pos = written + incl - c;
+      while (bits) {
+        const int b = __ffs(bits) - 1;
+        bits &= bits - 1;
+        out[pos++] = wd * 32 + b;
+      }
+      written += __shfl_sync(0xffffffffu, incl, 31);
+    }
+  } else {
+    const CutState c = w.cut[h];
+    const float* row = w.amat + (static_cast<size_t>(h) * d.nb + m) * d.nb;
+    const int take = w.take[static_cast<size_t>(h) * d.nb + m];
+    int ties_seen = 0;
+    for (int J0 = 0; J0 <= m; J0 += 32) {
+      const int J = J0 + lane;
+      bool gt = false, eq = false;
+      if (J <= m) {
+        const unsigned int key = __float_as_uint(row[J]);
+        gt = key > c.cutkey;
+        eq = key == c.cutkey;
+      }
+      const uint32_t eqmask = __ballot_sync(0xffffffffu, eq);
+      const int my_tie = ties_seen + __popc(eqmask & ((1u << lane) - 1u));
+      const bool keep = (J <= m) && (gt || (eq && my_tie < take) || J == 0 || J == m);
+      const uint32_t keepmask = __ballot_sync(0xffffffffu, keep);
+      if (keep) out[written + __popc(keepmask & ((1u << lane) - 1u))] = J;
+      written += __popc(keepmask);
+      ties_seen += __popc(eqmask);
+    }
+  }
+}
+
+SelectPtrs carve(const Dims& d, void* ws, size_t* total) {
+  SelectPtrs w;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  size_t off = kWsHeader;
+  auto take = [&](size_t bytes) {
+    void* r = base + off;
+    off += align_up(bytes, 256);
+    return r;
+  };
+  w.words = (d.nb + 31) / 32;
+  w.selv = static_cast<uint32_t*>(take(sizeof(uint32_t) * d.hq * w.words));
+  w.selsr = static_cast<uint32_t*>(take(sizeof(uint32_t) * d.hq * (w.words + 2)));
+  w.kbar = static_cast<float*>(take(sizeof(float) * d.hkv * d.nb * kHeadDim));
+  w.qbar = static_cast<float*>(take(sizeof(float) * static_cast<size_t>(d.hq) * d.nb * kHeadDim));
+  w.amat = static_cast<float*>(take(sizeof(float) * static_cast<size_t>(d.hq) * d.nb * d.nb));
+  w.hcount = static_cast<unsigned int*>(take(sizeof(unsigned int) * d.hq * kHistStride));
+  w.hmass = static_cast<double*>(take(sizeof(double) * d.hq * kHistStride));
+  w.cut = static_cast<CutState*>(take(sizeof(CutState) * d.hq));
+  w.n_gt = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  w.n_eq = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  w.flags = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  w.take = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  w.counts = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  *total = off;
+  return w;
+}
+
+}  // namespace
+
+size_t select_ws_bytes(const Dims& d) {
+  size_t total;
+  carve(d, nullptr, &total);
+  return total;
+}
+
+int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pattern, const float* p_v,
+                  const float* p_s, void* ws, int64_t* row_ptr, int32_t* col_idx, int64_t capacity,
+                  int64_t* nnz_needed, cudaStream_t stream) {
+  if (d.nb > 8192) return CRISP_ERR_UNSUPPORTED;
+  size_t total;
+  SelectPtrs w = carve(d, ws, &total);
+  int* status = static_cast<int*>(ws);
+  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "select: clear status");
+  CRISP_CUDA_TRY(cudaMemsetAsync(w.hcount, 0, sizeof(unsigned int) * d.hq * kHistStride, stream), "select: clear");
+  CRISP_CUDA_TRY(cudaMemsetAsync(w.hmass, 0, sizeof(double) * d.hq * kHistStride, stream), "select: clear");
+
+  // VS heads
+  const size_t vs_smem = (sizeof(double) + sizeof(float) + sizeof(int) + 1) * static_cast<size_t>(d.nb) + 16;
+  CRISP_CUDA_TRY(cudaFuncSetAttribute(select_vs_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(vs_smem)),
+                 "select: smem attribute");
+  select_vs_kernel<<<dim3(d.hq, 2), 1024, vs_smem, stream>>>(d, pattern, p_v, p_s, w);
+
+  // PE heads (every kernel returns at once for heads routed to VS)
+  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
+  const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
+  pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, kb, d.hkv, 0, pattern, w.kbar);
+  pool_kernel<<<dim3(d.nb, d.hq), 128, 0, stream>>>(d, qb, d.hq, 1, pattern, w.qbar);
+  const int nt = (d.nb + 63) / 64;
+  pe_logits_kernel<<<dim3(nt, nt, d.hq), 256, 0, stream>>>(d, pattern, w);
+  pe_normalise_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w);
+  const int hist_ctas = d.nb < 128 ? d.nb : 128;
+  for (int level = 0; level < 3; ++level) {
+    pe_hist_kernel<<<dim3(hist_ctas, d.hq), 256, 0, stream>>>(d, pattern, w, level);
+    pe_cut_kernel<<<(d.hq + 31) / 32, 32, 0, stream>>>(d, pattern, w, level);
+  }
+  pe_row_stats_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w);
+  pe_take_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w);
+
+  // expansion + compaction
+  count_vs_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w);
+  scan_rows_kernel<<<1, 1024, 0, stream>>>(d, w, row_ptr, capacity, nnz_needed, status);
+  fill_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w, row_ptr, col_idx, capacity,
+                                                              nnz_needed);
+  CRISP_CUDA_TRY(cudaGetLastError(), "select: launch");
+  return CRISP_OK;
+}
+
+}  // namespace crisp

@@ -1,0 +1,192 @@
+"""GPU parity: every stage of the CUDA path against the fp64 oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import crisp_oracle as orc
+from workloads import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _pu():
+    from tests import parity_utils
+    return parity_utils
+
+
+def _full_check(w, p=None, per_head=6, dense=True, seed=0):
+    pu = _pu()
+    p = p or pu.params_of(w)
+    q, k, v = synth.make_qkv(w, device="cuda")
+    g = pu.run_gpu(p, q, k, v, dense=dense)
+    qc, kc, vc = q.cpu(), k.cpu(), v.cpu()
+    res = orc.layer_pipeline(qc.float().numpy(), kc.float().numpy(), **pu.oracle_kwargs(p))
+    n_lab = pu.check_route(g, res, p)
+    n_exc = pu.check_lists(g, res, p)
+    nb = w.n_blocks
+    samples = pu.sample_blocks(nb, w.n_q_heads, per_head, seed)
+    rel, mab = pu.check_attention(g, qc, kc, vc, p, samples)
+    if dense:
+        pu.check_attention(g, qc, kc, vc, p, samples, key="o_dense", dense=True)
+    print(f"{w.name}: excused labels {n_lab}, excused blocks {n_exc}, nnz {g['nnz']}, "
+          f"rel-L2 {rel:.2e}, max-abs {mab:.2e}")
+    return g, res
+
+
+def test_tiny_config_full():
+    w = synth.CONFIGS["Tiny"]
+    g, res = _full_check(w, per_head=32)
+    assert [int(x) for x in g["pattern"]] == [1, 1, 0, 0]
+
+
+def test_tiny_every_block_dense_and_sparse():
+    pu = _pu()
+    w = synth.tiny(n=2048)
+    p = pu.params_of(w)
+    q, k, v = synth.make_qkv(w, device="cuda")
+    g = pu.run_gpu(p, q, k, v, dense=True)
+    samples = [(h, m) for h in range(4) for m in range(w.n_blocks)]
+    pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples)
+    pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples, key="o_dense", dense=True)
+
+
+@pytest.mark.parametrize("n", [256, 384, 640, 1152])
+def test_small_and_odd_block_counts(n):
+    """N_b = 2 (everything kept), odd N_b (a lone last tile), N_b not a multiple of the tile pair."""
+    pu = _pu()
+    w = synth.tiny(n=n).with_(k_min_blocks=2)
+    _full_check(w, per_head=16)
+
+
+def test_paper_window_sizes_and_identity():
+    """w_sink = w_local = 128: C_struct equals p_v[0] + p_v[N_b-1] (Section 4.3)."""
+    pu = _pu()
+    w = synth.tiny(n=4096).with_(sink_tokens=128, local_tokens=128, tau=0.2)
+    g, _ = _full_check(w, per_head=4, dense=False)
+    np.testing.assert_allclose(g["c_struct"], g["p_v"][:, 0] + g["p_v"][:, -1], rtol=1e-5)
+    np.testing.assert_allclose(g["p_v"].sum(1), 1.0, rtol=1e-5)
+    np.testing.assert_allclose(g["p_s"].sum(1), 1.0, rtol=1e-5)
+
+
+def test_wide_anchor_windows():
+    pu = _pu()
+    w = synth.tiny(n=2048).with_(sink_tokens=300, local_tokens=200)
+    _full_check(w, per_head=4, dense=False)
+
+
+@pytest.mark.parametrize("alpha", [0.5, 2.0])
+def test_alpha_sweep_and_monotonicity(alpha):
+    pu = _pu()
+    w = synth.tiny(n=4096)
+    g1, _ = _full_check(w, per_head=4, dense=False)
+    g2, _ = _full_check(w.with_(alpha=alpha), per_head=4, dense=False)
+    a, b = (g2, g1) if alpha > 1 else (g1, g2)    # a: larger alpha
+    for h in (0, 1):
+        for m in range(w.n_blocks):
+            assert set(pu.gpu_cols(a, h, m).tolist()) <= set(pu.gpu_cols(b, h, m).tolist())
+
+
+def test_gamma_selector():
+    pu = _pu()
+    w = synth.tiny(n=4096)
+    _full_check(w, p=pu.params_of(w, selector=1), per_head=4, dense=False)
+    _full_check(w, p=pu.params_of(w, selector=1, gamma=0.5), per_head=4, dense=False)
+
+
+@pytest.mark.parametrize("force", [1, 2])
+def test_forced_patterns(force):
+    pu = _pu()
+    w = synth.tiny(n=2048)
+    g, _ = _full_check(w, p=pu.params_of(w, force_pattern=force), per_head=4, dense=False)
+    assert (g["pattern"] == (1 if force == 1 else 0)).all()
+
+
+def test_k_min_fill_and_large_alpha():
+    pu = _pu()
+    w = synth.tiny(n=4096).with_(alpha=1e6, k_min_blocks=5)
+    g, res = _full_check(w, per_head=4, dense=False)
+    assert res[0]["raw_v"] < 5 and res[0]["k_v"] == 5
+
+
+def test_gqa_llama_shape_reduced():
+    """32k generator recipe at a reduced length: 8 query / 2 KV heads, slash lines present."""
+    w = synth.llama_shaped("L8k", 8192, 32).with_(n_q_heads=8, n_kv_heads=2,
+                                                  head_classes=("conc", "diffuse") * 4)
+    _full_check(w, per_head=6)
+
+
+def test_qwen_shape_reduced():
+    """GQA group of 7, sink scale 16 (p_v[0] ~ 1: the noise floor must not cancel)."""
+    w = synth.qwen_shaped("Q8k", 8192).with_(n_q_heads=14, n_kv_heads=2,
+                                             head_classes=("sink", "slash", "diffuse", "diffuse") * 3
+                                             + ("sink", "slash"))
+    _full_check(w, per_head=4)
+
+
+def test_iid_inputs_custom_scale():
+    pu = _pu()
+    import paper_2609_01925_b200 as crisp
+    n, hq, hkv = 1024, 4, 2
+    q, k, v = synth.random_qkv(n, hq, hkv, seed=3, device="cuda")
+    p = crisp.make_params(n, hq, hkv, sink_tokens=4, tau=0.05, softmax_scale=0.05, k_min_blocks=2)
+    g = pu.run_gpu(p, q, k, v, dense=True)
+    res = orc.layer_pipeline(q.cpu().float().numpy(), k.cpu().float().numpy(), **pu.oracle_kwargs(p))
+    pu.check_route(g, res, p)
+    pu.check_lists(g, res, p)
+    samples = [(h, m) for h in range(hq) for m in range(n // 128)]
+    pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples)
+    pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples, key="o_dense", dense=True)
+
+
+def test_zero_inputs_massive_ties():
+    """Q = K = 0: every proxy row is uniform and every pooled row is flat (ties everywhere)."""
+    pu = _pu()
+    import paper_2609_01925_b200 as crisp
+    n, hq, hkv = 1024, 2, 1
+    q = torch.zeros(n, hq, 128, dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros(n, hkv, 128, dtype=torch.bfloat16, device="cuda")
+    v = synth.random_qkv(n, hq, hkv, seed=5, device="cuda")[2]
+    for force in (1, 2):
+        p = crisp.make_params(n, hq, hkv, sink_tokens=4, force_pattern=force, gamma=0.5, k_min_blocks=2)
+        g = pu.run_gpu(p, q, k, v)
+        nb = n // 128
+        for h in range(hq):
+            for m in range(nb):
+                c = pu.gpu_cols(g, h, m)
+                assert c[0] == 0 and c[-1] == m and np.all(np.diff(c) > 0)
+        if force == 2:
+            # rows in order until half of the mass: rows 0..3 of 8 (mass 4/8), later rows only {0, m}
+            for m in range(4):
+                assert len(pu.gpu_cols(g, 0, m)) == m + 1
+            assert len(pu.gpu_cols(g, 0, 7)) == 2
+        samples = [(h, m) for h in range(hq) for m in range(nb)]
+        pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples)
+
+
+def test_capacity_overflow_is_reported():
+    pu = _pu()
+    import paper_2609_01925_b200 as crisp
+    from paper_2609_01925_b200 import binding as B
+    w = synth.tiny(n=2048)
+    p = pu.params_of(w)
+    q, k, v = synth.make_qkv(w, device="cuda")
+    layer = crisp.CrispLayer(p, capacity=10)
+    layer.col_idx.fill_(-7)
+    layer.route(q, k)
+    layer.select(q, k)
+    rc = B.crisp_poll_device_status(layer.select_ws)
+    assert rc == B.ERR_CAPACITY
+    assert int(layer.nnz.item()) > 10
+    assert (layer.col_idx == -7).all()
+    assert B.crisp_poll_device_status(layer.select_ws) == B.OK   # cleared by the poll
+
+
+def test_results_are_reproducible():
+    pu = _pu()
+    w = synth.tiny(n=2048)
+    p = pu.params_of(w)
+    q, k, v = synth.make_qkv(w, device="cuda")
+    a = pu.run_gpu(p, q, k, v)
+    b = pu.run_gpu(p, q, k, v)
+    for key in ("c_struct", "p_v", "p_s", "row_ptr", "col_idx", "o"):
+        assert np.array_equal(a[key], b[key]), key
