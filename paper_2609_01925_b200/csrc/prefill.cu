@@ -306,14 +306,19 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             if (!diag || (c * 32 + i) <= r) mx = fmaxf(mx, val);
           }
         mx *= d.scale_log2;
+        // The rescale decision is taken per warp (the TMEM accesses below are warp-collective):
+        // if any row of the warp outgrew its reference maximum by more than the threshold, every row
+        // of the warp moves to its own current maximum.
+        const bool grow = !first && __any_sync(0xffffffffu, mx > m_used + kRescaleThreshold);
         if (first) {
           m_used = mx;
-        } else if (mx > m_used + kRescaleThreshold) {
+        } else if (grow) {
           // rescale the accumulator in place once every earlier P*V of this tile has completed
           ok = mbar_wait_warp(&s.o_done[t], (step_count - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
-          const float f = ex2(m_used - mx);
+          const float m_new = fmaxf(m_used, mx);
+          const float f = ex2(m_used - m_new);
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t ov[32];
@@ -324,7 +329,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
             tmem_st_x32(o_addr + c * 32, ov);
           }
           l_run *= f;
-          m_used = mx;
+          m_used = m_new;
         }
         float sum = 0.f;
 #pragma unroll

@@ -38,12 +38,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  `abort_flag` (shared memory) lets one role's timeout end every other
-// role's waits quickly.  Returns false when it gave up.
-constexpr uint32_t kMaxPolls = 1u << 22;
+// role's waits quickly.  Gives up after kWaitLimitNs of wall time (every legitimate wait in these
+// kernels lasts microseconds).  Returns false when it gave up.
+constexpr unsigned long long kWaitLimitNs = 400ull * 1000ull * 1000ull;
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kMaxPolls; ++i) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_timer_ns();
+  for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 63u && *abort_flag) return false;
+    if (*abort_flag) return false;
+    if (global_timer_ns() - t0 > kWaitLimitNs) break;
   }
   *abort_flag = 1;
   return false;

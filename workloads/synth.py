@@ -169,7 +169,7 @@ _ST_KNOISE, _ST_QNOISE, _ST_V, _ST_COLS = 0, 1, 2, 3
 
 def planted_columns(w: Workload, kv_head: int) -> List[int]:
     """Token positions of the planted vertical columns of one KV head (in [B, n-B))."""
-    if w.n_columns == 0:
+    if w.n_columns == 0 or w.seq_len <= 2 * BLOCK:
         return []
     idx = torch.arange(w.n_columns, dtype=torch.int64) + kv_head * 1_000_003
     z = hash64(w.seed, _ST_COLS, idx)
