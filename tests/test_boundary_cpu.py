@@ -1,0 +1,123 @@
+"""Host-side checks that need no GPU: the library loads, exports every declared symbol, validates
+its arguments and sizes its workspaces.  No compute call is made."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2609_01925_b200 as crisp
+from paper_2609_01925_b200 import binding as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = B.load()
+    header = open(os.path.join(ROOT, "include", "crisp.h")).read()
+    declared = set(re.findall(r"\b(crisp_[a-z_]+)\s*\(", header))
+    declared -= {"crisp_params", "crisp_status"}
+    assert declared == set(B.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_version_and_status_strings():
+    assert crisp.crisp_version() >= 100
+    assert B.status_string(B.OK) == "ok"
+    for code in (B.ERR_INVALID_ARG, B.ERR_UNSUPPORTED, B.ERR_WORKSPACE, B.ERR_CAPACITY, B.ERR_CUDA,
+                 B.ERR_DEVICE_TIMEOUT):
+        assert B.status_string(code) not in ("ok", "unknown status")
+    assert B.status_string(12345) == "unknown status"
+
+
+def test_params_struct_matches_header():
+    assert ctypes.sizeof(B.CrispParams) == 15 * 4
+    header = open(os.path.join(ROOT, "include", "crisp.h")).read()
+    body = header[header.index("typedef struct crisp_params"):header.index("} crisp_params;")]
+    fields = re.findall(r"^\s*(?:int32_t|float)\s+(\w+);", body, flags=re.M)
+    assert fields == [f[0] for f in B.CrispParams._fields_]
+
+
+def test_workspace_sizes_grow_with_the_problem():
+    small = B.crisp_workspace_bytes(crisp.make_params(4096, 4, 1))
+    big = B.crisp_workspace_bytes(crisp.make_params(32768, 32, 8))
+    assert all(s > 0 for s in small) and all(b > s for s, b in zip(small, big))
+    # 512k: everything must fit comfortably in 180 GB
+    huge = B.crisp_workspace_bytes(crisp.make_params(524288, 32, 8))
+    assert sum(huge) < 8 << 30
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(seq_len=4096 + 64), B.ERR_UNSUPPORTED),        # ragged n
+    (dict(seq_len=128), B.ERR_UNSUPPORTED),              # fewer than two blocks
+    (dict(head_dim=64), B.ERR_UNSUPPORTED),
+    (dict(block=64), B.ERR_UNSUPPORTED),
+    (dict(n_q_heads=6, n_kv_heads=4), B.ERR_INVALID_ARG),
+    (dict(n_q_heads=34, n_kv_heads=2), B.ERR_UNSUPPORTED),   # group of 17
+    (dict(sink_tokens=0), B.ERR_INVALID_ARG),
+    (dict(local_tokens=10 ** 7), B.ERR_INVALID_ARG),
+    (dict(k_min_blocks=-1), B.ERR_INVALID_ARG),
+    (dict(selector=2), B.ERR_INVALID_ARG),
+    (dict(force_pattern=3), B.ERR_INVALID_ARG),
+    (dict(alpha=-1.0), B.ERR_INVALID_ARG),
+    (dict(gamma=0.0), B.ERR_INVALID_ARG),
+    (dict(tau=float("nan")), B.ERR_INVALID_ARG),
+    (dict(softmax_scale=-0.5), B.ERR_INVALID_ARG),
+])
+def test_invalid_parameters_are_rejected(kw, code):
+    base = dict(seq_len=4096, n_q_heads=4, n_kv_heads=1)
+    base.update(kw)
+    n, hq, hkv = base.pop("seq_len"), base.pop("n_q_heads"), base.pop("n_kv_heads")
+    p = crisp.make_params(n, hq, hkv, **base)
+    with pytest.raises(crisp.CrispError) as e:
+        B.crisp_workspace_bytes(p)
+    assert e.value.status == code
+
+
+def test_abi_guard_and_null_pointers():
+    lib = B.load()
+    p = crisp.make_params(4096, 4, 1)
+    p.struct_size = 8
+    assert lib.crisp_workspace_bytes(ctypes.byref(p), None, None, None) == B.ERR_INVALID_ARG
+    assert lib.crisp_workspace_bytes(None, None, None, None) == B.ERR_INVALID_ARG
+    p = crisp.make_params(4096, 4, 1)
+    assert lib.crisp_workspace_bytes(ctypes.byref(p), None, None, None) == B.OK
+    # null data pointers are caught before anything is launched (no GPU needed)
+    assert lib.crisp_route(ctypes.byref(p), None, None, None, 0, None, None, None, None, None) == B.ERR_INVALID_ARG
+    assert lib.crisp_select(ctypes.byref(p), None, None, None, None, None, None, 0, None, None, 0, None,
+                            None) == B.ERR_INVALID_ARG
+    assert lib.crisp_sparse_prefill(ctypes.byref(p), None, None, None, None, None, None, 0, None, None,
+                                    None) == B.ERR_INVALID_ARG
+    assert lib.crisp_dense_prefill(ctypes.byref(p), None, None, None, None, 0, None, None, None) == B.ERR_INVALID_ARG
+    assert lib.crisp_poll_device_status(None, None) == B.ERR_INVALID_ARG
+
+
+def test_misaligned_and_short_workspace_are_rejected():
+    lib = B.load()
+    p = crisp.make_params(4096, 4, 1)
+    fake = ctypes.c_void_p(0x1000)          # never dereferenced: validation fails first
+    odd = ctypes.c_void_p(0x1004)
+    assert lib.crisp_route(ctypes.byref(p), fake, fake, fake, 16, fake, fake, fake, fake, None) == B.ERR_WORKSPACE
+    assert lib.crisp_route(ctypes.byref(p), fake, fake, odd, 1 << 30, fake, fake, fake, fake, None) == B.ERR_WORKSPACE
+    assert lib.crisp_route(ctypes.byref(p), odd, fake, fake, 1 << 30, fake, fake, fake, fake, None) == B.ERR_INVALID_ARG
+    assert lib.crisp_dense_prefill(ctypes.byref(p), fake, fake, fake, fake, 8, fake, None, None) == B.ERR_WORKSPACE
+    assert lib.crisp_select(ctypes.byref(p), fake, fake, fake, fake, fake, fake, 1 << 30, fake, None, 5, fake,
+                            None) == B.ERR_INVALID_ARG   # capacity > 0 without col_idx
+
+
+def test_layer_refuses_to_run_without_cuda():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("CUDA present")
+    with pytest.raises(RuntimeError):
+        crisp.CrispLayer(crisp.make_params(4096, 4, 1))
+
+
+def test_product_package_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2609_01925_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in text.lower().replace("no cpu or pytorch fallback", ""), f
