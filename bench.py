@@ -31,8 +31,8 @@ import torch
 from workloads import synth
 
 FLOP_PER_BLOCK = 4 * 128 ** 3          # QK^T + PV of one 128 x 128 x 128 block pair
-# kernels launched per step: route 5, select 16, sparse prefill 2 (merge + attention)
-LAUNCHES_ROUTE, LAUNCHES_SELECT, LAUNCHES_PREFILL = 5, 16, 2
+# kernels launched per step: route 5, select 16, sparse prefill 4 (merge, 2 x schedule, attention)
+LAUNCHES_ROUTE, LAUNCHES_SELECT, LAUNCHES_PREFILL = 5, 16, 4
 
 
 def load_peaks():

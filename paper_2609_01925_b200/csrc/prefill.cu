@@ -31,6 +31,7 @@ struct PrefillArgs {
   const int32_t* merged;   // per item: union list, entry = key block | flags (sparse only)
   const int64_t* row_ptr;  // [hq][nb+1]
   const int* item_len;     // [hq][n_pairs] number of union entries (sparse only)
+  const int* order;        // [n_items] item ids sorted by decreasing cost (sparse only)
   __nv_bfloat16* o;        // [n][hq][128]
   float* lse;              // [hq][n] or null
   int* status;
@@ -57,8 +58,9 @@ struct Item {
 };
 
 template <bool kDense>
-__device__ __forceinline__ Item decode_item(int idx, const Dims& d, const PrefillArgs& a) {
+__device__ __forceinline__ Item decode_item(int pos, const Dims& d, const PrefillArgs& a) {
   Item it;
+  const int idx = kDense ? pos : a.order[pos];
   it.h = idx % d.hq;
   const int u = a.n_pairs - 1 - idx / d.hq;  // long rows first
   it.kvh = it.h / d.group;
@@ -101,6 +103,72 @@ struct EntryReader {
   }
 };
 
+template <int N>
+__device__ __forceinline__ void reg_alloc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void reg_dealloc() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// Lane 0 polls; the outcome is broadcast so the warp stays converged.
+__device__ __forceinline__ bool mbar_wait_lane0(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
+  int ok = 1;
+  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+
+// Maximum of one row of raw logits; on the diagonal block only keys j <= r are visible.
+template <bool kDiag>
+__device__ __forceinline__ float row_max(const uint32_t (&x)[4][32], int r) {
+  float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+      float a0 = __uint_as_float(x[c][i]), a1 = __uint_as_float(x[c][i + 1]);
+      float a2 = __uint_as_float(x[c][i + 2]), a3 = __uint_as_float(x[c][i + 3]);
+      if (kDiag) {
+        const int j = c * 32 + i;
+        if (j > r) a0 = -INFINITY;
+        if (j + 1 > r) a1 = -INFINITY;
+        if (j + 2 > r) a2 = -INFINITY;
+        if (j + 3 > r) a3 = -INFINITY;
+      }
+      m0 = fmaxf(m0, a0);
+      m1 = fmaxf(m1, a1);
+      m2 = fmaxf(m2, a2);
+      m3 = fmaxf(m3, a3);
+    }
+  return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+}
+
+// P = 2^(x * scale - m) as bf16 into TMEM (two keys per 32-bit column); returns the fp32 row sum.
+template <bool kDiag>
+__device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int r, float scale_log2, float m_used,
+                                                uint32_t s_addr) {
+  float sum0 = 0.f, sum1 = 0.f;
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      float p0 = ex2(fmaf(__uint_as_float(x[c][2 * i]), scale_log2, -m_used));
+      float p1 = ex2(fmaf(__uint_as_float(x[c][2 * i + 1]), scale_log2, -m_used));
+      if (kDiag) {
+        if (c * 32 + 2 * i > r) p0 = 0.f;
+        if (c * 32 + 2 * i + 1 > r) p1 = 0.f;
+      }
+      sum0 += p0;
+      sum1 += p1;
+      pk[i] = pack_bf16(p0, p1);
+    }
+    tmem_st_x16(s_addr + c * 16, pk);
+  }
+  return sum0 + sum1;
+}
+
 template <bool kDense>
 __global__ void __launch_bounds__(384, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -134,8 +202,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   const uint32_t tm = s.tmem_base;
   volatile int* abort_flag = &s.abort_flag;
 
+  // Register budget: the two softmax warpgroups hold a full 128-column row of S per thread; the third
+  // warpgroup (producer, issuer, two idle warps) needs very few registers and gives the rest away.
+  // (each role changes its own budget at the top of its branch)
   if (warp == 8) {
     // =============================================================== TMA producer
+    reg_dealloc<56>();
     if (lane == 0) {
       prefetch_tmap(&tmap_q);
       prefetch_tmap(&tmap_k);
@@ -148,7 +220,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const Item it = decode_item<kDense>(idx, d, a);
       EntryReader<kDense> rd;
       rd.init(it, a);
-      if (it_count > 0) ok = mbar_wait_warp(&s.q_free, (it_count - 1) & 1, abort_flag);
+      if (it_count > 0) ok = mbar_wait_lane0(&s.q_free, (it_count - 1) & 1, abort_flag, lane);
       if (!ok) break;
       if (lane == 0) {
         mbar_arrive_expect_tx(&s.q_full, it.tile1 ? 65536u : 32768u);
@@ -164,14 +236,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const int J = static_cast<int>(ent & kColMask);
         const int st = ecount & 1;
         const uint32_t use = ecount >> 1;
-        if (use > 0) ok = mbar_wait_warp(&s.k_empty[st], (use - 1) & 1, abort_flag);
+        if (use > 0) ok = mbar_wait_lane0(&s.k_empty[st], (use - 1) & 1, abort_flag, lane);
         if (!ok) break;
         if (lane == 0) {
           mbar_arrive_expect_tx(&s.k_full[st], 32768u);
           tma_load_3d(s.k[st][0], &tmap_k, &s.k_full[st], 0, it.kvh, J * kBlock);
           tma_load_3d(s.k[st][1], &tmap_k, &s.k_full[st], 64, it.kvh, J * kBlock);
         }
-        if (use > 0) ok = mbar_wait_warp(&s.v_empty[st], (use - 1) & 1, abort_flag);
+        if (use > 0) ok = mbar_wait_lane0(&s.v_empty[st], (use - 1) & 1, abort_flag, lane);
         if (!ok) break;
         if (lane == 0) {
           mbar_arrive_expect_tx(&s.v_full[st], 32768u);
@@ -182,6 +254,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
   } else if (warp == 9) {
     // =============================================================== MMA issuer
+    reg_dealloc<56>();
     constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 128, false, false);
     constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, false, true);
     uint32_t ecount_base = 0;
@@ -191,7 +264,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 
     auto issue_qk = [&](int t, uint32_t ecount, bool last_use, bool last_of_item) {
       const int st = ecount & 1;
-      ok = ok && mbar_wait_warp(&s.k_full[st], (ecount >> 1) & 1, abort_flag);
+      ok = ok && mbar_wait_lane0(&s.k_full[st], (ecount >> 1) & 1, abort_flag, lane);
       if (!ok) return;
       tc_fence_after_sync();
       if (lane == 0) {
@@ -209,8 +282,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     };
     auto issue_pv = [&](int t, uint32_t ecount, bool last_use, bool first_of_tile) {
       const int st = ecount & 1;
-      ok = ok && mbar_wait_warp(&s.p_ready[t], pv_count[t] & 1, abort_flag);
-      ok = ok && mbar_wait_warp(&s.v_full[st], (ecount >> 1) & 1, abort_flag);
+      ok = ok && mbar_wait_lane0(&s.p_ready[t], pv_count[t] & 1, abort_flag, lane);
+      ok = ok && mbar_wait_lane0(&s.v_full[st], (ecount >> 1) & 1, abort_flag, lane);
       if (!ok) return;
       ++pv_count[t];
       tc_fence_after_sync();
@@ -231,7 +304,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const Item it = decode_item<kDense>(idx, d, a);
       EntryReader<kDense> rd;
       rd.init(it, a);
-      ok = mbar_wait_warp(&s.q_full, it_count & 1, abort_flag);
+      ok = mbar_wait_lane0(&s.q_full, it_count & 1, abort_flag, lane);
       if (!ok) break;
       // pending step whose P*V has not been issued yet
       bool have_prev = false;
@@ -270,6 +343,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
   } else if (warp < 8) {
     // =============================================================== softmax / epilogue, one row per thread
+    reg_alloc<216>();
     const int t = warp >> 2;                     // tile
     const int r = tid & 127;                     // row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -297,14 +371,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         for (int c = 0; c < 4; ++c) tmem_ld_x32(s_addr + c * 32, x[c]);
         tmem_ld_wait();
         const bool diag = (J == m_t);
-        float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float val = __uint_as_float(x[c][i]);
-            if (!diag || (c * 32 + i) <= r) mx = fmaxf(mx, val);
-          }
+        float mx;
+        if (diag) {
+          mx = row_max<true>(x, r);
+        } else {
+          mx = row_max<false>(x, r);
+        }
         mx *= d.scale_log2;
         // The rescale decision is taken per warp (the TMEM accesses below are warp-collective):
         // if any row of the warp outgrew its reference maximum by more than the threshold, every row
@@ -331,22 +403,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           l_run *= f;
           m_used = m_new;
         }
-        float sum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float p0 = ex2(fmaf(__uint_as_float(x[c][2 * i]), d.scale_log2, -m_used));
-            float p1 = ex2(fmaf(__uint_as_float(x[c][2 * i + 1]), d.scale_log2, -m_used));
-            if (diag) {
-              if (c * 32 + 2 * i > r) p0 = 0.f;
-              if (c * 32 + 2 * i + 1 > r) p1 = 0.f;
-            }
-            sum += p0 + p1;
-            pk[i] = pack_bf16(p0, p1);
-          }
-          tmem_st_x16(s_addr + c * 16, pk);
+        float sum;
+        if (diag) {
+          sum = exp_pack_store<true>(x, r, d.scale_log2, m_used, s_addr);
+        } else {
+          sum = exp_pack_store<false>(x, r, d.scale_log2, m_used, s_addr);
         }
         l_run += sum;
         tmem_st_wait();
@@ -383,6 +444,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       tc_fence_before_sync();
     }
   }
+  else {
+    reg_dealloc<56>();  // idle warps of the third warpgroup
+  }
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0 && s.abort_flag) atomicExch(a.status, CRISP_ERR_DEVICE_TIMEOUT);
@@ -393,7 +457,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 // the two lists become bitmaps in shared memory, the union is emitted in ascending order.
 __global__ void __launch_bounds__(128)
 merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                   int32_t* __restrict__ merged, int* __restrict__ item_len, int n_pairs) {
+                   int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
+                   int n_pairs) {
   extern __shared__ uint32_t bm[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
@@ -443,11 +508,50 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
     }
     written += __shfl_sync(0xffffffffu, incl, 31);
   }
-  if (lane == 0) item_len[h * n_pairs + u] = written;
+  if (lane == 0) {
+    item_len[h * n_pairs + u] = written;
+    atomicAdd(&cost_hist[static_cast<int>(e1 - s0)], 1);  // cost = tile steps = len(m0) + len(m1)
+  }
+}
+
+// Counting sort of the items by decreasing cost, so that the round-robin assignment of items to
+// CTAs balances heads with long lists (PE) against heads with short ones (VS).
+__global__ void __launch_bounds__(1024) sched_scan_kernel(int* __restrict__ cost_hist, int n_bins) {
+  __shared__ int seg_tot[1024];
+  const int tid = threadIdx.x;
+  const int seg = (n_bins + 1023) / 1024;
+  // bins are visited from the largest cost down
+  const int b0 = min(tid * seg, n_bins), b1 = min(b0 + seg, n_bins);
+  int local = 0;
+  for (int i = b0; i < b1; ++i) local += cost_hist[n_bins - 1 - i];
+  seg_tot[tid] = local;
+  __syncthreads();
+  int run = 0;
+  for (int t = 0; t < tid; ++t) run += seg_tot[t];
+  for (int i = b0; i < b1; ++i) {
+    const int c = cost_hist[n_bins - 1 - i];
+    cost_hist[n_bins - 1 - i] = run;  // first position of this cost in the sorted order
+    run += c;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, int* __restrict__ cost_hist,
+                     int* __restrict__ order, int n_pairs) {
+  const int u = blockIdx.x * blockDim.x + threadIdx.x, h = blockIdx.y;
+  if (u >= n_pairs) return;
+  const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
+  const int m0 = 2 * u, mend = min(2 * u + 2, d.nb);
+  const int cost = static_cast<int>(rp[mend] - rp[m0]);
+  const int pos = atomicAdd(&cost_hist[cost], 1);
+  order[pos] = (n_pairs - 1 - u) * d.hq + h;
 }
 
 struct PrefillWs {
   int* item_len;
+  int* order;
+  int* cost_hist;
+  int n_bins;
   int32_t* merged;
 };
 
@@ -458,6 +562,11 @@ PrefillWs carve(const Dims& d, void* ws, size_t* total) {
   const int n_pairs = (d.nb + 1) / 2;
   w.item_len = reinterpret_cast<int*>(base + off);
   off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
+  w.order = reinterpret_cast<int*>(base + off);
+  off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
+  w.n_bins = 2 * d.nb + 2;
+  w.cost_hist = reinterpret_cast<int*>(base + off);
+  off += align_up(sizeof(int) * static_cast<size_t>(w.n_bins), 256);
   w.merged = reinterpret_cast<int32_t*>(base + off);
   off += align_up(sizeof(int32_t) * static_cast<size_t>(d.hq) * d.nb * (static_cast<size_t>(d.nb) + 1) / 2, 256);
   *total = off;
@@ -490,6 +599,7 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   a.merged = w.merged;
   a.row_ptr = row_ptr;
   a.item_len = w.item_len;
+  a.order = w.order;
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.status = static_cast<int*>(ws);
@@ -506,8 +616,12 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
     prefill_kernel<true><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a);
   } else {
     const int words = (d.nb + 31) / 32;
+    CRISP_CUDA_TRY(cudaMemsetAsync(w.cost_hist, 0, sizeof(int) * w.n_bins, stream), "prefill: clear histogram");
     merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
-        d, row_ptr, col_idx, w.merged, w.item_len, a.n_pairs);
+        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs);
+    sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins);
+    sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, 0, stream>>>(d, row_ptr, w.cost_hist,
+                                                                               w.order, a.n_pairs);
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
