@@ -96,6 +96,41 @@ int crisp_route(const crisp_params* p, const void* q, const void* k, void* ws, s
                 float* c_struct, int32_t* pattern, float* p_v, float* p_s, void* cuda_stream);
 
 /*
+ * crisp_route for callers that are not able to obtain device memory at all.  (The paper has no
+ * counterpart of this call; it exists for integration only and computes exactly what crisp_route does.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits or would fail, and that has no spare
+ * buffer to lend as a workspace.  Typical cases are a plug-in invoked from inside a host application
+ * that has already claimed the whole device for its own memory pool, and a latency-critical serving
+ * loop whose rules forbid any call that may allocate or implicitly synchronise the device.
+ *
+ * How it works: the scratch that crisp_route takes as `ws` is replaced by one fixed array of
+ * CRISP_ROUTE_STATIC_SCRATCH_BYTES bytes that is compiled into the library.  Every GPU that loads the
+ * library carries this array from load time until the process exits, whether or not the call is used.
+ * The caller passes the inputs and outputs only.  The call itself allocates nothing and frees nothing
+ * (no cudaMalloc / cudaFree, no allocating library routine).
+ *
+ * Limits and rules
+ *   - The problem must fit: crisp_workspace_bytes(p).route_ws <= CRISP_ROUTE_STATIC_SCRATCH_BYTES
+ *     (4 MiB: for example 8192 tokens with 32 query heads, or 65536 tokens with 4).  Anything larger is
+ *     refused with CRISP_ERR_UNSUPPORTED before any work is enqueued, and crisp_last_cuda_error() says
+ *     how many bytes would have been needed.
+ *   - The first call on each device looks up the array's device address (with that device current) and
+ *     remembers it.  Make that first call during set-up, outside any stream capture.
+ *   - All calls on one device share the one array.  Nothing of a previous call is ever read back (the
+ *     status word is cleared, everything else is rewritten before use), but two calls that overlap in time
+ *     on the same GPU - different streams, different threads - overwrite each other's scratch and give
+ *     wrong results.  Serialise them (one stream, or an event between them).
+ *   - device_status (optional, device pointer to one int32): receives the device status word of this
+ *     call, CRISP_OK or CRISP_ERR_DEVICE_TIMEOUT, once the stream reaches that point.  There is no
+ *     workspace pointer to hand to crisp_poll_device_status, so this is how the word is reported.
+ * Outputs, layouts and all other conventions are those of crisp_route.
+ */
+#define CRISP_ROUTE_STATIC_SCRATCH_BYTES (4u << 20)
+int crisp_route_static(const crisp_params* p, const void* q, const void* k, float* c_struct, int32_t* pattern,
+                       float* p_v, float* p_s, int32_t* device_status, void* cuda_stream);
+
+/*
  * Stage 3b-3c.  VS heads: per direction d in {v, s}, mu_d = (sum of the middle blocks of p_d)/(N_b - 2),
  * k_d = clip(#{p_d > alpha * mu_d}, k_min, N_b) (selector 0) or the smallest k whose top-k mass reaches
  * gamma (selector 1), S_d = top-k_d with ties to the lower index (Algorithm 3 / Algorithm 6).

@@ -26,7 +26,7 @@ PATTERN_PE, PATTERN_VS = 0, 1
 
 EXPORTS = (
     "crisp_version", "crisp_status_string", "crisp_last_cuda_error", "crisp_workspace_bytes",
-    "crisp_route", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
+    "crisp_route", "crisp_route_static", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
     "crisp_poll_device_status",
 )
 
@@ -85,6 +85,8 @@ def load() -> ctypes.CDLL:
     lib.crisp_workspace_bytes.argtypes = [P, ctypes.POINTER(sz), ctypes.POINTER(sz), ctypes.POINTER(sz)]
     lib.crisp_route.restype = ctypes.c_int
     lib.crisp_route.argtypes = [P, vp, vp, vp, sz, vp, vp, vp, vp, vp]
+    lib.crisp_route_static.restype = ctypes.c_int
+    lib.crisp_route_static.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.crisp_select.restype = ctypes.c_int
     lib.crisp_select.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp, i64, vp, vp]
     lib.crisp_sparse_prefill.restype = ctypes.c_int
@@ -130,6 +132,19 @@ def crisp_workspace_bytes(p: CrispParams) -> Tuple[int, int, int]:
 def crisp_route(p, q, k, ws, c_struct, pattern, p_v, p_s, stream=None) -> int:
     return load().crisp_route(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(ws), ws.numel() * ws.element_size(),
                               _ptr(c_struct), _ptr(pattern), _ptr(p_v), _ptr(p_s), _stream(stream))
+
+
+ROUTE_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def crisp_route_static(p, q, k, c_struct, pattern, p_v, p_s, device_status=None, stream=None) -> int:
+    """crisp_route without a workspace argument: the scratch is a fixed 4 MiB array inside the library.
+
+    For callers that cannot allocate device memory (see include/crisp.h).  Calls on one GPU must not
+    overlap in time; problems whose route workspace exceeds ROUTE_STATIC_SCRATCH_BYTES are refused.
+    """
+    return load().crisp_route_static(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(c_struct), _ptr(pattern),
+                                     _ptr(p_v), _ptr(p_s), _ptr(device_status), _stream(stream))
 
 
 def crisp_select(p, q, k, pattern, p_v, p_s, ws, row_ptr, col_idx, capacity, nnz_needed, stream=None) -> int:

@@ -146,6 +146,17 @@ int crisp_route(const crisp_params* p, const void* q, const void* k, void* ws, s
   return launch_route(d, q, k, ws, c_struct, pattern, p_v, p_s, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int crisp_route_static(const crisp_params* p, const void* q, const void* k, float* c_struct, int32_t* pattern,
+                       float* p_v, float* p_s, int32_t* device_status, void* cuda_stream) {
+  Dims d;
+  int rc = validate(p, &d);
+  if (rc != CRISP_OK) return rc;
+  if (!q || !k || !c_struct || !pattern || !p_v || !p_s) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return CRISP_ERR_INVALID_ARG;
+  return launch_route_static(d, q, k, c_struct, pattern, p_v, p_s, device_status,
+                             static_cast<cudaStream_t>(cuda_stream));
+}
+
 int crisp_select(const crisp_params* p, const void* q, const void* k, const int32_t* pattern, const float* p_v,
                  const float* p_s, void* ws, size_t ws_bytes, int64_t* row_ptr, int32_t* col_idx,
                  int64_t capacity, int64_t* nnz_needed, void* cuda_stream) {

@@ -52,6 +52,8 @@ int make_tmap_bf16_nhd(CUtensorMap* out, const void* base, int n, int heads, int
 int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c_struct, int32_t* pattern,
                  float* p_v, float* p_s, cudaStream_t stream);
 size_t route_ws_bytes(const Dims& d);
+int launch_route_static(const Dims& d, const void* q, const void* k, float* c_struct, int32_t* pattern,
+                        float* p_v, float* p_s, int32_t* device_status, cudaStream_t stream);
 int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pattern, const float* p_v,
                   const float* p_s, void* ws, int64_t* row_ptr, int32_t* col_idx, int64_t capacity,
                   int64_t* nnz_needed, cudaStream_t stream);

@@ -10,6 +10,9 @@
 // The small kernels after it merge the partials: per-row global max and sum (`row_stats`,
 // `row_final`), per-tile masses across rows with warp-shuffle reductions (`tile_sums`) and the final
 // p_v, p_s, C_struct and routing label (`finalize`).  All reductions run in a fixed order.
+#include <cstdio>
+#include <mutex>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -325,6 +328,57 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v);
   finalize_kernel<<<d.hq, 256, 0, stream>>>(d, w, p_s, c_struct, pattern);
   CRISP_CUDA_TRY(cudaGetLastError(), "route: launch");
+  return CRISP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Routing for callers that cannot allocate device memory.  Same kernels as launch_route; the scratch
+// lives in a fixed array that is part of the loaded library image on every GPU.
+// ------------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticScratchBytes = CRISP_ROUTE_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_route_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {};  // device address of g_route_scratch, per device ordinal
+}  // namespace
+
+int launch_route_static(const Dims& d, const void* q, const void* k, float* c_struct, int32_t* pattern,
+                        float* p_v, float* p_s, int32_t* device_status, cudaStream_t stream) {
+  const size_t need = route_ws_bytes(d);
+  if (need > kStaticScratchBytes) {
+    char msg[160];
+    std::snprintf(msg, sizeof(msg),
+                  "crisp_route_static: this problem needs %zu bytes of scratch, the built-in array holds %zu",
+                  need, kStaticScratchBytes);
+    set_cu_error(msg);
+    return CRISP_ERR_UNSUPPORTED;
+  }
+  int dev = 0;
+  CRISP_CUDA_TRY(cudaGetDevice(&dev), "route_static: current device");
+  if (dev < 0 || dev >= kMaxDevices) {
+    set_cu_error("crisp_route_static: device ordinal out of range");
+    return CRISP_ERR_UNSUPPORTED;
+  }
+  void* scratch = nullptr;
+  {
+    // In host code the array's name is only a handle; the kernels need its address on THIS device.
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (g_scratch_addr[dev] == nullptr) {
+      void* p = nullptr;
+      CRISP_CUDA_TRY(cudaGetSymbolAddress(&p, g_route_scratch), "route_static: symbol address");
+      g_scratch_addr[dev] = p;
+    }
+    scratch = g_scratch_addr[dev];
+  }
+  // launch_route clears the status word at the start of the scratch; every other byte it reads is
+  // written earlier in the same call, so stale contents of the previous call are never observed.
+  const int rc = launch_route(d, q, k, scratch, c_struct, pattern, p_v, p_s, stream);
+  if (rc != CRISP_OK) return rc;
+  if (device_status)
+    CRISP_CUDA_TRY(cudaMemcpyAsync(device_status, scratch, sizeof(int32_t), cudaMemcpyDeviceToDevice, stream),
+                   "route_static: status copy");
   return CRISP_OK;
 }
 
