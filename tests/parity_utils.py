@@ -105,6 +105,31 @@ def _ambiguous_vs(pd, p, k_d, raw):
     return amb
 
 
+def _rows_to_matrix(cols_per_row, nb):
+    m = np.zeros((nb, nb), dtype=bool)
+    for r, c in enumerate(cols_per_row):
+        m[r, c] = True
+    return m
+
+
+def gpu_matrix(g, h, nb):
+    """Boolean [N_b, N_b] matrix of the GPU lists of head h; also checks order and bounds."""
+    rp = g["row_ptr"][h]
+    cols = g["col_idx"][rp[0]:rp[nb]].astype(np.int64)
+    lens = np.diff(rp)
+    rows = np.repeat(np.arange(nb), lens)
+    assert lens.min() >= 1
+    assert np.all(cols <= rows) and np.all(cols >= 0), (h, "column out of range")
+    same_row = rows[1:] == rows[:-1]
+    assert np.all(np.diff(cols)[same_row] > 0), (h, "not ascending/unique")
+    first = rp[:-1] - rp[0]
+    last = rp[1:] - rp[0] - 1
+    assert np.all(cols[first] == 0) and np.all(cols[last] == np.arange(nb)), (h, "forced blocks missing")
+    m = np.zeros((nb, nb), dtype=bool)
+    m[rows, cols] = True
+    return m
+
+
 def check_lists(g, res, p, heads=None):
     """GPU lists vs oracle lists under the matching rule.  Returns the count of excused blocks."""
     nb = p.seq_len // p.block
@@ -112,17 +137,17 @@ def check_lists(g, res, p, heads=None):
     heads = range(len(res)) if heads is None else heads
     for h in heads:
         r = res[h]
-        if g["pattern"][h] != r["pattern"]:
+        if r is None or g["pattern"][h] != r["pattern"]:
             continue  # label excused by check_route; lists follow the other branch
         if nb <= 2:
-            lo = hi = r["cols"]
+            lo = hi = _rows_to_matrix(r["cols"], nb)
         elif r["pattern"] == orc.VS:
             amb_v = _ambiguous_vs(r["p_v"], p, r["k_v"], r["raw_v"])
             amb_s = _ambiguous_vs(r["p_s"], p, r["k_s"], r["raw_s"])
             sv = np.zeros(nb, bool); sv[r["s_v"]] = True
             ss = np.zeros(nb, bool); ss[r["s_s"]] = True
-            lo = orc.expand_vs(np.nonzero(sv & ~amb_v)[0], np.nonzero(ss & ~amb_s)[0], nb)
-            hi = orc.expand_vs(np.nonzero(sv | amb_v)[0], np.nonzero(ss | amb_s)[0], nb)
+            lo = _rows_to_matrix(orc.expand_vs(np.nonzero(sv & ~amb_v)[0], np.nonzero(ss & ~amb_s)[0], nb), nb)
+            hi = _rows_to_matrix(orc.expand_vs(np.nonzero(sv | amb_v)[0], np.nonzero(ss | amb_s)[0], nb), nb)
             excused_total += int(amb_v.sum() + amb_s.sum())
         else:
             flat = r["a_bar"] / r["a_bar"].sum()
@@ -138,16 +163,14 @@ def check_lists(g, res, p, heads=None):
                 amb.reshape(-1)[order[kstar]] = True
             if kstar >= 2 and p.gamma - cs[kstar - 2] <= MASS_BAND:
                 amb.reshape(-1)[order[kstar - 1]] = True
-            lo = orc.expand_pe(r["pe_sel"] & ~amb)
-            hi = orc.expand_pe(r["pe_sel"] | amb)
+            lo = _rows_to_matrix(orc.expand_pe(r["pe_sel"] & ~amb), nb)
+            hi = _rows_to_matrix(orc.expand_pe(r["pe_sel"] | amb), nb)
             excused_total += int(amb.sum())
-        for m in range(nb):
-            got = gpu_cols(g, h, m)
-            assert np.all(np.diff(got) > 0), (h, m, "not ascending/unique")
-            assert got[0] == 0 and got[-1] == m, (h, m, got[:4], got[-4:])
-            gs = set(got.tolist())
-            assert set(lo[m].tolist()) <= gs, (h, m, sorted(set(lo[m].tolist()) - gs)[:8])
-            assert gs <= set(hi[m].tolist()), (h, m, sorted(gs - set(hi[m].tolist()))[:8])
+        got = gpu_matrix(g, h, nb)
+        missing = lo & ~got
+        extra = got & ~hi
+        assert not missing.any(), (h, "missing", np.argwhere(missing)[:8].tolist())
+        assert not extra.any(), (h, "extra", np.argwhere(extra)[:8].tolist())
     return excused_total
 
 
