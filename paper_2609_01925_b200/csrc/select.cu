@@ -6,8 +6,8 @@
 //   PE heads  (Algorithm 4): block means of Q and K (`pool_kernel`), pooled logits (`pe_logits_kernel`),
 //     causal row softmax normalised by the total (`pe_normalise_kernel`), then the gamma cut WITHOUT a
 //     sort: a three-level radix histogram over the fp32 bit patterns (`pe_hist_kernel`,
-//     `pe_cut_kernel`) finds the value at the cut and how many entries tied with it are taken
-//     (ties in row-major order).
+//     `pe_cut_kernel`), with masses in exact fixed point, finds the value at the cut and how many
+//     entries tied with it are taken (ties in row-major order).
 //   Expansion + compaction: per (head, query block) a bitmap over key blocks is formed from the
 //     vertical bitmap, the shifted slash bitmap and the forced blocks {0, m}; popcounts give the row
 //     lengths (`count_vs_kernel`), one scan gives row_ptr (`scan_rows_kernel`), a second pass writes the
@@ -21,11 +21,15 @@ namespace {
 constexpr int kL0Bins = 2048, kL1Bins = 2048, kL2Bins = 512;  // key bits 30..20, 19..9, 8..0
 constexpr int kHistStride = kL0Bins + kL1Bins + kL2Bins;
 
-struct CutState {      // per head, device memory
-  unsigned int prefix; // key bits fixed so far
-  unsigned int cutkey; // final: fp32 bit pattern of the value at the cut
-  double mass_above;   // mass of entries strictly above the current prefix range
-  long long take;      // number of entries equal to cutkey that are selected
+// Masses are accumulated in 2^-60 fixed point: integer adds are exact and order independent, so the
+// histograms (built with atomics) and everything derived from them are reproducible.
+constexpr float kMassScale = 1152921504606846976.0f;  // 2^60
+
+struct CutState {                 // per head, device memory
+  unsigned int prefix;            // key bits fixed so far
+  unsigned int cutkey;            // final: fp32 bit pattern of the value at the cut
+  unsigned long long mass_above;  // mass (fixed point) of entries strictly above the current prefix range
+  long long take;                 // number of entries equal to cutkey that are selected; -1 = everything
 };
 
 struct SelectPtrs {
@@ -35,7 +39,7 @@ struct SelectPtrs {
   float* qbar;      // [hq][nb][128]
   float* amat;      // [hq][nb][nb] pooled map (row m uses columns 0..m)
   unsigned int* hcount;  // [hq][kHistStride]
-  double* hmass;         // [hq][kHistStride]
+  unsigned long long* hmass;  // [hq][kHistStride] fixed-point mass per bin
   CutState* cut;         // [hq]
   int* n_gt;        // [hq][nb]
   int* n_eq;        // [hq][nb]
@@ -296,14 +300,15 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   const int h = blockIdx.y, tid = threadIdx.x;
   if (pattern[h] != CRISP_PATTERN_PE) return;
   __shared__ unsigned int cnt[2048];
-  __shared__ double mass[2048];
+  __shared__ unsigned long long mass[2048];
   const int nbins = level == 2 ? kL2Bins : 2048;
   for (int i = tid; i < nbins; i += 256) {
     cnt[i] = 0u;
-    mass[i] = 0.0;
+    mass[i] = 0ull;
   }
   __syncthreads();
   const unsigned int prefix = w.cut[h].prefix;
+  if (level > 0 && w.cut[h].take == -1) return;  // gamma is out of reach: everything is kept
   const float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
   for (int m = blockIdx.x; m < d.nb; m += gridDim.x) {
     const float* row = am + static_cast<size_t>(m) * d.nb;
@@ -312,14 +317,14 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
       int bin;
       if (key_in_level(__float_as_uint(v), prefix, level, &bin)) {
         atomicAdd(&cnt[bin], 1u);
-        atomicAdd(&mass[bin], static_cast<double>(v));
+        atomicAdd(&mass[bin], __float2ull_rn(v * kMassScale));
       }
     }
   }
   __syncthreads();
   const int off = level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins);
   unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + off;
-  double* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
+  unsigned long long* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
   for (int i = tid; i < nbins; i += 256)
     if (cnt[i]) {
       atomicAdd(&gc[i], cnt[i]);
@@ -327,34 +332,52 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
     }
 }
 
-// One thread per head walks the bins from the largest values down until the mass reaches gamma.
-__global__ void pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int level) {
-  const int h = blockIdx.x * blockDim.x + threadIdx.x;
-  if (h >= d.hq || pattern[h] != CRISP_PATTERN_PE) return;
+// One warp per head walks the bins from the largest values down, 32 bins at a time, until the mass
+// reaches gamma.
+__global__ void __launch_bounds__(32)
+pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int level) {
+  const int h = blockIdx.x, lane = threadIdx.x;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
   const int nbins = level == 2 ? kL2Bins : 2048;
   const int off = level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins);
   const unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + off;
-  const double* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
+  const unsigned long long* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
   CutState c = w.cut[h];
   if (level == 0) {
     c.prefix = 0u;
-    c.mass_above = 0.0;
+    c.mass_above = 0ull;
     c.cutkey = 0u;
     c.take = 0x7fffffffffffffffLL;
   } else if (c.take == -1) {  // gamma was never reached at an earlier level: everything is kept
     return;
   }
-  const double gamma = static_cast<double>(d.gamma);
+  const double gd = static_cast<double>(d.gamma) * static_cast<double>(kMassScale);
+  const unsigned long long gamma = gd >= 1.8e19 ? 0xffffffffffffffffull : static_cast<unsigned long long>(gd);
   int found = -1;
-  double above = c.mass_above;
-  for (int b = nbins - 1; b >= 0; --b) {
-    if (gc[b] == 0u) continue;
-    if (above + gm[b] >= gamma) {
-      found = b;
-      break;
+  unsigned long long above = c.mass_above;
+  unsigned int found_count = 0;
+  for (int top = nbins - 1; top >= 0 && found < 0; top -= 32) {
+    const int b = top - lane;
+    const unsigned long long mine = b >= 0 ? gm[b] : 0ull;
+    const unsigned int mycnt = b >= 0 ? gc[b] : 0u;
+    unsigned long long incl = mine;  // inclusive prefix over lanes = over bins from `top` downwards
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
     }
-    above += gm[b];
+    const bool hit = mycnt != 0u && (above + incl >= gamma);
+    const unsigned int mask = __ballot_sync(0xffffffffu, hit);
+    if (mask) {
+      const int l = __ffs(mask) - 1;
+      found = top - l;
+      above += __shfl_sync(0xffffffffu, incl - mine, l);
+      found_count = __shfl_sync(0xffffffffu, mycnt, l);
+    } else {
+      above += __shfl_sync(0xffffffffu, incl, 31);
+    }
   }
+  if (lane != 0) return;
   if (found < 0) {
     // the target exceeds the total mass (gamma >= 1 or rounding): keep every causal entry
     c.cutkey = 0u;
@@ -368,13 +391,15 @@ __global__ void pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern,
   c.prefix |= static_cast<unsigned int>(found) << shift;
   if (level == 2) {
     c.cutkey = c.prefix;
-    const double v = static_cast<double>(__uint_as_float(c.cutkey));
-    long long t = static_cast<long long>(ceil((gamma - above) / v));
-    // guard the division against rounding: t is the smallest count whose mass reaches gamma
-    while (t > 1 && above + static_cast<double>(t - 1) * v >= gamma) --t;
-    while (above + static_cast<double>(t) * v < gamma && t < static_cast<long long>(gc[found])) ++t;
+    // all entries of this bin are equal; t = the smallest count whose mass reaches gamma
+    const unsigned long long v = __float2ull_rn(__uint_as_float(c.cutkey) * kMassScale);
+    long long t = 1;
+    if (v > 0ull) {
+      const unsigned long long need = gamma - above;  // > 0 here
+      t = static_cast<long long>((need + v - 1ull) / v);
+    }
     if (t < 1) t = 1;
-    if (t > static_cast<long long>(gc[found])) t = static_cast<long long>(gc[found]);
+    if (t > static_cast<long long>(found_count)) t = static_cast<long long>(found_count);
     c.take = t;
   }
   w.cut[h] = c;
@@ -576,7 +601,7 @@ SelectPtrs carve(const Dims& d, void* ws, size_t* total) {
   w.qbar = static_cast<float*>(take(sizeof(float) * static_cast<size_t>(d.hq) * d.nb * kHeadDim));
   w.amat = static_cast<float*>(take(sizeof(float) * static_cast<size_t>(d.hq) * d.nb * d.nb));
   w.hcount = static_cast<unsigned int*>(take(sizeof(unsigned int) * d.hq * kHistStride));
-  w.hmass = static_cast<double*>(take(sizeof(double) * d.hq * kHistStride));
+  w.hmass = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * d.hq * kHistStride));
   w.cut = static_cast<CutState*>(take(sizeof(CutState) * d.hq));
   w.n_gt = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
   w.n_eq = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
@@ -604,7 +629,7 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   int* status = static_cast<int*>(ws);
   CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "select: clear status");
   CRISP_CUDA_TRY(cudaMemsetAsync(w.hcount, 0, sizeof(unsigned int) * d.hq * kHistStride, stream), "select: clear");
-  CRISP_CUDA_TRY(cudaMemsetAsync(w.hmass, 0, sizeof(double) * d.hq * kHistStride, stream), "select: clear");
+  CRISP_CUDA_TRY(cudaMemsetAsync(w.hmass, 0, sizeof(unsigned long long) * d.hq * kHistStride, stream), "select: clear");
 
   // VS heads
   const size_t vs_smem = (sizeof(double) + sizeof(float) + sizeof(int) + 1) * static_cast<size_t>(d.nb) + 16;
@@ -624,7 +649,7 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   const int hist_ctas = d.nb < 128 ? d.nb : 128;
   for (int level = 0; level < 3; ++level) {
     pe_hist_kernel<<<dim3(hist_ctas, d.hq), 256, 0, stream>>>(d, pattern, w, level);
-    pe_cut_kernel<<<(d.hq + 31) / 32, 32, 0, stream>>>(d, pattern, w, level);
+    pe_cut_kernel<<<d.hq, 32, 0, stream>>>(d, pattern, w, level);
   }
   pe_row_stats_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w);
   pe_take_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w);
