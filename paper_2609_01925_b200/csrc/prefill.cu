@@ -8,7 +8,7 @@
 // Warp roles (384 threads):
 //   warps 0-3  softmax of tile 0 (one thread per query row; TMEM lanes 0-127)
 //   warps 4-7  softmax of tile 1
-//   warp  8    TMA producer: Q once per item, K and V blocks through two-stage rings
+//   warp  8    TMA producer: Q once per item, K and V blocks through one five-slot ring
 //   warp  9    MMA issuer: S_t = Q_t K^T (SS) and O_t += P_t V (P read from TMEM)
 // TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each; P_t (bf16) overwrites the first
 // 64 columns of S_t.  The issuer interleaves the two tiles so that the tensor pipe works on one
@@ -26,6 +26,11 @@ namespace {
 
 constexpr uint32_t kFlag0 = 1u << 30, kFlag1 = 1u << 31, kColMask = kFlag0 - 1u;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr int kStages = 5;                 // K/V ring slots of 32 KB
+#ifndef CRISP_SPLIT_P
+#define CRISP_SPLIT_P 0
+#endif
+constexpr bool kSplitP = CRISP_SPLIT_P != 0;  // hand P to the MMA issuer in two halves (measured: no gain, off)
 
 struct PrefillArgs {
   const int32_t* merged;   // per item: union list, entry = key block | flags (sparse only)
@@ -41,11 +46,10 @@ struct PrefillArgs {
 
 struct PrefillSmem {
   alignas(1024) uint8_t q[2][2][16384];  // [tile][half]
-  alignas(1024) uint8_t k[2][2][16384];  // [stage][half]
-  alignas(1024) uint8_t v[2][2][16384];  // [stage][half]
+  alignas(1024) uint8_t kv[kStages][2][16384];  // ring of K and V blocks [slot][half]; load 2e is K_e, 2e+1 is V_e
   uint64_t q_full, q_free;
-  uint64_t k_full[2], k_empty[2], v_full[2], v_empty[2];
-  uint64_t s_full[2], p_ready[2], o_done[2];
+  uint64_t kv_full[kStages], kv_empty[kStages];
+  uint64_t s_full[2], p_ready[2][2], o_done[2];  // p_ready[tile][half of the keys]
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -119,6 +123,58 @@ __device__ __forceinline__ bool mbar_wait_lane0(uint64_t* bar, uint32_t parity, 
   return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
+// ---- packed fp32x2 arithmetic (two lanes per instruction on the FMA pipe)
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+  return v;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// 2^t for a pair of values on the FMA pipe instead of the MUFU: t = n + f with n = round(t),
+// f in [-0.5, 0.5]; 2^f by a degree-4 minimax polynomial (max relative error 2.6e-6, far below the
+// bf16 rounding of P); 2^n by adding n to the exponent field.  t is clamped at -125.
+__device__ __forceinline__ void exp2_poly2(uint64_t t2, float& p0, float& p1) {
+  float t0, t1;
+  unpack2(t2, t0, t1);
+  t0 = fmaxf(t0, -125.0f);
+  t1 = fmaxf(t1, -125.0f);
+  t2 = pack2(t0, t1);
+  const uint64_t magic = pack2(12582912.0f, 12582912.0f);      // 1.5 * 2^23: rounds to an integer
+  const uint64_t neg_magic = pack2(-12582912.0f, -12582912.0f);
+  const uint64_t neg_one = pack2(-1.0f, -1.0f);
+  const uint64_t r2 = add2(t2, magic);
+  const uint64_t n2 = add2(r2, neg_magic);
+  const uint64_t f2 = fma2(n2, neg_one, t2);
+  uint64_t q2 = fma2(f2, pack2(0.009570101276040077f, 0.009570101276040077f),
+                     pack2(0.05591785907745361f, 0.05591785907745361f));
+  q2 = fma2(q2, f2, pack2(0.240247443318367f, 0.240247443318367f));
+  q2 = fma2(q2, f2, pack2(0.6931217908859253f, 0.6931217908859253f));
+  q2 = fma2(q2, f2, pack2(0.9999992847442627f, 0.9999992847442627f));
+  float r0, r1, q0, q1;
+  unpack2(r2, r0, r1);
+  unpack2(q2, q0, q1);
+  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(r0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(r1) << 23));
+}
+
 // Maximum of one row of raw logits; on the diagonal block only keys j <= r are visible.
 template <bool kDiag>
 __device__ __forceinline__ float row_max(const uint32_t (&x)[4][32], int r) {
@@ -126,47 +182,68 @@ __device__ __forceinline__ float row_max(const uint32_t (&x)[4][32], int r) {
 #pragma unroll
   for (int c = 0; c < 4; ++c)
 #pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-      float a0 = __uint_as_float(x[c][i]), a1 = __uint_as_float(x[c][i + 1]);
-      float a2 = __uint_as_float(x[c][i + 2]), a3 = __uint_as_float(x[c][i + 3]);
-      if (kDiag) {
-        const int j = c * 32 + i;
-        if (j > r) a0 = -INFINITY;
-        if (j + 1 > r) a1 = -INFINITY;
-        if (j + 2 > r) a2 = -INFINITY;
-        if (j + 3 > r) a3 = -INFINITY;
+    for (int i = 0; i < 32; i += 8) {
+      float a[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        a[u] = __uint_as_float(x[c][i + u]);
+        if (kDiag && (c * 32 + i + u) > r) a[u] = -INFINITY;
       }
-      m0 = fmaxf(m0, a0);
-      m1 = fmaxf(m1, a1);
-      m2 = fmaxf(m2, a2);
-      m3 = fmaxf(m3, a3);
+      m0 = max3(m0, a[0], a[1]);
+      m1 = max3(m1, a[2], a[3]);
+      m2 = max3(m2, a[4], a[5]);
+      m3 = max3(m3, a[6], a[7]);
     }
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
-// P = 2^(x * scale - m) as bf16 into TMEM (two keys per 32-bit column); returns the fp32 row sum.
+// P = 2^(x * scale - m) as bf16 into TMEM (two keys per 32-bit column) for one half of the keys
+// (half 0: keys 0-63, half 1: keys 64-127); returns the fp32 sum of that half of the row.
+// With kPolyEvery > 0 one pair in every kPolyEvery goes through exp2_poly2 (FMA pipe) instead of the MUFU.
+// Measured on B200 (L32k dense): 959 TFLOP/s with 0, 893 with 4, 854 with 2 - the softmax warps are bound
+// by issue slots, not by the MUFU, so the default is 0 (every exponential on the MUFU).
+#ifndef CRISP_POLY_EVERY
+#define CRISP_POLY_EVERY 0
+#endif
+constexpr int kPolyEvery = CRISP_POLY_EVERY;
 template <bool kDiag>
-__device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int r, float scale_log2, float m_used,
-                                                uint32_t s_addr) {
-  float sum0 = 0.f, sum1 = 0.f;
+__device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int half, int r, float scale_log2,
+                                                float m_used, uint32_t s_addr) {
+  const uint64_t scale2 = pack2(scale_log2, scale_log2);
+  const uint64_t negm2 = pack2(-m_used, -m_used);
+  uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
+  for (int c = 2 * half; c < 2 * half + 2; ++c) {
     uint32_t pk[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-      float p0 = ex2(fmaf(__uint_as_float(x[c][2 * i]), scale_log2, -m_used));
-      float p1 = ex2(fmaf(__uint_as_float(x[c][2 * i + 1]), scale_log2, -m_used));
+      const uint64_t t2 = fma2(pack2(__uint_as_float(x[c][2 * i]), __uint_as_float(x[c][2 * i + 1])), scale2, negm2);
+      float p0, p1;
+      if (kPolyEvery > 0 && (i % kPolyEvery) == kPolyEvery - 1) {
+        exp2_poly2(t2, p0, p1);
+      } else {
+        float t0, t1;
+        unpack2(t2, t0, t1);
+        p0 = ex2(t0);
+        p1 = ex2(t1);
+      }
       if (kDiag) {
         if (c * 32 + 2 * i > r) p0 = 0.f;
         if (c * 32 + 2 * i + 1 > r) p1 = 0.f;
       }
-      sum0 += p0;
-      sum1 += p1;
+      if (i & 1) {
+        sum_a = add2(sum_a, pack2(p0, p1));
+      } else {
+        sum_b = add2(sum_b, pack2(p0, p1));
+      }
       pk[i] = pack_bf16(p0, p1);
     }
     tmem_st_x16(s_addr + c * 16, pk);
   }
-  return sum0 + sum1;
+  float s0, s1, s2, s3;
+  unpack2(sum_a, s0, s1);
+  unpack2(sum_b, s2, s3);
+  return (s0 + s1) + (s2 + s3);
 }
 
 template <bool kDense>
@@ -181,13 +258,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     s.abort_flag = 0;
     mbar_init(&s.q_full, 1);
     mbar_init(&s.q_free, 1);
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(&s.kv_full[i], 1);
+      mbar_init(&s.kv_empty[i], 1);
+    }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&s.k_full[i], 1);
-      mbar_init(&s.k_empty[i], 1);
-      mbar_init(&s.v_full[i], 1);
-      mbar_init(&s.v_empty[i], 1);
       mbar_init(&s.s_full[i], 1);
-      mbar_init(&s.p_ready[i], 128);
+      mbar_init(&s.p_ready[i][0], 128);
+      mbar_init(&s.p_ready[i][1], 128);
       mbar_init(&s.o_done[i], 1);
     }
     fence_mbar_init();
@@ -234,22 +312,22 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       for (int e = 0; e < it.n_entries; ++e, ++ecount) {
         const uint32_t ent = rd.get(e, it.n_entries, lane);
         const int J = static_cast<int>(ent & kColMask);
-        const int st = ecount & 1;
-        const uint32_t use = ecount >> 1;
-        if (use > 0) ok = mbar_wait_lane0(&s.k_empty[st], (use - 1) & 1, abort_flag, lane);
-        if (!ok) break;
-        if (lane == 0) {
-          mbar_arrive_expect_tx(&s.k_full[st], 32768u);
-          tma_load_3d(s.k[st][0], &tmap_k, &s.k_full[st], 0, it.kvh, J * kBlock);
-          tma_load_3d(s.k[st][1], &tmap_k, &s.k_full[st], 64, it.kvh, J * kBlock);
+        // loads 2*ecount (K) and 2*ecount + 1 (V) go to consecutive ring slots
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+          const uint32_t load = 2u * ecount + which;
+          const int slot = load % kStages;
+          const uint32_t use = load / kStages;
+          if (use > 0) ok = mbar_wait_lane0(&s.kv_empty[slot], (use - 1) & 1, abort_flag, lane);
+          if (!ok) break;
+          if (lane == 0) {
+            const CUtensorMap* tmap = which == 0 ? &tmap_k : &tmap_v;
+            mbar_arrive_expect_tx(&s.kv_full[slot], 32768u);
+            tma_load_3d(s.kv[slot][0], tmap, &s.kv_full[slot], 0, it.kvh, J * kBlock);
+            tma_load_3d(s.kv[slot][1], tmap, &s.kv_full[slot], 64, it.kvh, J * kBlock);
+          }
         }
-        if (use > 0) ok = mbar_wait_lane0(&s.v_empty[st], (use - 1) & 1, abort_flag, lane);
         if (!ok) break;
-        if (lane == 0) {
-          mbar_arrive_expect_tx(&s.v_full[st], 32768u);
-          tma_load_3d(s.v[st][0], &tmap_v, &s.v_full[st], 0, it.kvh, J * kBlock);
-          tma_load_3d(s.v[st][1], &tmap_v, &s.v_full[st], 64, it.kvh, J * kBlock);
-        }
       }
     }
   } else if (warp == 9) {
@@ -262,40 +340,67 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     int it_count = 0;
     bool ok = true;
 
+    // Operand descriptors are built once; inside the loops only the 14-bit start-address field moves
+    // (a compile-time offset per K step), so issuing an MMA costs two integer adds.
+    const uint64_t q_desc[2] = {umma_desc_sw128(smem_u32(s.q[0][0]), 0, 1024),
+                                umma_desc_sw128(smem_u32(s.q[1][0]), 0, 1024)};
+    // slot s of the ring starts 32 KB after slot s - 1: +2048 in the descriptor's address field
+    const uint64_t k_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 0, 1024);      // K block: K-major B operand
+    const uint64_t v_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 16384, 1024);  // V block: MN-major B operand
+
     auto issue_qk = [&](int t, uint32_t ecount, bool last_use, bool last_of_item) {
-      const int st = ecount & 1;
-      ok = ok && mbar_wait_lane0(&s.k_full[st], (ecount >> 1) & 1, abort_flag, lane);
+      const uint32_t load = 2u * ecount;
+      const int st = load % kStages;
+      ok = ok && mbar_wait_lane0(&s.kv_full[st], (load / kStages) & 1, abort_flag, lane);
       if (!ok) return;
       tc_fence_after_sync();
       if (lane == 0) {
+        const uint64_t ad0 = q_desc[t], bd0 = k_desc0 + static_cast<uint64_t>(st) * 2048u;
+        const uint32_t dst = tm + t * 128;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t ad = umma_desc_sw128(smem_u32(s.q[t][kk >> 2]) + (kk & 3) * 32, 0, 1024);
-          const uint64_t bd = umma_desc_sw128(smem_u32(s.k[st][kk >> 2]) + (kk & 3) * 32, 0, 1024);
-          umma_ss(tm + t * 128, ad, bd, idesc_qk, kk > 0);
+          // K step kk: 64-column half kk / 4 (16 KB apart), 32 bytes per step inside the swizzle atom
+          constexpr uint32_t kHalf = 16384 >> 4, kStep = 32 >> 4;
+          const uint64_t off = static_cast<uint64_t>((kk >> 2) * kHalf + (kk & 3) * kStep);
+          umma_ss(dst, ad0 + off, bd0 + off, idesc_qk, kk > 0);
         }
         umma_commit(&s.s_full[t]);
-        if (last_use) umma_commit(&s.k_empty[st]);
+        if (last_use) umma_commit(&s.kv_empty[st]);
         if (last_of_item) umma_commit(&s.q_free);
       }
       __syncwarp();
     };
     auto issue_pv = [&](int t, uint32_t ecount, bool last_use, bool first_of_tile) {
-      const int st = ecount & 1;
-      ok = ok && mbar_wait_lane0(&s.p_ready[t], pv_count[t] & 1, abort_flag, lane);
-      ok = ok && mbar_wait_lane0(&s.v_full[st], (ecount >> 1) & 1, abort_flag, lane);
+      const uint32_t load = 2u * ecount + 1u;
+      const int st = load % kStages;
+      const uint64_t bd0 = v_desc0 + static_cast<uint64_t>(st) * 2048u;
+      const uint32_t dst = tm + 256 + t * 128, src = tm + t * 128;
+      // P arrives in two halves (keys 0-63, 64-127): the first four MMAs start while the softmax warps
+      // still work on the second half
+      ok = ok && mbar_wait_lane0(&s.p_ready[t][0], pv_count[t] & 1, abort_flag, lane);
+      ok = ok && mbar_wait_lane0(&s.kv_full[st], (load / kStages) & 1, abort_flag, lane);
+      if (!ok) return;
+      tc_fence_after_sync();
+      if (lane == 0) {
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          // V block as the MN-major B operand: 16 keys per step = two groups of 8 key rows = 2048 B
+          const uint64_t off = static_cast<uint64_t>(kk * (2048 >> 4));
+          umma_ts(dst, src + kk * 8, bd0 + off, idesc_pv, (kk > 0 || !first_of_tile) ? 1u : 0u);
+        }
+      }
+      if (kSplitP) ok = ok && mbar_wait_lane0(&s.p_ready[t][1], pv_count[t] & 1, abort_flag, lane);
       if (!ok) return;
       ++pv_count[t];
       tc_fence_after_sync();
       if (lane == 0) {
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          // V block as the MN-major B operand: 16 keys per step = two groups of 8 key rows
-          const uint64_t bd = umma_desc_sw128(smem_u32(s.v[st][0]) + kk * 2048, 16384, 1024);
-          umma_ts(tm + 256 + t * 128, tm + t * 128 + kk * 8, bd, idesc_pv, (kk > 0 || !first_of_tile) ? 1u : 0u);
+        for (int kk = 4; kk < 8; ++kk) {
+          const uint64_t off = static_cast<uint64_t>(kk * (2048 >> 4));
+          umma_ts(dst, src + kk * 8, bd0 + off, idesc_pv, 1u);
         }
         umma_commit(&s.o_done[t]);
-        if (last_use) umma_commit(&s.v_empty[st]);
+        if (last_use) umma_commit(&s.kv_empty[st]);
       }
       __syncwarp();
     };
@@ -403,16 +508,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           l_run *= f;
           m_used = m_new;
         }
-        float sum;
-        if (diag) {
-          sum = exp_pack_store<true>(x, r, d.scale_log2, m_used, s_addr);
-        } else {
-          sum = exp_pack_store<false>(x, r, d.scale_log2, m_used, s_addr);
+        float sum = 0.f;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+          if (diag) {
+            sum += exp_pack_store<true>(x, half, r, d.scale_log2, m_used, s_addr);
+          } else {
+            sum += exp_pack_store<false>(x, half, r, d.scale_log2, m_used, s_addr);
+          }
+          if (kSplitP || half == 1) {
+            tmem_st_wait();
+            tc_fence_before_sync();
+            mbar_arrive(&s.p_ready[t][kSplitP ? half : 0]);
+          }
         }
         l_run += sum;
-        tmem_st_wait();
-        tc_fence_before_sync();
-        mbar_arrive(&s.p_ready[t]);
         first = false;
         ++step_count;
       }
