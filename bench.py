@@ -137,6 +137,20 @@ def oracle_sample(w, q, k, v, seed=0, budget_blocks=6):
     return ms, desc, cores
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Step time of the job = the slowest rank's (all ranks run the same number of steps)."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_ms_per_layer(ms_per_step: float, world: int) -> float:
+    """Weak scaling: every rank processes one layer per step, so the job does `world` layers per step."""
+    return ms_per_step / world
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -252,11 +266,7 @@ def main():
     layer.poll()
     clocks = sampler.stop()
 
-    ms_per_step = total_ms / args.steps
-    if dist is not None:
-        t = torch.tensor([ms_per_step], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step = float(t.item())
+    ms_per_step = max_over_ranks(total_ms / args.steps, dist, dev)
     med = {kk: statistics.median(vv) for kk, vv in stage_ms.items()}
     dense = statistics.median(dense_ms)
     sparse_tflops = nnz * FLOP_PER_BLOCK / (med["sparse_prefill"] * 1e-3) / 1e12
@@ -279,14 +289,10 @@ def main():
             oh.copy_(layer.o, non_blocking=True)
         b = ev(); b.record()
         barrier()
-        e2e_ms = a.elapsed_time(b) / e2e_steps
-        if dist is not None:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(a.elapsed_time(b) / e2e_steps, dist, dev)
         h2d = sum(x.numel() * x.element_size() for x in (qh, kh, vh))
         d2h = oh.numel() * oh.element_size()
-        e2e = {"value": e2e_ms / world, "unit": "ms/layer", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        e2e = {"value": job_ms_per_layer(e2e_ms, world), "unit": "ms/layer", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
         del qh, kh, vh, oh, qd, kd, vd
 
     cpu_baseline = None
@@ -301,7 +307,7 @@ def main():
         return
     out = {
         "metric": "prefill attention ms/layer (route+select+sparse prefill)",
-        "value": ms_per_step / world, "unit": "ms/layer", "n_gpus": world, "steps": args.steps,
+        "value": job_ms_per_layer(ms_per_step, world), "unit": "ms/layer", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
         "stages_ms": med, "dense_prefill_ms": dense, "speedup_vs_own_dense": dense / ms_per_step,

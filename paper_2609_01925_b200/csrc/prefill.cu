@@ -42,6 +42,7 @@ struct PrefillArgs {
   int* status;
   int n_pairs;
   int n_items;
+  int group_kv;            // 1: schedule one KV head at a time (K/V larger than L2), 0: one global order
 };
 
 struct PrefillSmem {
@@ -64,7 +65,19 @@ struct Item {
 template <bool kDense>
 __device__ __forceinline__ Item decode_item(int pos, const Dims& d, const PrefillArgs& a) {
   Item it;
-  const int idx = kDense ? pos : a.order[pos];
+  // Item id = (n_pairs - 1 - u) * H_q + h.  Dense: positions walk one KV head at a time (its G query
+  // heads interleaved, long rows first), so the CTAs running at any moment stream the same K/V blocks
+  // and share them in L2.  Sparse: the same grouping, sorted by cost inside each KV head.
+  int idx;
+  if (kDense && !a.group_kv) {
+    idx = pos;
+  } else if (kDense) {
+    const int per_kv = a.n_pairs * d.group;
+    const int kvh = pos / per_kv, rem = pos % per_kv;
+    idx = (rem / d.group) * d.hq + kvh * d.group + rem % d.group;
+  } else {
+    idx = a.order[pos];
+  }
   it.h = idx % d.hq;
   const int u = a.n_pairs - 1 - idx / d.hq;  // long rows first
   it.kvh = it.h / d.group;
@@ -568,7 +581,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 __global__ void __launch_bounds__(128)
 merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                    int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
-                   int n_pairs) {
+                   int n_pairs, int n_cost, int group_kv) {
   extern __shared__ uint32_t bm[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
@@ -620,40 +633,41 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   }
   if (lane == 0) {
     item_len[h * n_pairs + u] = written;
-    atomicAdd(&cost_hist[static_cast<int>(e1 - s0)], 1);  // cost = tile steps = len(m0) + len(m1)
+    // sort key: KV head first, then decreasing cost (= tile steps = len(m0) + len(m1))
+    atomicAdd(&cost_hist[(group_kv ? h / d.group : 0) * n_cost + (n_cost - 1 - static_cast<int>(e1 - s0))], 1);
   }
 }
 
-// Counting sort of the items by decreasing cost, so that the round-robin assignment of items to
-// CTAs balances heads with long lists (PE) against heads with short ones (VS).
+// Counting sort of the items by (KV head, decreasing cost).  Grouping by KV head keeps the CTAs that
+// run at the same time on the same K/V blocks (L2 reuse); sorting by cost inside a group lets the
+// round-robin assignment balance heads with long lists (PE) against heads with short ones (VS).
 __global__ void __launch_bounds__(1024) sched_scan_kernel(int* __restrict__ cost_hist, int n_bins) {
   __shared__ int seg_tot[1024];
   const int tid = threadIdx.x;
   const int seg = (n_bins + 1023) / 1024;
-  // bins are visited from the largest cost down
   const int b0 = min(tid * seg, n_bins), b1 = min(b0 + seg, n_bins);
   int local = 0;
-  for (int i = b0; i < b1; ++i) local += cost_hist[n_bins - 1 - i];
+  for (int i = b0; i < b1; ++i) local += cost_hist[i];
   seg_tot[tid] = local;
   __syncthreads();
   int run = 0;
   for (int t = 0; t < tid; ++t) run += seg_tot[t];
   for (int i = b0; i < b1; ++i) {
-    const int c = cost_hist[n_bins - 1 - i];
-    cost_hist[n_bins - 1 - i] = run;  // first position of this cost in the sorted order
+    const int c = cost_hist[i];
+    cost_hist[i] = run;  // first position of this key in the sorted order
     run += c;
   }
 }
 
 __global__ void __launch_bounds__(256)
 sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, int* __restrict__ cost_hist,
-                     int* __restrict__ order, int n_pairs) {
+                     int* __restrict__ order, int n_pairs, int n_cost, int group_kv) {
   const int u = blockIdx.x * blockDim.x + threadIdx.x, h = blockIdx.y;
   if (u >= n_pairs) return;
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int m0 = 2 * u, mend = min(2 * u + 2, d.nb);
   const int cost = static_cast<int>(rp[mend] - rp[m0]);
-  const int pos = atomicAdd(&cost_hist[cost], 1);
+  const int pos = atomicAdd(&cost_hist[(group_kv ? h / d.group : 0) * n_cost + (n_cost - 1 - cost)], 1);
   order[pos] = (n_pairs - 1 - u) * d.hq + h;
 }
 
@@ -661,7 +675,8 @@ struct PrefillWs {
   int* item_len;
   int* order;
   int* cost_hist;
-  int n_bins;
+  int n_cost;  // distinct cost values (0 .. 2 N_b + 1)
+  int n_bins;  // n_cost per KV head
   int32_t* merged;
 };
 
@@ -674,7 +689,8 @@ PrefillWs carve(const Dims& d, void* ws, size_t* total) {
   off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
   w.order = reinterpret_cast<int*>(base + off);
   off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
-  w.n_bins = 2 * d.nb + 2;
+  w.n_cost = 2 * d.nb + 2;
+  w.n_bins = w.n_cost * d.hkv;
   w.cost_hist = reinterpret_cast<int*>(base + off);
   off += align_up(sizeof(int) * static_cast<size_t>(w.n_bins), 256);
   w.merged = reinterpret_cast<int32_t*>(base + off);
@@ -713,6 +729,8 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.status = static_cast<int*>(ws);
+  // K + V of all KV heads against the 126 MB L2: group the schedule by KV head only when they do not fit
+  a.group_kv = (static_cast<size_t>(d.n) * d.hkv * kHeadDim * 2 * 2 > (256u << 20)) ? 1 : 0;
 
   int dev = 0, n_sm = 0;
   CRISP_CUDA_TRY(cudaGetDevice(&dev), "prefill: device");
@@ -728,10 +746,10 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
     const int words = (d.nb + 31) / 32;
     CRISP_CUDA_TRY(cudaMemsetAsync(w.cost_hist, 0, sizeof(int) * w.n_bins, stream), "prefill: clear histogram");
     merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
-        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs);
+        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv);
     sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins);
     sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, 0, stream>>>(d, row_ptr, w.cost_hist,
-                                                                               w.order, a.n_pairs);
+                                                                               w.order, a.n_pairs, w.n_cost, a.group_kv);
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
