@@ -137,6 +137,19 @@ def oracle_sample(w, q, k, v, seed=0, budget_blocks=6):
     return ms, desc, cores
 
 
+def ncu_traffic_bytes(kernel: str, workload: str):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary of `workload`, or None."""
+    path = os.path.join(ROOT, "profiles", f"dram_traffic_{workload}_ncu.md")
+    if not os.path.exists(path):
+        return None
+    key = f"traffic_bytes_per_launch {kernel} {workload} ="
+    with open(path) as f:
+        for line in f:
+            if line.startswith(key):
+                return int(line.split("=")[1])
+    return None
+
+
 def max_over_ranks(ms: float, dist, device) -> float:
     """Step time of the job = the slowest rank's (all ranks run the same number of steps)."""
     if dist is None:
@@ -320,7 +333,9 @@ def main():
         "roofline": {"bound": "tensor", "kernel": "prefill_kernel<sparse>", "achieved": sparse_tflops,
                      "peak": peak, "unit": "TFLOP/s", "frac": sparse_tflops / peak,
                      "peak_source": f"{peaks['source']} ({'sustained' if peak == peaks['bf16_sustained'] else 'burst'})",
-                     "traffic": None},
+                     "traffic": ncu_traffic_bytes("prefill_kernel<sparse>", w.name),
+                     "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)",
+                     "algorithmic_flop_per_launch": nnz * FLOP_PER_BLOCK},
         "cpu_baseline": cpu_baseline, "e2e": e2e,
         "gpu_launches": args.steps * (LAUNCHES_ROUTE + LAUNCHES_SELECT + LAUNCHES_PREFILL),
         "clocks": clocks,

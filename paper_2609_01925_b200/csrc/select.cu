@@ -312,12 +312,28 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   const float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
   for (int m = blockIdx.x; m < d.nb; m += gridDim.x) {
     const float* row = am + static_cast<size_t>(m) * d.nb;
-    for (int J = tid; J <= m; J += 256) {
-      const float v = row[J];
-      int bin;
-      if (key_in_level(__float_as_uint(v), prefix, level, &bin)) {
-        atomicAdd(&cnt[bin], 1u);
-        atomicAdd(&mass[bin], __float2ull_rn(v * kMassScale));
+    for (int J0 = 0; J0 <= m; J0 += 256) {
+      const int J = J0 + tid;
+      int bin = -1;
+      unsigned long long fixed = 0ull;
+      if (J <= m) {
+        const float v = row[J];
+        int b;
+        if (key_in_level(__float_as_uint(v), prefix, level, &b)) {
+          bin = b;
+          fixed = __float2ull_rn(v * kMassScale);
+        }
+      }
+      // Neighbouring entries of a flat map fall into a handful of bins: lanes with the same bin elect a
+      // leader and add their counts and masses (three 20-bit limbs, summed exactly) in one atomic each.
+      const unsigned int peers = __match_any_sync(0xffffffffu, bin);
+      const unsigned int l0 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed & 0xFFFFFull));
+      const unsigned int l1 = __reduce_add_sync(peers, static_cast<unsigned int>((fixed >> 20) & 0xFFFFFull));
+      const unsigned int l2 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed >> 40));
+      if (bin >= 0 && (tid & 31) == __ffs(peers) - 1) {
+        atomicAdd(&cnt[bin], static_cast<unsigned int>(__popc(peers)));
+        atomicAdd(&mass[bin], static_cast<unsigned long long>(l0) + (static_cast<unsigned long long>(l1) << 20) +
+                                  (static_cast<unsigned long long>(l2) << 40));
       }
     }
   }
