@@ -8,12 +8,15 @@
 // Warp roles (384 threads):
 //   warps 0-3  softmax of tile 0 (one thread per query row; TMEM lanes 0-127)
 //   warps 4-7  softmax of tile 1
-//   warp  8    TMA producer: Q once per item, K and V blocks through one five-slot ring
-//   warp  9    MMA issuer: S_t = Q_t K^T (SS) and O_t += P_t V (P read from TMEM)
+//   warp  8    TMA producer (one thread): Q once per item, K and V blocks through one five-slot ring
+//   warp  9    MMA issuer (one thread): S_t = Q_t K^T (SS) and O_t += P_t V (P read from TMEM)
 // TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each; P_t (bf16) overwrites the first
 // 64 columns of S_t.  The issuer interleaves the two tiles so that the tensor pipe works on one
 // tile while the other tile's softmax runs.  The online softmax rescales O lazily, only when the
 // running maximum grows by more than 2^8, and does it in place in TMEM.
+// Measured alternatives that were slower and are not kept: one issuing thread per tile (the two tiles
+// fall into phase, both softmax phases collide and the tensor pipe idles: 726 vs 970 TFLOP/s dense);
+// handing P over in two halves; computing part of the exponentials on the FMA pipe (see kPolyEvery).
 // Every mbarrier wait is bounded; a wait that gives up sets a flag that ends all roles, and the
 // status word reports CRISP_ERR_DEVICE_TIMEOUT.
 #include "common.cuh"
@@ -27,10 +30,6 @@ namespace {
 constexpr uint32_t kFlag0 = 1u << 30, kFlag1 = 1u << 31, kColMask = kFlag0 - 1u;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 constexpr int kStages = 5;                 // K/V ring slots of 32 KB
-#ifndef CRISP_SPLIT_P
-#define CRISP_SPLIT_P 0
-#endif
-constexpr bool kSplitP = CRISP_SPLIT_P != 0;  // hand P to the MMA issuer in two halves (measured: no gain, off)
 
 struct PrefillArgs {
   const int32_t* merged;   // per item: union list, entry = key block | flags (sparse only)
@@ -50,7 +49,7 @@ struct PrefillSmem {
   alignas(1024) uint8_t kv[kStages][2][16384];  // ring of K and V blocks [slot][half]; load 2e is K_e, 2e+1 is V_e
   uint64_t q_full, q_free;
   uint64_t kv_full[kStages], kv_empty[kStages];
-  uint64_t s_full[2], p_ready[2][2], o_done[2];  // p_ready[tile][half of the keys]
+  uint64_t s_full[2], p_ready[2], o_done[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -119,6 +118,12 @@ struct EntryReader {
     return __shfl_sync(0xffffffffu, chunk, e & 31);
   }
 };
+
+// Register budgets after setmaxnreg.  The CTA's pool is what the launch allocated (384 threads x 168
+// registers); setmaxnreg.inc waits, without a bound, until the pool can serve it, so the budgets of the
+// three warpgroups must never add up to more than the pool.
+constexpr int kRegsSoftmax = 208, kRegsOther = 88, kRegsLaunch = 168;
+static_assert(256 * kRegsSoftmax + 128 * kRegsOther <= 384 * kRegsLaunch, "setmaxnreg budgets exceed the CTA's pool");
 
 template <int N>
 __device__ __forceinline__ void reg_alloc() {
@@ -210,8 +215,7 @@ __device__ __forceinline__ float row_max(const uint32_t (&x)[4][32], int r) {
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
-// P = 2^(x * scale - m) as bf16 into TMEM (two keys per 32-bit column) for one half of the keys
-// (half 0: keys 0-63, half 1: keys 64-127); returns the fp32 sum of that half of the row.
+// P = 2^(x * scale - m) as bf16 into TMEM (two keys per 32-bit column); returns the fp32 row sum.
 // With kPolyEvery > 0 one pair in every kPolyEvery goes through exp2_poly2 (FMA pipe) instead of the MUFU.
 // Measured on B200 (L32k dense): 959 TFLOP/s with 0, 893 with 4, 854 with 2 - the softmax warps are bound
 // by issue slots, not by the MUFU, so the default is 0 (every exponential on the MUFU).
@@ -220,13 +224,13 @@ __device__ __forceinline__ float row_max(const uint32_t (&x)[4][32], int r) {
 #endif
 constexpr int kPolyEvery = CRISP_POLY_EVERY;
 template <bool kDiag>
-__device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int half, int r, float scale_log2,
-                                                float m_used, uint32_t s_addr) {
+__device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int r, float scale_log2, float m_used,
+                                                uint32_t s_addr) {
   const uint64_t scale2 = pack2(scale_log2, scale_log2);
   const uint64_t negm2 = pack2(-m_used, -m_used);
   uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
 #pragma unroll
-  for (int c = 2 * half; c < 2 * half + 2; ++c) {
+  for (int c = 0; c < 4; ++c) {
     uint32_t pk[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
@@ -259,6 +263,34 @@ __device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int 
   return (s0 + s1) + (s2 + s3);
 }
 
+// Entry stream for a role run by a single thread: the next entry is fetched one iteration early, so the
+// global-load latency hides behind the current step.
+template <bool kDense>
+struct EntryStream {
+  const int32_t* list;
+  uint32_t next;
+  int m0, n_entries;
+  bool tile1;
+  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& a) {
+    list = kDense ? nullptr : a.merged + it.base;
+    m0 = it.m0;
+    tile1 = it.tile1;
+    n_entries = it.n_entries;
+    next = (!kDense && n_entries > 0) ? static_cast<uint32_t>(__ldg(list)) : 0u;
+  }
+  __device__ __forceinline__ uint32_t get(int e) {
+    if (kDense) {
+      uint32_t x = static_cast<uint32_t>(e);
+      if (e <= m0) x |= kFlag0;
+      if (tile1) x |= kFlag1;
+      return x;
+    }
+    const uint32_t cur = next;
+    if (e + 1 < n_entries) next = static_cast<uint32_t>(__ldg(list + e + 1));
+    return cur;
+  }
+};
+
 template <bool kDense>
 __global__ void __launch_bounds__(384, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -277,8 +309,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s.s_full[i], 1);
-      mbar_init(&s.p_ready[i][0], 128);
-      mbar_init(&s.p_ready[i][1], 128);
+      mbar_init(&s.p_ready[i], 128);
       mbar_init(&s.o_done[i], 1);
     }
     fence_mbar_init();
@@ -298,22 +329,22 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   // (each role changes its own budget at the top of its branch)
   if (warp == 8) {
     // =============================================================== TMA producer
-    reg_dealloc<56>();
+    reg_dealloc<kRegsOther>();
     if (lane == 0) {
       prefetch_tmap(&tmap_q);
       prefetch_tmap(&tmap_k);
       prefetch_tmap(&tmap_v);
     }
-    uint32_t ecount = 0;
-    int it_count = 0;
-    bool ok = true;
-    for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
-      const Item it = decode_item<kDense>(idx, d, a);
-      EntryReader<kDense> rd;
-      rd.init(it, a);
-      if (it_count > 0) ok = mbar_wait_lane0(&s.q_free, (it_count - 1) & 1, abort_flag, lane);
-      if (!ok) break;
-      if (lane == 0) {
+    if (lane == 0) {
+      uint32_t ecount = 0;
+      int it_count = 0;
+      bool ok = true;
+      for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
+        const Item it = decode_item<kDense>(idx, d, a);
+        EntryStream<kDense> rd;
+        rd.init(it, a);
+        if (it_count > 0) ok = mbar_wait(&s.q_free, (it_count - 1) & 1, abort_flag);
+        if (!ok) break;
         mbar_arrive_expect_tx(&s.q_full, it.tile1 ? 65536u : 32768u);
         tma_load_3d(s.q[0][0], &tmap_q, &s.q_full, 0, it.h, it.m0 * kBlock);
         tma_load_3d(s.q[0][1], &tmap_q, &s.q_full, 64, it.h, it.m0 * kBlock);
@@ -321,53 +352,55 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           tma_load_3d(s.q[1][0], &tmap_q, &s.q_full, 0, it.h, it.m1 * kBlock);
           tma_load_3d(s.q[1][1], &tmap_q, &s.q_full, 64, it.h, it.m1 * kBlock);
         }
-      }
-      for (int e = 0; e < it.n_entries; ++e, ++ecount) {
-        const uint32_t ent = rd.get(e, it.n_entries, lane);
-        const int J = static_cast<int>(ent & kColMask);
-        // loads 2*ecount (K) and 2*ecount + 1 (V) go to consecutive ring slots
+        for (int e = 0; e < it.n_entries && ok; ++e, ++ecount) {
+          const uint32_t ent = rd.get(e);
+          const int J = static_cast<int>(ent & kColMask);
+          // loads 2*ecount (K) and 2*ecount + 1 (V) go to consecutive ring slots
 #pragma unroll
-        for (int which = 0; which < 2; ++which) {
-          const uint32_t load = 2u * ecount + which;
-          const int slot = load % kStages;
-          const uint32_t use = load / kStages;
-          if (use > 0) ok = mbar_wait_lane0(&s.kv_empty[slot], (use - 1) & 1, abort_flag, lane);
-          if (!ok) break;
-          if (lane == 0) {
+          for (int which = 0; which < 2; ++which) {
+            const uint32_t load = 2u * ecount + which;
+            const int slot = load % kStages;
+            const uint32_t use = load / kStages;
+            if (use > 0) ok = mbar_wait(&s.kv_empty[slot], (use - 1) & 1, abort_flag);
+            if (!ok) break;
             const CUtensorMap* tmap = which == 0 ? &tmap_k : &tmap_v;
             mbar_arrive_expect_tx(&s.kv_full[slot], 32768u);
             tma_load_3d(s.kv[slot][0], tmap, &s.kv_full[slot], 0, it.kvh, J * kBlock);
             tma_load_3d(s.kv[slot][1], tmap, &s.kv_full[slot], 64, it.kvh, J * kBlock);
           }
         }
-        if (!ok) break;
       }
     }
+    __syncwarp();
   } else if (warp == 9) {
     // =============================================================== MMA issuer
-    reg_dealloc<56>();
+    reg_dealloc<kRegsOther>();
     constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 128, false, false);
     constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, false, true);
-    uint32_t ecount_base = 0;
-    uint32_t pv_count[2] = {0, 0};  // P-ready phases consumed per tile
-    int it_count = 0;
-    bool ok = true;
+    if (lane == 0) {
+      uint32_t ecount_base = 0;
+      uint32_t pv_count[2] = {0, 0};  // P-ready phases consumed per tile
+      int it_count = 0;
+      bool ok = true;
 
-    // Operand descriptors are built once; inside the loops only the 14-bit start-address field moves
-    // (a compile-time offset per K step), so issuing an MMA costs two integer adds.
-    const uint64_t q_desc[2] = {umma_desc_sw128(smem_u32(s.q[0][0]), 0, 1024),
-                                umma_desc_sw128(smem_u32(s.q[1][0]), 0, 1024)};
-    // slot s of the ring starts 32 KB after slot s - 1: +2048 in the descriptor's address field
-    const uint64_t k_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 0, 1024);      // K block: K-major B operand
-    const uint64_t v_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 16384, 1024);  // V block: MN-major B operand
+      // Operand descriptors are built once; inside the loops only the 14-bit start-address field moves
+      // (a compile-time offset per K step), so issuing an MMA costs two integer adds.
+      const uint64_t q_desc[2] = {umma_desc_sw128(smem_u32(s.q[0][0]), 0, 1024),
+                                  umma_desc_sw128(smem_u32(s.q[1][0]), 0, 1024)};
+      // slot s of the ring starts 32 KB after slot s - 1: +2048 in the descriptor's address field
+      const uint64_t k_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 0, 1024);      // K block: K-major B operand
+      const uint64_t v_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 16384, 1024);  // V block: MN-major B operand
+      uint32_t k_seen = 0xffffffffu, v_seen = 0xffffffffu;  // loads whose arrival has been observed already
 
-    auto issue_qk = [&](int t, uint32_t ecount, bool last_use, bool last_of_item) {
-      const uint32_t load = 2u * ecount;
-      const int st = load % kStages;
-      ok = ok && mbar_wait_lane0(&s.kv_full[st], (load / kStages) & 1, abort_flag, lane);
-      if (!ok) return;
-      tc_fence_after_sync();
-      if (lane == 0) {
+      auto issue_qk = [&](int t, uint32_t ecount, bool last_use, bool last_of_item) {
+        const uint32_t load = 2u * ecount;
+        const int st = load % kStages;
+        if (k_seen != load) {
+          ok = ok && mbar_wait(&s.kv_full[st], (load / kStages) & 1, abort_flag);
+          k_seen = load;
+        }
+        if (!ok) return;
+        tc_fence_after_sync();
         const uint64_t ad0 = q_desc[t], bd0 = k_desc0 + static_cast<uint64_t>(st) * 2048u;
         const uint32_t dst = tm + t * 128;
 #pragma unroll
@@ -380,88 +413,76 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         umma_commit(&s.s_full[t]);
         if (last_use) umma_commit(&s.kv_empty[st]);
         if (last_of_item) umma_commit(&s.q_free);
-      }
-      __syncwarp();
-    };
-    auto issue_pv = [&](int t, uint32_t ecount, bool last_use, bool first_of_tile) {
-      const uint32_t load = 2u * ecount + 1u;
-      const int st = load % kStages;
-      const uint64_t bd0 = v_desc0 + static_cast<uint64_t>(st) * 2048u;
-      const uint32_t dst = tm + 256 + t * 128, src = tm + t * 128;
-      // P arrives in two halves (keys 0-63, 64-127): the first four MMAs start while the softmax warps
-      // still work on the second half
-      ok = ok && mbar_wait_lane0(&s.p_ready[t][0], pv_count[t] & 1, abort_flag, lane);
-      ok = ok && mbar_wait_lane0(&s.kv_full[st], (load / kStages) & 1, abort_flag, lane);
-      if (!ok) return;
-      tc_fence_after_sync();
-      if (lane == 0) {
+      };
+      auto issue_pv = [&](int t, uint32_t ecount, bool last_use, bool first_of_tile) {
+        const uint32_t load = 2u * ecount + 1u;
+        const int st = load % kStages;
+        const uint64_t bd0 = v_desc0 + static_cast<uint64_t>(st) * 2048u;
+        const uint32_t dst = tm + 256 + t * 128, src = tm + t * 128;
+        ok = ok && mbar_wait(&s.p_ready[t], pv_count[t] & 1, abort_flag);
+        if (v_seen != load) {
+          ok = ok && mbar_wait(&s.kv_full[st], (load / kStages) & 1, abort_flag);
+          v_seen = load;
+        }
+        if (!ok) return;
+        ++pv_count[t];
+        tc_fence_after_sync();
 #pragma unroll
-        for (int kk = 0; kk < 4; ++kk) {
+        for (int kk = 0; kk < 8; ++kk) {
           // V block as the MN-major B operand: 16 keys per step = two groups of 8 key rows = 2048 B
           const uint64_t off = static_cast<uint64_t>(kk * (2048 >> 4));
           umma_ts(dst, src + kk * 8, bd0 + off, idesc_pv, (kk > 0 || !first_of_tile) ? 1u : 0u);
         }
-      }
-      if (kSplitP) ok = ok && mbar_wait_lane0(&s.p_ready[t][1], pv_count[t] & 1, abort_flag, lane);
-      if (!ok) return;
-      ++pv_count[t];
-      tc_fence_after_sync();
-      if (lane == 0) {
-#pragma unroll
-        for (int kk = 4; kk < 8; ++kk) {
-          const uint64_t off = static_cast<uint64_t>(kk * (2048 >> 4));
-          umma_ts(dst, src + kk * 8, bd0 + off, idesc_pv, 1u);
-        }
         umma_commit(&s.o_done[t]);
         if (last_use) umma_commit(&s.kv_empty[st]);
-      }
-      __syncwarp();
-    };
+      };
 
-    for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
-      const Item it = decode_item<kDense>(idx, d, a);
-      EntryReader<kDense> rd;
-      rd.init(it, a);
-      ok = mbar_wait_lane0(&s.q_full, it_count & 1, abort_flag, lane);
-      if (!ok) break;
-      // pending step whose P*V has not been issued yet
-      bool have_prev = false;
-      int prev_t = 0;
-      uint32_t prev_ec = 0;
-      bool prev_last_use = false, prev_first = false;
-      bool seen[2] = {false, false};
-      for (int e = 0; e < it.n_entries && ok; ++e) {
-        const uint32_t ent = rd.get(e, it.n_entries, lane);
-        const bool f0 = (ent & kFlag0) != 0, f1 = (ent & kFlag1) != 0;
-        const uint32_t ec = ecount_base + e;
-        for (int t = 0; t < 2; ++t) {
-          if (!(t == 0 ? f0 : f1)) continue;
-          const bool last_use = (t == 1) || !f1;
-          // the last step of an item is the diagonal block of its last tile
-          const bool last_of_item = (e == it.n_entries - 1) && last_use;
-          if (have_prev && prev_t != t) {
-            issue_qk(t, ec, last_use, last_of_item);
-            issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
-          } else if (have_prev) {
-            issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
-            issue_qk(t, ec, last_use, last_of_item);
-          } else {
-            issue_qk(t, ec, last_use, last_of_item);
+      for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
+        const Item it = decode_item<kDense>(idx, d, a);
+        EntryStream<kDense> rd;
+        rd.init(it, a);
+        ok = mbar_wait(&s.q_full, it_count & 1, abort_flag);
+        if (!ok) break;
+        // pending step whose P*V has not been issued yet
+        bool have_prev = false;
+        int prev_t = 0;
+        uint32_t prev_ec = 0;
+        bool prev_last_use = false, prev_first = false;
+        bool seen[2] = {false, false};
+        for (int e = 0; e < it.n_entries && ok; ++e) {
+          const uint32_t ent = rd.get(e);
+          const bool f0 = (ent & kFlag0) != 0, f1 = (ent & kFlag1) != 0;
+          const uint32_t ec = ecount_base + e;
+          for (int t = 0; t < 2; ++t) {
+            if (!(t == 0 ? f0 : f1)) continue;
+            const bool last_use = (t == 1) || !f1;
+            // the last step of an item is the diagonal block of its last tile
+            const bool last_of_item = (e == it.n_entries - 1) && last_use;
+            if (have_prev && prev_t != t) {
+              issue_qk(t, ec, last_use, last_of_item);
+              issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
+            } else if (have_prev) {
+              issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
+              issue_qk(t, ec, last_use, last_of_item);
+            } else {
+              issue_qk(t, ec, last_use, last_of_item);
+            }
+            have_prev = true;
+            prev_t = t;
+            prev_ec = ec;
+            prev_last_use = last_use;
+            prev_first = !seen[t];
+            seen[t] = true;
           }
-          have_prev = true;
-          prev_t = t;
-          prev_ec = ec;
-          prev_last_use = last_use;
-          prev_first = !seen[t];
-          seen[t] = true;
         }
+        if (have_prev && ok) issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
+        ecount_base += it.n_entries;
       }
-      if (have_prev && ok) issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
-      ecount_base += it.n_entries;
     }
+    __syncwarp();
   } else if (warp < 8) {
     // =============================================================== softmax / epilogue, one row per thread
-    reg_alloc<216>();
+    reg_alloc<kRegsSoftmax>();
     const int t = warp >> 2;                     // tile
     const int r = tid & 127;                     // row within the tile
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -521,21 +542,16 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           l_run *= f;
           m_used = m_new;
         }
-        float sum = 0.f;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          if (diag) {
-            sum += exp_pack_store<true>(x, half, r, d.scale_log2, m_used, s_addr);
-          } else {
-            sum += exp_pack_store<false>(x, half, r, d.scale_log2, m_used, s_addr);
-          }
-          if (kSplitP || half == 1) {
-            tmem_st_wait();
-            tc_fence_before_sync();
-            mbar_arrive(&s.p_ready[t][kSplitP ? half : 0]);
-          }
+        float sum;
+        if (diag) {
+          sum = exp_pack_store<true>(x, r, d.scale_log2, m_used, s_addr);
+        } else {
+          sum = exp_pack_store<false>(x, r, d.scale_log2, m_used, s_addr);
         }
         l_run += sum;
+        tmem_st_wait();
+        tc_fence_before_sync();
+        mbar_arrive(&s.p_ready[t]);
         first = false;
         ++step_count;
       }
@@ -568,7 +584,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
   }
   else {
-    reg_dealloc<56>();  // idle warps of the third warpgroup
+    reg_dealloc<kRegsOther>();  // idle warps of the third warpgroup
   }
   tc_fence_before_sync();
   __syncthreads();
