@@ -59,7 +59,8 @@ typedef struct crisp_params {
   int32_t sink_tokens;   /* w_sink: anchor keys j < w_sink (Eq. 2; paper value 128), 1..seq_len      */
   int32_t local_tokens;  /* w_local: anchor keys j >= n - w_local (Eq. 2; paper value 128)           */
   int32_t k_min_blocks;  /* minimum budget per direction in blocks (paper: 1024 tokens = 8), >= 0    */
-  int32_t selector;      /* 0 = noise floor alpha (Algorithm 3); 1 = cumulative gamma (Algorithm 6)  */
+  int32_t selector;      /* 0 = noise floor alpha (Algorithm 3); 1 = cumulative gamma (Algorithm 6);
+                            2 = median noise floor (Appendix H: median instead of mean of the middle blocks) */
   int32_t force_pattern; /* 0 = route by C_struct; 1 = every head VS; 2 = every head PE              */
   float tau;             /* tau_proxy: VS iff C_struct >= tau (paper 0.2)                            */
   float alpha;           /* noise-floor multiplier (paper 1.0 / 1.25), >= 0                          */

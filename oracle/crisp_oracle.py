@@ -142,6 +142,18 @@ def select_noise_floor(p: np.ndarray, alpha: float, k_min: int) -> Tuple[np.ndar
     return np.sort(stable_topk(p, k_d)), k_d, raw
 
 
+def select_median_floor(p: np.ndarray, alpha: float, k_min: int) -> Tuple[np.ndarray, int, int]:
+    """Appendix H variant: the floor is the MEDIAN mass of the non-retained blocks instead of their mean.
+
+    k_d = clip(#{p > alpha * median(p[1 : N_b-1])}, k_min, N_b); the rest is Algorithm 3 unchanged.
+    """
+    nb = p.shape[0]
+    med = float(np.median(p[1:nb - 1]))
+    raw = int(np.count_nonzero(p > alpha * med))
+    k_d = min(max(raw, k_min), nb)
+    return np.sort(stable_topk(p, k_d)), k_d, raw
+
+
 # ----------------------------------------------------------------------------------------
 # Algorithm 6, lines 4-5: cumulative-gamma budget (comparison selector)
 # ----------------------------------------------------------------------------------------
@@ -290,7 +302,8 @@ def head_pipeline(q_h: np.ndarray, k_h: np.ndarray, *, block: int = 128, sink_to
                   force_pattern: int = 0, scale: float | None = None) -> Dict:
     """Route one head and build its per-query-block key-block lists.
 
-    selector 0 = noise floor (Algorithm 3), 1 = cumulative gamma (Algorithm 6), VS heads only.
+    selector 0 = noise floor (Algorithm 3), 1 = cumulative gamma (Algorithm 6), 2 = median floor
+    (Appendix H); VS heads only.
     force_pattern 0 = by C_struct, 1 = VS, 2 = PE.
     """
     n = np.asarray(q_h).shape[0]
@@ -311,6 +324,9 @@ def head_pipeline(q_h: np.ndarray, k_h: np.ndarray, *, block: int = 128, sink_to
         if selector == 0:
             s_v, kv_, raw_v = select_noise_floor(p_v, alpha, k_min_blocks)
             s_s, ks_, raw_s = select_noise_floor(p_s, alpha, k_min_blocks)
+        elif selector == 2:
+            s_v, kv_, raw_v = select_median_floor(p_v, alpha, k_min_blocks)
+            s_s, ks_, raw_s = select_median_floor(p_s, alpha, k_min_blocks)
         else:
             s_v, kv_, raw_v = select_gamma(p_v, gamma, k_min_blocks)
             s_s, ks_, raw_s = select_gamma(p_s, gamma, k_min_blocks)

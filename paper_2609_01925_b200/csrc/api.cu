@@ -68,7 +68,7 @@ int validate(const crisp_params* p, Dims* d) {
   if (p->sink_tokens < 1 || p->sink_tokens > p->seq_len) return CRISP_ERR_INVALID_ARG;
   if (p->local_tokens < 1 || p->local_tokens > p->seq_len) return CRISP_ERR_INVALID_ARG;
   if (p->k_min_blocks < 0) return CRISP_ERR_INVALID_ARG;
-  if (p->selector < 0 || p->selector > 1) return CRISP_ERR_INVALID_ARG;
+  if (p->selector < 0 || p->selector > 2) return CRISP_ERR_INVALID_ARG;
   if (p->force_pattern < 0 || p->force_pattern > 2) return CRISP_ERR_INVALID_ARG;
   if (!(p->alpha >= 0.f) || !(p->gamma > 0.f) || !std::isfinite(p->tau) || !std::isfinite(p->alpha) ||
       !std::isfinite(p->gamma) || !(p->softmax_scale >= 0.f) || !std::isfinite(p->softmax_scale))

@@ -1,6 +1,7 @@
 // Stage 3b-3c: block selection and expansion into per-query-block key-block lists.
 //
-//   VS heads  (Algorithm 3 lines 6-12 / Eq. 3-4, or Algorithm 6 when selector == 1):
+//   VS heads  (Algorithm 3 lines 6-12 / Eq. 3-4; Algorithm 6 when selector == 1; the median floor of
+//     Appendix H when selector == 2):
 //     `select_vs_kernel`, one CTA per (head, direction), keeps p_d in shared memory, computes the
 //     noise floor, the budget k_d and the top-k_d set (ties to the lower index) as a bitmap.
 //   PE heads  (Algorithm 4): block means of Q and K (`pool_kernel`), pooled logits (`pe_logits_kernel`),
@@ -89,6 +90,7 @@ select_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const float*
   __shared__ float fscratch[32];
   __shared__ int iscratch[32];
   __shared__ int s_k;
+  __shared__ float s_med[2];
   const int h = blockIdx.x, dir = blockIdx.y, tid = threadIdx.x;
   uint32_t* out = dir == 0 ? w.selv + static_cast<size_t>(h) * w.words
                            : w.selsr + static_cast<size_t>(h) * (w.words + 2);
@@ -109,9 +111,27 @@ select_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const float*
     float part = 0.f;
     for (int i = 1 + tid; i < nb - 1; i += blockDim.x) part += p[i];
     const float r = block_sum<float>(part, fscratch);
-    const float mu = r / static_cast<float>(nb - 2);
+    float mu = r / static_cast<float>(nb - 2);
+    if (d.selector == 2) {
+      // median of the middle blocks instead of their mean (Appendix H): the two central order statistics
+      // are found by ranking the middle blocks among themselves
+      const int n_mid = nb - 2;
+      const int lo_rank = n_mid - 1 - (n_mid - 1) / 2, hi_rank = n_mid - 1 - n_mid / 2;  // descending ranks
+      for (int e = 1 + tid; e < nb - 1; e += blockDim.x) {
+        const float pe = p[e];
+        int rank = 0;
+        for (int j = 1; j < nb - 1; ++j) {
+          const float pj = p[j];
+          rank += (pj > pe || (pj == pe && j < e)) ? 1 : 0;
+        }
+        if (rank == lo_rank) s_med[0] = pe;
+        if (rank == hi_rank) s_med[1] = pe;
+      }
+      __syncthreads();
+      mu = 0.5f * (s_med[0] + s_med[1]);
+    }
     thr = d.alpha * mu;
-    if (d.selector == 0) {
+    if (d.selector == 0 || d.selector == 2) {
       int c = 0;
       for (int i = tid; i < nb; i += blockDim.x) c += (p[i] > thr) ? 1 : 0;
       const int cnt = block_sum<int>(c, iscratch);
@@ -324,8 +344,16 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
           fixed = __float2ull_rn(v * kMassScale);
         }
       }
-      // Neighbouring entries of a flat map fall into a handful of bins: lanes with the same bin elect a
+      // Level 0: neighbouring entries of a flat map fall into a handful of bins: lanes with the same bin elect a
       // leader and add their counts and masses (three 20-bit limbs, summed exactly) in one atomic each.
+      if (level > 0) {
+        // lower levels: the 11 / 9 bits below the fixed prefix spread the entries over many bins
+        if (bin >= 0) {
+          atomicAdd(&cnt[bin], 1u);
+          atomicAdd(&mass[bin], fixed);
+        }
+        continue;
+      }
       const unsigned int peers = __match_any_sync(0xffffffffu, bin);
       const unsigned int l0 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed & 0xFFFFFull));
       const unsigned int l1 = __reduce_add_sync(peers, static_cast<unsigned int>((fixed >> 20) & 0xFFFFFull));

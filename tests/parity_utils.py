@@ -85,8 +85,8 @@ def _ambiguous_vs(pd, p, k_d, raw):
     nb = pd.shape[0]
     order = np.argsort(-pd, kind="stable")
     amb = np.zeros(nb, dtype=bool)
-    if p.selector == 0:
-        _, mu = orc.noise_floor(pd)
+    if p.selector in (0, 2):
+        mu = orc.noise_floor(pd)[1] if p.selector == 0 else float(np.median(pd[1:nb - 1]))
         thr = p.alpha * mu
         amb |= np.abs(pd - thr) <= REL_BAND * thr
     if p.selector == 1 and raw < nb:

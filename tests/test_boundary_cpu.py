@@ -58,7 +58,7 @@ def test_workspace_sizes_grow_with_the_problem():
     (dict(sink_tokens=0), B.ERR_INVALID_ARG),
     (dict(local_tokens=10 ** 7), B.ERR_INVALID_ARG),
     (dict(k_min_blocks=-1), B.ERR_INVALID_ARG),
-    (dict(selector=2), B.ERR_INVALID_ARG),
+    (dict(selector=3), B.ERR_INVALID_ARG),
     (dict(force_pattern=3), B.ERR_INVALID_ARG),
     (dict(alpha=-1.0), B.ERR_INVALID_ARG),
     (dict(gamma=0.0), B.ERR_INVALID_ARG),

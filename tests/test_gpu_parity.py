@@ -93,6 +93,16 @@ def test_gamma_selector():
     _full_check(w, p=pu.params_of(w, selector=1, gamma=0.5), per_head=4, dense=False)
 
 
+def test_median_floor_selector():
+    """selector 2: the median noise floor of Appendix H (even and odd numbers of middle blocks)."""
+    pu = _pu()
+    for n in (4096, 4224):
+        w = synth.tiny(n=n)
+        _full_check(w, p=pu.params_of(w, selector=2), per_head=4, dense=False)
+    w = synth.tiny(n=4096).with_(alpha=1e6, k_min_blocks=5)
+    _full_check(w, p=pu.params_of(w, selector=2), per_head=2, dense=False)
+
+
 @pytest.mark.parametrize("force", [1, 2])
 def test_forced_patterns(force):
     pu = _pu()

@@ -209,6 +209,38 @@ def test_noise_floor_hand_worked_example():
         assert list(s) == want and k_d == raw == len(want)
 
 
+def test_median_floor_hand_worked_example_and_properties():
+    """Appendix H: the floor is the median of the non-retained blocks."""
+    p = None
+    sets = {}
+    with open(os.path.join(GOLDEN, "noise_floor_toy.txt")) as f:
+        for line in f:
+            tok = line.split()
+            if tok and tok[0] == "p":
+                p = np.array([float(x) for x in tok[1:]])
+            elif tok and tok[0] == "median_alpha":
+                sets[float(tok[1])] = [int(x) for x in tok[3:]]
+    assert len(sets) == 3
+    for alpha, want in sets.items():
+        s, k_d, raw = orc.select_median_floor(p, alpha, k_min=0)
+        assert list(s) == want and k_d == raw == len(want)
+    # a single dominant middle block lifts the mean floor above weaker signal but not the median floor
+    q = np.array([0.5, 0.3, 0.004, 0.004, 0.004, 0.001, 0.001, 0.001, 0.001, 0.184])
+    mean_set = set(orc.select_noise_floor(q, 1.0, 0)[0])
+    med_set = set(orc.select_median_floor(q, 1.0, 0)[0])
+    assert mean_set == {0, 1, 9} and med_set == {0, 1, 2, 3, 4, 9}
+    # odd and even numbers of middle blocks; monotone in alpha; k_min fill
+    r_ = rng(21)
+    for nb in (7, 8, 33):
+        x = r_.dirichlet(np.ones(nb) * 0.4)
+        srt = np.sort(x[1:-1])
+        med = srt[(nb - 2) // 2] if (nb - 2) % 2 else 0.5 * (srt[(nb - 2) // 2 - 1] + srt[(nb - 2) // 2])
+        s1 = set(orc.select_median_floor(x, 1.0, 0)[0])
+        assert s1 == set(np.nonzero(x > med)[0])
+        assert set(orc.select_median_floor(x, 2.0, 0)[0]) <= s1 <= set(orc.select_median_floor(x, 0.5, 0)[0])
+        assert orc.select_median_floor(x, 1e9, 3)[1] == 3
+
+
 def test_noise_floor_literal_formula():
     """r = max(1 - p[0] - p[N_b-1], 0) as printed in Algorithm 3 line 6."""
     r_ = rng(6)
