@@ -166,6 +166,24 @@ int crisp_dense_prefill(const crisp_params* p, const void* q, const void* k, con
                         size_t ws_bytes, void* o, float* lse, void* cuda_stream);
 
 /*
+ * Algorithm 1 in one call, with the context-length gate the paper recommends for deployments that serve
+ * short prompts (Section 5.3, "Short contexts": routing is a fixed per-head cost that dominates what it
+ * saves below some length).
+ *   seq_len <  dense_below_tokens : crisp_dense_prefill only; the routing / selection outputs are not
+ *                                   written and their pointers (and route_ws, select_ws) may be NULL.
+ *   seq_len >= dense_below_tokens : crisp_route, crisp_select, crisp_sparse_prefill, enqueued back to back
+ *                                   on the stream with no host synchronisation in between.
+ * If the selected lists do not fit `capacity`, the attention kernels see the CRISP_ERR_CAPACITY word of
+ * select_ws on the device and do nothing (O is left untouched); crisp_poll_device_status(select_ws)
+ * reports it.  dense_below_tokens <= 0 disables the gate.  Arguments as in the staged calls.
+ */
+int crisp_forward(const crisp_params* p, const void* q, const void* k, const void* v, void* route_ws,
+                  size_t route_ws_bytes, void* select_ws, size_t select_ws_bytes, void* prefill_ws,
+                  size_t prefill_ws_bytes, float* c_struct, int32_t* pattern, float* p_v, float* p_s,
+                  int64_t* row_ptr, int32_t* col_idx, int64_t capacity, int64_t* nnz_needed, void* o, float* lse,
+                  int32_t dense_below_tokens, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, reads the status word at the start of `ws`, clears it and returns it
  * (CRISP_OK, CRISP_ERR_CAPACITY or CRISP_ERR_DEVICE_TIMEOUT), or CRISP_ERR_CUDA if the stream failed.
  */

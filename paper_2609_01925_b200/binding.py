@@ -27,7 +27,7 @@ PATTERN_PE, PATTERN_VS = 0, 1
 EXPORTS = (
     "crisp_version", "crisp_status_string", "crisp_last_cuda_error", "crisp_workspace_bytes",
     "crisp_route", "crisp_route_static", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
-    "crisp_poll_device_status",
+    "crisp_poll_device_status", "crisp_forward",
 )
 
 
@@ -93,6 +93,9 @@ def load() -> ctypes.CDLL:
     lib.crisp_sparse_prefill.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp, vp]
     lib.crisp_dense_prefill.restype = ctypes.c_int
     lib.crisp_dense_prefill.argtypes = [P, vp, vp, vp, vp, sz, vp, vp, vp]
+    lib.crisp_forward.restype = ctypes.c_int
+    lib.crisp_forward.argtypes = [P, vp, vp, vp, vp, sz, vp, sz, vp, sz, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp,
+                                  ctypes.c_int32, vp]
     lib.crisp_poll_device_status.restype = ctypes.c_int
     lib.crisp_poll_device_status.argtypes = [vp, vp]
     _lib = lib
@@ -162,6 +165,19 @@ def crisp_sparse_prefill(p, q, k, v, row_ptr, col_idx, ws, o, lse=None, stream=N
 def crisp_dense_prefill(p, q, k, v, ws, o, lse=None, stream=None) -> int:
     return load().crisp_dense_prefill(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(ws),
                                       ws.numel() * ws.element_size(), _ptr(o), _ptr(lse), _stream(stream))
+
+
+def _nbytes(t) -> int:
+    return 0 if t is None else t.numel() * t.element_size()
+
+
+def crisp_forward(p, q, k, v, route_ws, select_ws, prefill_ws, c_struct, pattern, p_v, p_s, row_ptr, col_idx,
+                  capacity, nnz_needed, o, lse=None, dense_below_tokens=0, stream=None) -> int:
+    return load().crisp_forward(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(route_ws), _nbytes(route_ws),
+                                _ptr(select_ws), _nbytes(select_ws), _ptr(prefill_ws), _nbytes(prefill_ws),
+                                _ptr(c_struct), _ptr(pattern), _ptr(p_v), _ptr(p_s), _ptr(row_ptr),
+                                _ptr(col_idx), int(capacity), _ptr(nnz_needed), _ptr(o), _ptr(lse),
+                                int(dense_below_tokens), _stream(stream))
 
 
 def crisp_poll_device_status(ws, stream=None) -> int:

@@ -194,6 +194,35 @@ int crisp_dense_prefill(const crisp_params* p, const void* q, const void* k, con
   return launch_prefill(d, q, k, v, nullptr, nullptr, ws, o, lse, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int crisp_forward(const crisp_params* p, const void* q, const void* k, const void* v, void* route_ws,
+                  size_t route_ws_bytes_, void* select_ws, size_t select_ws_bytes_, void* prefill_ws,
+                  size_t prefill_ws_bytes_, float* c_struct, int32_t* pattern, float* p_v, float* p_s,
+                  int64_t* row_ptr, int32_t* col_idx, int64_t capacity, int64_t* nnz_needed, void* o, float* lse,
+                  int32_t dense_below_tokens, void* cuda_stream) {
+  Dims d;
+  int rc = validate(p, &d);
+  if (rc != CRISP_OK) return rc;
+  if (!q || !k || !v || !o || !prefill_ws) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(prefill_ws) || prefill_ws_bytes_ < prefill_ws_bytes(d)) return CRISP_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (d.n < dense_below_tokens) {
+    // short prompt: routing and selection would cost more than they save
+    return launch_prefill(d, q, k, v, nullptr, nullptr, prefill_ws, o, lse, st);
+  }
+  if (!route_ws || !select_ws || !c_struct || !pattern || !p_v || !p_s || !row_ptr || !nnz_needed)
+    return CRISP_ERR_INVALID_ARG;
+  if (capacity < 0 || (capacity > 0 && !col_idx)) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(route_ws) || route_ws_bytes_ < route_ws_bytes(d)) return CRISP_ERR_WORKSPACE;
+  if (!aligned16(select_ws) || select_ws_bytes_ < select_ws_bytes(d)) return CRISP_ERR_WORKSPACE;
+  rc = launch_route(d, q, k, route_ws, c_struct, pattern, p_v, p_s, st);
+  if (rc != CRISP_OK) return rc;
+  rc = launch_select(d, q, k, pattern, p_v, p_s, select_ws, row_ptr, col_idx, capacity, nnz_needed, st);
+  if (rc != CRISP_OK) return rc;
+  // the status word of the selection stage gates the attention kernels: lists that did not fit are never read
+  return launch_prefill(d, q, k, v, row_ptr, col_idx, prefill_ws, o, lse, st, static_cast<const int*>(select_ws));
+}
+
 int crisp_poll_device_status(void* ws, void* cuda_stream) {
   if (!ws) return CRISP_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

@@ -59,7 +59,8 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
                   int64_t* nnz_needed, cudaStream_t stream);
 size_t select_ws_bytes(const Dims& d);
 int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, const int64_t* row_ptr,
-                   const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream);
+                   const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream,
+                   const int* gate = nullptr);
 size_t prefill_ws_bytes(const Dims& d);
 
 }  // namespace crisp

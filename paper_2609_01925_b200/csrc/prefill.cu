@@ -42,6 +42,7 @@ struct PrefillArgs {
   int n_pairs;
   int n_items;
   int group_kv;            // 1: schedule one KV head at a time (K/V larger than L2), 0: one global order
+  const int* gate;         // optional device word: when non-zero the lists are invalid and nothing is done
 };
 
 struct PrefillSmem {
@@ -323,6 +324,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   tc_fence_after_sync();
   const uint32_t tm = s.tmem_base;
   volatile int* abort_flag = &s.abort_flag;
+  const int n_items = (a.gate != nullptr && *a.gate != 0) ? 0 : a.n_items;
 
   // Register budget: the two softmax warpgroups hold a full 128-column row of S per thread; the third
   // warpgroup (producer, issuer, two idle warps) needs very few registers and gives the rest away.
@@ -339,7 +341,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       uint32_t ecount = 0;
       int it_count = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
+      for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x, ++it_count) {
         const Item it = decode_item<kDense>(idx, d, a);
         EntryStream<kDense> rd;
         rd.init(it, a);
@@ -437,7 +439,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (last_use) umma_commit(&s.kv_empty[st]);
       };
 
-      for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x, ++it_count) {
+      for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x, ++it_count) {
         const Item it = decode_item<kDense>(idx, d, a);
         EntryStream<kDense> rd;
         rd.init(it, a);
@@ -490,7 +492,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const uint32_t o_addr = tm + lane_addr + 256 + t * 128;
     uint32_t step_count = 0;  // steps of this tile so far (all items): phase of s_full / o_done
     bool ok = true;
-    for (int idx = blockIdx.x; idx < a.n_items && ok; idx += gridDim.x) {
+    for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
       const Item it = decode_item<kDense>(idx, d, a);
       if (t == 1 && !it.tile1) continue;
       EntryReader<kDense> rd;
@@ -597,8 +599,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 __global__ void __launch_bounds__(128)
 merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                    int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
-                   int n_pairs, int n_cost, int group_kv) {
+                   int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate) {
   extern __shared__ uint32_t bm[];
+  if (gate != nullptr && *gate != 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
   const int words = (d.nb + 31) / 32;
@@ -677,9 +680,10 @@ __global__ void __launch_bounds__(1024) sched_scan_kernel(int* __restrict__ cost
 
 __global__ void __launch_bounds__(256)
 sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, int* __restrict__ cost_hist,
-                     int* __restrict__ order, int n_pairs, int n_cost, int group_kv) {
+                     int* __restrict__ order, int n_pairs, int n_cost, int group_kv,
+                     const int* __restrict__ gate) {
   const int u = blockIdx.x * blockDim.x + threadIdx.x, h = blockIdx.y;
-  if (u >= n_pairs) return;
+  if (u >= n_pairs || (gate != nullptr && *gate != 0)) return;
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int m0 = 2 * u, mend = min(2 * u + 2, d.nb);
   const int cost = static_cast<int>(rp[mend] - rp[m0]);
@@ -724,7 +728,7 @@ size_t prefill_ws_bytes(const Dims& d) {
 }
 
 int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, const int64_t* row_ptr,
-                   const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream) {
+                   const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream, const int* gate) {
   const bool dense = (row_ptr == nullptr);
   size_t total;
   PrefillWs w = carve(d, ws, &total);
@@ -745,6 +749,7 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
   a.status = static_cast<int*>(ws);
+  a.gate = gate;
   // K + V of all KV heads against the 126 MB L2: group the schedule by KV head only when they do not fit
   a.group_kv = (static_cast<size_t>(d.n) * d.hkv * kHeadDim * 2 * 2 > (256u << 20)) ? 1 : 0;
 
@@ -762,10 +767,10 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
     const int words = (d.nb + 31) / 32;
     CRISP_CUDA_TRY(cudaMemsetAsync(w.cost_hist, 0, sizeof(int) * w.n_bins, stream), "prefill: clear histogram");
     merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
-        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv);
+        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate);
     sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins);
     sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, 0, stream>>>(d, row_ptr, w.cost_hist,
-                                                                               w.order, a.n_pairs, w.n_cost, a.group_kv);
+                                                                               w.order, a.n_pairs, w.n_cost, a.group_kv, gate);
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");

@@ -58,11 +58,12 @@ class CrispLayer:
         B.check(B.crisp_dense_prefill(self.p, q, k, v, self.prefill_ws, self.o, self.lse, stream),
                 "crisp_dense_prefill")
 
-    def forward(self, q, k, v, stream=None):
-        """Algorithm 1: route, select, sparse attention.  Returns O [n, H_q, 128] bf16."""
-        self.route(q, k, stream)
-        self.select(q, k, stream)
-        self.sparse_prefill(q, k, v, stream)
+    def forward(self, q, k, v, stream=None, dense_below_tokens: int = 0):
+        """Algorithm 1 through crisp_forward (one C call: route, select, sparse attention, or the dense
+        kernel when seq_len < dense_below_tokens).  Returns O [n, H_q, 128] bf16."""
+        B.check(B.crisp_forward(self.p, q, k, v, self.route_ws, self.select_ws, self.prefill_ws, self.c_struct,
+                                self.pattern, self.p_v, self.p_s, self.row_ptr, self.col_idx, self.capacity,
+                                self.nnz, self.o, self.lse, dense_below_tokens, stream), "crisp_forward")
         return self.o
 
     def poll(self, stream=None):
