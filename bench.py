@@ -94,7 +94,7 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(w, q, k, v, seed=0, budget_blocks=6):
+def oracle_sample(w, q, k, v, seed=0, blocks_per_head=4):
     """Times the fp64 oracle (as it stands) on a bounded sample of the workload and extrapolates to
     ms/layer: route+select of two heads (one per class) scaled to H_q, attention of a few query
     blocks scaled by the number of listed blocks.  Returns (ms_per_layer, description, cores)."""
@@ -119,7 +119,7 @@ def oracle_sample(w, q, k, v, seed=0, budget_blocks=6):
         nnz_est += lens.sum() * (sum(1 for c in w.head_classes if c == w.head_classes[h]))
         # a few query blocks, kept small enough for a bounded run
         order = np.argsort(lens)
-        picks = [int(order[len(order) // 4]), int(order[len(order) // 2])][:max(1, budget_blocks // 4)]
+        picks = [int(order[(2 * i + 1) * len(order) // (2 * blocks_per_head)]) for i in range(blocks_per_head)]
         for m in picks:
             t0 = time.perf_counter()
             orc.sparse_attention_block(qh, kh, vh, m, res["cols"][m], 128)
