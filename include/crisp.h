@@ -51,7 +51,7 @@ typedef enum crisp_status {
 /* Problem description: the inputs of Algorithm 1 plus the constants of Sections 3.2 and 4.3. */
 typedef struct crisp_params {
   int32_t struct_size;   /* = sizeof(crisp_params); ABI guard                                        */
-  int32_t seq_len;       /* n; a multiple of `block`, at least 2 * block                             */
+  int32_t seq_len;       /* n; a multiple of `block`, 2 * block <= n <= 8192 * block (1,048,576)     */
   int32_t n_q_heads;     /* H_q                                                                      */
   int32_t n_kv_heads;    /* H_kv; H_q % H_kv == 0 and H_q / H_kv <= 16                               */
   int32_t head_dim;      /* 128 only                                                                 */

@@ -76,7 +76,7 @@ int validate(const crisp_params* p, Dims* d) {
   if (p->head_dim != kHeadDim || p->block != kBlock) return CRISP_ERR_UNSUPPORTED;
   if (p->seq_len % kBlock != 0 || p->seq_len < 2 * kBlock) return CRISP_ERR_UNSUPPORTED;
   if (p->n_q_heads / p->n_kv_heads > kMaxGroup) return CRISP_ERR_UNSUPPORTED;
-  if (p->seq_len / kBlock > 16384) return CRISP_ERR_UNSUPPORTED;  // N_b limit of the selection kernels
+  if (p->seq_len / kBlock > 8192) return CRISP_ERR_UNSUPPORTED;  // N_b limit of the selection kernels (1M tokens)
   d->n = p->seq_len;
   d->nb = p->seq_len / kBlock;
   d->hq = p->n_q_heads;

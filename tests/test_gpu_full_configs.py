@@ -152,3 +152,41 @@ def test_config_Q256k():
 
 def test_config_L512k():
     _config_check("L512k", pe_heads_default=1, blocks_default=3, blocks_full=64)
+
+
+def test_maximum_block_count_one_million_tokens():
+    """N_b = 8192 (the selection kernels' limit): 1,048,576 tokens, 2 query heads on 1 KV head."""
+    pu = _pu()
+    import paper_2609_01925_b200 as crisp
+    from paper_2609_01925_b200 import binding as B
+    n = 8192 * 128
+    w = synth.llama_shaped("M1M", n, 64).with_(n_q_heads=2, n_kv_heads=1, head_classes=("conc", "diffuse"))
+    p = pu.params_of(w, force_pattern=1)
+    q, k, v = synth.make_qkv(w, device="cuda", chunk_tokens=65536)
+    layer = crisp.CrispLayer(p, with_lse=True)
+    layer.forward(q, k, v)
+    layer.poll()
+    torch.cuda.synchronize()
+    nnz = int(layer.nnz.item())
+    g = dict(c_struct=layer.c_struct.cpu().numpy(), pattern=layer.pattern.cpu().numpy(),
+             p_v=layer.p_v.cpu().numpy(), p_s=layer.p_s.cpu().numpy(), row_ptr=layer.row_ptr.cpu().numpy(),
+             col_idx=layer.col_idx[:nnz].cpu().numpy(), nnz=nnz, lse=layer.lse.cpu().numpy())
+    qc, kc, vc = q.cpu(), k.cpu(), v.cpu()
+    res = _oracle_heads(qc, kc, p, [0, 1], pu)
+    pu.check_route(g, res, p)
+    excused = pu.check_lists(g, res, p)
+    nb = w.n_blocks
+    samples = [(0, 0), (0, nb - 1), (0, 5000), (1, nb - 1), (1, 1234)]
+    o_host = {(h, m): layer.o[m * 128:(m + 1) * 128, h].float().cpu().numpy() for h, m in samples}
+
+    class _O:
+        def __getitem__(self, idx):
+            rows, h = idx
+            return o_host[(h, rows.start // 128)]
+    g["o"] = _O()
+    rel, mab = pu.check_attention(g, qc, kc, vc, p, samples)
+    print(f"M1M: nnz {nnz}, excused blocks {excused}, rel-L2 {rel:.2e}, max-abs {mab:.2e}")
+    # one block more is refused on the host
+    p2 = crisp.make_params(n + 128, 2, 1)
+    assert B.load().crisp_select(__import__("ctypes").byref(p2), 1, 1, 1, 1, 1, 1, 1 << 40, 1, 1, 1, 1, None) \
+        in (B.ERR_UNSUPPORTED, B.ERR_INVALID_ARG, B.ERR_WORKSPACE)
