@@ -166,6 +166,18 @@ int crisp_dense_prefill(const crisp_params* p, const void* q, const void* k, con
                         size_t ws_bytes, void* o, float* lse, void* cuda_stream);
 
 /*
+ * Comparison router (Algorithm 5, the FlexPrefill rule that C_struct replaces): the Jensen-Shannon distance
+ *   jsd[h] = sqrt( 0.5 KL(a_hat || m) + 0.5 KL(a_bar || m) ),  m = (a_hat + a_bar) / 2,
+ * between the per-query mean a_hat (= p_v of crisp_route, the block masses of the proxy map) and the pooled
+ * estimate a_bar = Softmax(mean(Q_hat) . mean_block(K)^T * scale) over the N_b key blocks; natural logarithm,
+ * terms of zero probability contribute 0.  pattern[h] = VS iff jsd[h] >= tau_jsd.  Not on the CRISP path: it
+ * exists to measure how often the two routers agree.  Uses select_ws as scratch (block means of K), so it must
+ * not overlap in time with crisp_select on the same workspace.  jsd [H_q] f32, pattern [H_q] i32.
+ */
+int crisp_route_jsd(const crisp_params* p, const void* q, const void* k, const float* p_v, void* select_ws,
+                    size_t select_ws_bytes, float tau_jsd, float* jsd, int32_t* pattern, void* cuda_stream);
+
+/*
  * Algorithm 1 in one call, with the context-length gate the paper recommends for deployments that serve
  * short prompts (Section 5.3, "Short contexts": routing is a fixed per-head cost that dominates what it
  * saves below some length).

@@ -87,6 +87,37 @@ def route(c: float, tau: float) -> int:
 
 
 # ----------------------------------------------------------------------------------------
+# Algorithm 5 (Appendix A): the Jensen-Shannon router that C_struct replaces (comparison only)
+# ----------------------------------------------------------------------------------------
+def js_distance(a: np.ndarray, b: np.ndarray) -> float:
+    """sqrt(0.5 KL(a || m) + 0.5 KL(b || m)), m = (a + b) / 2; natural log, 0 log 0 = 0."""
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    m = 0.5 * (a + b)
+    kl_a = np.sum(np.where(a > 0, a * np.log(np.where(a > 0, a, 1.0) / np.where(m > 0, m, 1.0)), 0.0))
+    kl_b = np.sum(np.where(b > 0, b * np.log(np.where(b > 0, b, 1.0) / np.where(m > 0, m, 1.0)), 0.0))
+    return float(math.sqrt(max(0.5 * kl_a + 0.5 * kl_b, 0.0)))
+
+
+def jsd_router(q_h: np.ndarray, k_h: np.ndarray, block: int, scale: float | None = None) -> Tuple[float, np.ndarray, np.ndarray]:
+    """(D_JS, a_bar, a_hat): a_bar = Softmax(pool(Q_hat) pool(K)^T / sqrt(d)) over the key blocks
+    (pool = mean over the block's rows), a_hat = block sums of the mean proxy row (= p_v)."""
+    q_h = np.asarray(q_h, dtype=np.float64)
+    k_h = np.asarray(k_h, dtype=np.float64)
+    n, d = k_h.shape
+    nb = n // block
+    if scale is None:
+        scale = 1.0 / math.sqrt(d)
+    q_bar = q_h[n - block:].mean(axis=0)
+    k_bar = k_h.reshape(nb, block, d).mean(axis=1)
+    z = (k_bar @ q_bar) * scale
+    e = np.exp(z - z.max())
+    a_bar = e / e.sum()
+    a_hat, _ = block_scores(proxy_attention(q_h, k_h, block, scale), block)
+    return js_distance(a_hat, a_bar), a_bar, a_hat
+
+
+# ----------------------------------------------------------------------------------------
 # Algorithm 3, lines 3-5 (normalisation as in Algorithm 6, lines 2-3): block scores
 # ----------------------------------------------------------------------------------------
 def block_scores(a_hat: np.ndarray, block: int) -> Tuple[np.ndarray, np.ndarray]:

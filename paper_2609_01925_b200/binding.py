@@ -27,7 +27,7 @@ PATTERN_PE, PATTERN_VS = 0, 1
 EXPORTS = (
     "crisp_version", "crisp_status_string", "crisp_last_cuda_error", "crisp_workspace_bytes",
     "crisp_route", "crisp_route_static", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
-    "crisp_poll_device_status", "crisp_forward",
+    "crisp_poll_device_status", "crisp_forward", "crisp_route_jsd",
 )
 
 
@@ -93,6 +93,8 @@ def load() -> ctypes.CDLL:
     lib.crisp_sparse_prefill.argtypes = [P, vp, vp, vp, vp, vp, vp, sz, vp, vp, vp]
     lib.crisp_dense_prefill.restype = ctypes.c_int
     lib.crisp_dense_prefill.argtypes = [P, vp, vp, vp, vp, sz, vp, vp, vp]
+    lib.crisp_route_jsd.restype = ctypes.c_int
+    lib.crisp_route_jsd.argtypes = [P, vp, vp, vp, vp, sz, ctypes.c_float, vp, vp, vp]
     lib.crisp_forward.restype = ctypes.c_int
     lib.crisp_forward.argtypes = [P, vp, vp, vp, vp, sz, vp, sz, vp, sz, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp,
                                   ctypes.c_int32, vp]
@@ -165,6 +167,12 @@ def crisp_sparse_prefill(p, q, k, v, row_ptr, col_idx, ws, o, lse=None, stream=N
 def crisp_dense_prefill(p, q, k, v, ws, o, lse=None, stream=None) -> int:
     return load().crisp_dense_prefill(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(ws),
                                       ws.numel() * ws.element_size(), _ptr(o), _ptr(lse), _stream(stream))
+
+
+def crisp_route_jsd(p, q, k, p_v, select_ws, tau_jsd, jsd, pattern, stream=None) -> int:
+    return load().crisp_route_jsd(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(p_v), _ptr(select_ws),
+                                  select_ws.numel() * select_ws.element_size(), float(tau_jsd), _ptr(jsd),
+                                  _ptr(pattern), _stream(stream))
 
 
 def _nbytes(t) -> int:

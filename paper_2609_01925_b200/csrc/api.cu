@@ -194,6 +194,18 @@ int crisp_dense_prefill(const crisp_params* p, const void* q, const void* k, con
   return launch_prefill(d, q, k, v, nullptr, nullptr, ws, o, lse, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int crisp_route_jsd(const crisp_params* p, const void* q, const void* k, const float* p_v, void* select_ws,
+                    size_t select_ws_bytes_, float tau_jsd, float* jsd, int32_t* pattern, void* cuda_stream) {
+  Dims d;
+  int rc = validate(p, &d);
+  if (rc != CRISP_OK) return rc;
+  if (!q || !k || !p_v || !select_ws || !jsd || !pattern) return CRISP_ERR_INVALID_ARG;
+  if (!std::isfinite(tau_jsd)) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k)) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(select_ws) || select_ws_bytes_ < select_ws_bytes(d)) return CRISP_ERR_WORKSPACE;
+  return launch_route_jsd(d, q, k, p_v, select_ws, tau_jsd, jsd, pattern, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int crisp_forward(const crisp_params* p, const void* q, const void* k, const void* v, void* route_ws,
                   size_t route_ws_bytes_, void* select_ws, size_t select_ws_bytes_, void* prefill_ws,
                   size_t prefill_ws_bytes_, float* c_struct, int32_t* pattern, float* p_v, float* p_s,

@@ -58,6 +58,8 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
                   const float* p_s, void* ws, int64_t* row_ptr, int32_t* col_idx, int64_t capacity,
                   int64_t* nnz_needed, cudaStream_t stream);
 size_t select_ws_bytes(const Dims& d);
+int launch_route_jsd(const Dims& d, const void* q, const void* k, const float* p_v, void* ws, float tau_jsd,
+                     float* jsd, int32_t* pattern, cudaStream_t stream);
 int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, const int64_t* row_ptr,
                    const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream,
                    const int* gate = nullptr);

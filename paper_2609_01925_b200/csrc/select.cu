@@ -202,7 +202,9 @@ __global__ void __launch_bounds__(128)
 pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is_query,
             const int32_t* __restrict__ pattern, float* __restrict__ out) {
   const int J = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
-  if (is_query) {
+  if (pattern == nullptr) {
+    // comparison router: every head's block means are wanted
+  } else if (is_query) {
     if (pattern[h] != CRISP_PATTERN_PE) return;
   } else {
     bool any = false;
@@ -704,6 +706,101 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   fill_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w, row_ptr, col_idx, capacity,
                                                               nnz_needed);
   CRISP_CUDA_TRY(cudaGetLastError(), "select: launch");
+  return CRISP_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Comparison router (Algorithm 5): Jensen-Shannon distance between the pooled estimate
+//   a_bar = Softmax(pool(Q_hat) pool(K)^T / sqrt(d))      (one row over the N_b key blocks)
+// and the per-query mean a_hat = sumpool(Softmax(Q_hat K^T / sqrt(d))) = p_v from crisp_route.
+// ------------------------------------------------------------------------------------------------
+namespace {
+__global__ void __launch_bounds__(256)
+jsd_kernel(const Dims d, const __nv_bfloat16* __restrict__ q, const float* __restrict__ kbar,
+           const float* __restrict__ p_v, float tau_jsd, float* __restrict__ jsd, int32_t* __restrict__ pattern) {
+  extern __shared__ float z[];  // [nb] pooled logits, then a_bar
+  __shared__ float qbar[kHeadDim];
+  __shared__ float fscratch[32];
+  const int h = blockIdx.x, tid = threadIdx.x;
+  // mean of the last block's queries: thread pair (dim pair, half of the rows)
+  {
+    const int pair = tid & 63, part = tid >> 6;  // 4 parts of 32 rows
+    const __nv_bfloat162* base = reinterpret_cast<const __nv_bfloat162*>(
+        q + (static_cast<size_t>(d.n - kBlock) + part * 32) * d.hq * kHeadDim + static_cast<size_t>(h) * kHeadDim);
+    float a0 = 0.f, a1 = 0.f;
+    for (int t = 0; t < 32; ++t) {
+      const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * d.hq * (kHeadDim / 2) + pair]);
+      a0 += v.x;
+      a1 += v.y;
+    }
+    __shared__ float2 parts[4][64];
+    parts[part][pair] = make_float2(a0, a1);
+    __syncthreads();
+    if (tid < 64) {
+      float2 s0 = parts[0][tid];
+      for (int pp = 1; pp < 4; ++pp) {
+        s0.x += parts[pp][tid].x;
+        s0.y += parts[pp][tid].y;
+      }
+      qbar[2 * tid] = s0.x * (1.0f / kBlock);
+      qbar[2 * tid + 1] = s0.y * (1.0f / kBlock);
+    }
+    __syncthreads();
+  }
+  const float* kb = kbar + static_cast<size_t>(h / d.group) * d.nb * kHeadDim;
+  float mx = -INFINITY;
+  for (int J = tid; J < d.nb; J += 256) {
+    const float* kr = kb + static_cast<size_t>(J) * kHeadDim;
+    float acc = 0.f;
+    for (int c = 0; c < kHeadDim; ++c) acc = fmaf(qbar[c], kr[c], acc);
+    acc *= d.scale;
+    z[J] = acc;
+    mx = fmaxf(mx, acc);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  __shared__ float red[8];
+  if ((tid & 31) == 0) red[tid >> 5] = mx;
+  __syncthreads();
+  mx = red[0];
+  for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
+  float sum = 0.f;
+  for (int J = tid; J < d.nb; J += 256) {
+    const float e = expf(z[J] - mx);
+    z[J] = e;
+    sum += e;
+  }
+  const float total = block_sum<float>(sum, fscratch);
+  const float inv = 1.0f / total;
+  // 0.5 KL(a_hat || m) + 0.5 KL(a_bar || m), m = (a_hat + a_bar) / 2; zero-probability terms contribute 0
+  float acc = 0.f;
+  const float* ah = p_v + static_cast<size_t>(h) * d.nb;
+  for (int J = tid; J < d.nb; J += 256) {
+    const float a = ah[J], b = z[J] * inv;
+    const float m = 0.5f * (a + b);
+    if (a > 0.f) acc += 0.5f * a * logf(a / m);
+    if (b > 0.f) acc += 0.5f * b * logf(b / m);
+  }
+  const float js = block_sum<float>(acc, fscratch);
+  if (tid == 0) {
+    const float dist = sqrtf(fmaxf(js, 0.f));
+    jsd[h] = dist;
+    pattern[h] = dist >= tau_jsd ? CRISP_PATTERN_VS : CRISP_PATTERN_PE;
+  }
+}
+}  // namespace
+
+int launch_route_jsd(const Dims& d, const void* q, const void* k, const float* p_v, void* ws, float tau_jsd,
+                     float* jsd, int32_t* pattern, cudaStream_t stream) {
+  if (d.nb > 8192) return CRISP_ERR_UNSUPPORTED;
+  size_t total;
+  SelectPtrs w = carve(d, ws, &total);
+  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "route_jsd: clear status");
+  pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, static_cast<const __nv_bfloat16*>(k), d.hkv, 0, nullptr,
+                                                     w.kbar);
+  jsd_kernel<<<d.hq, 256, sizeof(float) * d.nb, stream>>>(d, static_cast<const __nv_bfloat16*>(q), w.kbar, p_v,
+                                                         tau_jsd, jsd, pattern);
+  CRISP_CUDA_TRY(cudaGetLastError(), "route_jsd: launch");
   return CRISP_OK;
 }
 

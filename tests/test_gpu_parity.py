@@ -200,3 +200,35 @@ def test_results_are_reproducible():
     b = pu.run_gpu(p, q, k, v)
     for key in ("c_struct", "p_v", "p_s", "row_ptr", "col_idx", "o"):
         assert np.array_equal(a[key], b[key]), key
+
+
+def test_jsd_comparison_router():
+    """Algorithm 5 on the GPU against the oracle, and the agreement of the two routers on synthetic heads."""
+    pu = _pu()
+    import paper_2609_01925_b200 as crisp
+    from paper_2609_01925_b200 import binding as B
+    cases = [synth.tiny(n=4096),
+             synth.qwen_shaped("Q8k", 8192).with_(n_q_heads=14, n_kv_heads=2,
+                                                  head_classes=("sink", "slash", "diffuse", "diffuse") * 3 + ("sink", "slash"))]
+    for w in cases:
+        p = pu.params_of(w)
+        q, k, v = synth.make_qkv(w, device="cuda")
+        layer = crisp.CrispLayer(p)
+        layer.route(q, k)
+        jsd = torch.full((w.n_q_heads,), -1.0, device="cuda")
+        pat = torch.full((w.n_q_heads,), -1, dtype=torch.int32, device="cuda")
+        tau_jsd = 0.1
+        B.check(B.crisp_route_jsd(p, q, k, layer.p_v, layer.select_ws, tau_jsd, jsd, pat), "crisp_route_jsd")
+        torch.cuda.synchronize()
+        assert B.crisp_poll_device_status(layer.select_ws) == B.OK
+        qc, kc = q.cpu().float().numpy(), k.cpu().float().numpy()
+        agree = 0
+        for h in range(w.n_q_heads):
+            want, _, _ = orc.jsd_router(qc[:, h], kc[:, h // w.group], 128)
+            got = float(jsd[h].item())
+            assert abs(got - want) <= 2e-4 + 2e-3 * want, (h, got, want)
+            if abs(want - tau_jsd) > 1e-3 * tau_jsd:
+                assert int(pat[h].item()) == (1 if want >= tau_jsd else 0)
+            agree += int(pat[h].item()) == int(layer.pattern[h].item())
+        print(f"{w.name}: JSD {jsd.cpu().numpy().round(3).tolist()}; C_struct and JSD routers agree on "
+              f"{agree}/{w.n_q_heads} heads")

@@ -535,3 +535,41 @@ def test_head_pipeline_invariants_on_synthetic_heads():
         lists[alpha] = rr["cols"]
     for m in range(nb):
         assert set(lists[2.0][m]) <= set(lists[1.0][m]) <= set(lists[0.5][m])
+
+
+# ------------------------------------------------------------------ Algorithm 5 (comparison router)
+def test_js_distance_hand_worked_and_limits():
+    """Hand-worked: a = (1, 0), b = (1/2, 1/2): m = (3/4, 1/4);
+    KL(a||m) = ln(4/3), KL(b||m) = 1/2 ln(2/3) + 1/2 ln 2 -> D = sqrt(0.5 * 0.2876821 + 0.5 * 0.1438410)."""
+    d = orc.js_distance(np.array([1.0, 0.0]), np.array([0.5, 0.5]))
+    assert np.isclose(d, math.sqrt(0.5 * math.log(4 / 3) + 0.5 * (0.5 * math.log(2 / 3) + 0.5 * math.log(2))), rtol=1e-12)
+    assert np.isclose(d, 0.4645014, rtol=1e-6)
+    r_ = rng(30)
+    a = r_.dirichlet(np.ones(16)); b = r_.dirichlet(np.ones(16))
+    assert orc.js_distance(a, a) == 0.0
+    assert np.isclose(orc.js_distance(a, b), orc.js_distance(b, a), rtol=1e-13)
+    # disjoint supports: the distance reaches its maximum sqrt(ln 2)
+    assert np.isclose(orc.js_distance(np.array([0.5, 0.5, 0, 0]), np.array([0, 0, 0.3, 0.7])), math.sqrt(math.log(2)), rtol=1e-13)
+    assert 0.0 < orc.js_distance(a, b) < math.sqrt(math.log(2))
+
+
+def test_jsd_router_closed_forms():
+    """Q = 0: both estimates are known in closed form (uniform pooled estimate, uniform proxy rows)."""
+    nb, d = 6, 8
+    n = nb * B
+    k = rng(31).normal(size=(n, d))
+    dist, a_bar, a_hat = orc.jsd_router(np.zeros((n, d)), k, B)
+    assert np.allclose(a_bar, 1.0 / nb)
+    # a_hat[J] = (1/B) sum_i (keys of block J visible to row i) / (t_i + 1)
+    want = np.zeros(nb)
+    for i in range(B):
+        t = n - B + i
+        for J in range(nb):
+            want[J] += min(max(t + 1 - J * B, 0), B) / (t + 1) / B
+    assert np.allclose(a_hat, want, rtol=1e-12)
+    assert np.isclose(dist, orc.js_distance(want, np.full(nb, 1 / nb)), rtol=1e-12)
+    # a head whose queries all point at one key block: the pooled estimate and the per-query mean agree
+    q = np.zeros((n, d)); q[:, 0] = 8.0
+    k2 = np.zeros((n, d)); k2[2 * B:3 * B, 0] = 8.0
+    dist2, a_bar2, a_hat2 = orc.jsd_router(q, k2, B)
+    assert a_bar2[2] > 0.999 and a_hat2[2] > 0.999 and dist2 < 0.05
