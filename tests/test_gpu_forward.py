@@ -71,3 +71,26 @@ def test_lists_that_do_not_fit_are_never_read():
     big = crisp.CrispLayer(p)
     big.forward(q, k, v); big.poll()
     assert not (big.o == 7.0).all()
+
+
+def test_forward_replays_from_a_cuda_graph():
+    """The staged kernels of crisp_forward contain no host synchronisation, so one capture replays the
+    whole of Algorithm 1 (this is how a caller removes the per-launch host cost at short contexts)."""
+    w, p, q, k, v = _setup(n=4096)
+    layer = crisp.CrispLayer(p)
+    layer.forward(q, k, v); layer.poll()
+    torch.cuda.synchronize()
+    ref = layer.o.clone()
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        layer.forward(q, k, v, stream=s)          # warm-up on the side stream
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=s):
+            layer.forward(q, k, v, stream=torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    layer.o.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    layer.poll()
+    assert torch.equal(layer.o, ref)
