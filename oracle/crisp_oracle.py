@@ -6,6 +6,9 @@ It shares no code with the CUDA library: it is written from the paper's
 definitions, step by step, with numpy matmul / sort / cumsum as library steps
 and no blocking, fusion or reordering beyond what the definitions state.
 
+Sequence lengths need not be multiples of the block size: N_b = ceil(n / B) as in Section 4.3, the last
+block simply holds fewer tokens.
+
 Conventions (one attention layer):
   q [n, H_q, d], k, v [n, H_kv, d]: arrays holding bf16-representable values
   (float32 or float64); query head h reads KV head h // (H_q // H_kv).
@@ -105,11 +108,10 @@ def jsd_router(q_h: np.ndarray, k_h: np.ndarray, block: int, scale: float | None
     q_h = np.asarray(q_h, dtype=np.float64)
     k_h = np.asarray(k_h, dtype=np.float64)
     n, d = k_h.shape
-    nb = n // block
     if scale is None:
         scale = 1.0 / math.sqrt(d)
     q_bar = q_h[n - block:].mean(axis=0)
-    k_bar = k_h.reshape(nb, block, d).mean(axis=1)
+    k_bar = block_means(k_h, block)
     z = (k_bar @ q_bar) * scale
     e = np.exp(z - z.max())
     a_bar = e / e.sum()
@@ -127,7 +129,7 @@ def block_scores(a_hat: np.ndarray, block: int) -> Tuple[np.ndarray, np.ndarray]
     pooling adds the `block` consecutive entries of a block.  sum(A) = number of rows.
     """
     b, n = a_hat.shape
-    nb = n // block
+    nb = -(-n // block)                      # N_b = ceil(n / B); the last block may be partial
     total = a_hat.sum()
     a_v = a_hat.sum(axis=0) / total
     a_s = np.zeros(n, dtype=np.float64)
@@ -136,8 +138,10 @@ def block_scores(a_hat: np.ndarray, block: int) -> Tuple[np.ndarray, np.ndarray]
         # offset o = t - j for j = 0..t  <=>  reversed visible part of the row
         a_s[:t + 1] += a_hat[i, t::-1]
     a_s /= total
-    p_v = a_v.reshape(nb, block).sum(axis=1)
-    p_s = a_s.reshape(nb, block).sum(axis=1)
+    starts = np.arange(0, n, block)
+    p_v = np.add.reduceat(a_v, starts)
+    p_s = np.add.reduceat(a_s, starts)
+    assert p_v.shape[0] == nb
     return p_v, p_s
 
 
@@ -207,6 +211,14 @@ def select_gamma(p: np.ndarray, gamma: float, k_min: int) -> Tuple[np.ndarray, i
 # ----------------------------------------------------------------------------------------
 # Algorithm 4: pooled estimation (PE) index set
 # ----------------------------------------------------------------------------------------
+def block_means(x: np.ndarray, block: int) -> np.ndarray:
+    """Mean over the rows of every block of `block` tokens (the last block may hold fewer rows)."""
+    n = x.shape[0]
+    starts = np.arange(0, n, block)
+    counts = np.minimum(starts + block, n) - starts
+    return np.add.reduceat(x, starts, axis=0) / counts[:, None]
+
+
 def pooled_map(q_h: np.ndarray, k_h: np.ndarray, block: int,
                scale: float | None = None) -> np.ndarray:
     """A_bar = row softmax of pool(Q) pool(K)^T / sqrt(d), causal at block level (J <= m).
@@ -216,11 +228,11 @@ def pooled_map(q_h: np.ndarray, k_h: np.ndarray, block: int,
     q_h = np.asarray(q_h, dtype=np.float64)
     k_h = np.asarray(k_h, dtype=np.float64)
     n, d = q_h.shape
-    nb = n // block
+    nb = -(-n // block)
     if scale is None:
         scale = 1.0 / math.sqrt(d)
-    q_bar = q_h.reshape(nb, block, d).mean(axis=1)
-    k_bar = k_h.reshape(nb, block, d).mean(axis=1)
+    q_bar = block_means(q_h, block)
+    k_bar = block_means(k_h, block)
     z = (q_bar @ k_bar.T) * scale
     m = np.arange(nb)[:, None]
     jj = np.arange(nb)[None, :]
@@ -295,16 +307,18 @@ def sparse_attention_block(q_h: np.ndarray, k_h: np.ndarray, v_h: np.ndarray, m:
 
     Returns (O [block, d] fp64, lse [block] fp64 = log sum exp of the kept scaled logits).
     """
-    q_h = np.asarray(q_h[m * block:(m + 1) * block], dtype=np.float64)
+    n = np.asarray(k_h).shape[0]
+    q_h = np.asarray(q_h[m * block:min((m + 1) * block, n)], dtype=np.float64)
     d = q_h.shape[1]
     if scale is None:
         scale = 1.0 / math.sqrt(d)
     cols = np.asarray(cols, dtype=np.int64)
     key_idx = (cols[:, None] * block + np.arange(block)[None, :]).reshape(-1)
+    key_idx = key_idx[key_idx < n]           # the last key block may be partial
     kk = np.asarray(k_h[key_idx], dtype=np.float64)
     vv = np.asarray(v_h[key_idx], dtype=np.float64)
     s = (q_h @ kk.T) * scale
-    t = m * block + np.arange(block)[:, None]
+    t = m * block + np.arange(q_h.shape[0])[:, None]
     s = np.where(key_idx[None, :] <= t, s, -np.inf)
     mx = s.max(axis=1, keepdims=True)
     e = np.exp(s - mx)
@@ -319,8 +333,8 @@ def sparse_attention_head(q_h, k_h, v_h, cols_per_block: Sequence[Sequence[int]]
     o = np.empty((n, d), dtype=np.float64)
     lse = np.empty(n, dtype=np.float64)
     for m, cols in enumerate(cols_per_block):
-        o[m * block:(m + 1) * block], lse[m * block:(m + 1) * block] = \
-            sparse_attention_block(q_h, k_h, v_h, m, cols, block, scale)
+        hi = min((m + 1) * block, n)
+        o[m * block:hi], lse[m * block:hi] = sparse_attention_block(q_h, k_h, v_h, m, cols, block, scale)
     return o, lse
 
 
@@ -338,7 +352,7 @@ def head_pipeline(q_h: np.ndarray, k_h: np.ndarray, *, block: int = 128, sink_to
     force_pattern 0 = by C_struct, 1 = VS, 2 = PE.
     """
     n = np.asarray(q_h).shape[0]
-    nb = n // block
+    nb = -(-n // block)
     a_hat = proxy_attention(q_h, k_h, block, scale)
     c = c_struct(a_hat, sink_tokens, local_tokens)
     pattern = route(c, tau)

@@ -573,3 +573,57 @@ def test_jsd_router_closed_forms():
     k2 = np.zeros((n, d)); k2[2 * B:3 * B, 0] = 8.0
     dist2, a_bar2, a_hat2 = orc.jsd_router(q, k2, B)
     assert a_bar2[2] > 0.999 and a_hat2[2] > 0.999 and dist2 < 0.05
+
+
+# ------------------------------------------------------------------ ragged n: N_b = ceil(n / B) (Section 4.3)
+def test_ragged_length_block_scores_bruteforce_and_unit_mass():
+    n, d, blk = 53, 4, 8              # 7 blocks, the last one holds 5 tokens
+    r = rng(40)
+    a = orc.proxy_attention(r.normal(size=(n, d)), r.normal(size=(n, d)), blk)
+    nb = 7
+    pv = [0.0] * nb
+    ps = [0.0] * nb
+    for i in range(blk):
+        t = n - blk + i
+        for j in range(t + 1):
+            pv[j // blk] += a[i, j] / blk
+            ps[(t - j) // blk] += a[i, j] / blk
+    p_v, p_s = orc.block_scores(a, blk)
+    assert p_v.shape == p_s.shape == (nb,)
+    assert np.allclose(p_v, pv, rtol=1e-12) and np.allclose(p_s, ps, rtol=1e-12)
+    assert np.isclose(p_v.sum(), 1) and np.isclose(p_s.sum(), 1)
+
+
+def test_ragged_length_attention_matches_library():
+    d = 8
+    n = 5 * B + 7
+    r = rng(41)
+    q, k, v = (r.normal(size=(n, d)) for _ in range(3))
+    nb = 6
+    o, _ = orc.sparse_attention_head(q, k, v, orc.dense_cols(nb), B)
+    assert np.allclose(o, sdpa64(q, k, v, causal=True), rtol=1e-11, atol=1e-12)
+    cols = orc.expand_vs([2], [1], nb)
+    mask = np.zeros((n, n), dtype=bool)
+    for m in range(nb):
+        for J in cols[m]:
+            mask[m * B:(m + 1) * B, J * B:(J + 1) * B] = True
+    mask &= np.tril(np.ones((n, n), dtype=bool))
+    o2, _ = orc.sparse_attention_head(q, k, v, cols, B)
+    assert np.allclose(o2, sdpa64(q, k, v, mask=mask), rtol=1e-11, atol=1e-12)
+
+
+def test_ragged_length_pooling_and_pipeline():
+    d = 8
+    n = 4 * B + 3
+    r = rng(42)
+    x = r.normal(size=(n, d))
+    bm = orc.block_means(x, B)
+    assert bm.shape == (5, d)
+    assert np.allclose(bm[4], x[4 * B:].mean(axis=0)) and np.allclose(bm[1], x[B:2 * B].mean(axis=0))
+    res = orc.head_pipeline(x * 2, r.normal(size=(n, d)) * 2, block=B, sink_tokens=4, local_tokens=B, tau=0.0,
+                            k_min_blocks=1)
+    assert len(res["cols"]) == 5 and res["p_v"].shape == (5,)
+    for m, c in enumerate(res["cols"]):
+        assert c[0] == 0 and c[-1] == m
+    res = orc.head_pipeline(np.zeros((n, d)), np.zeros((n, d)), block=B, tau=2.0, gamma=0.5)
+    assert res["pattern"] == orc.PE and res["a_bar"].shape == (5, 5)
