@@ -37,7 +37,7 @@ extern "C" {
 typedef enum crisp_status {
   CRISP_OK = 0,
   CRISP_ERR_INVALID_ARG = -1,    /* null pointer, non-positive size, inconsistent head counts, ...   */
-  CRISP_ERR_UNSUPPORTED = -2,    /* head_dim != 128, block != 128, seq_len not a multiple of block, ... */
+  CRISP_ERR_UNSUPPORTED = -2,    /* head_dim != 128, block != 128, seq_len out of range, ...         */
   CRISP_ERR_WORKSPACE = -3,      /* workspace too small or misaligned                                */
   CRISP_ERR_CAPACITY = -4,       /* col_idx capacity too small for the selected blocks               */
   CRISP_ERR_CUDA = -5,           /* a CUDA runtime / driver call failed (see crisp_last_cuda_error)  */
@@ -51,7 +51,8 @@ typedef enum crisp_status {
 /* Problem description: the inputs of Algorithm 1 plus the constants of Sections 3.2 and 4.3. */
 typedef struct crisp_params {
   int32_t struct_size;   /* = sizeof(crisp_params); ABI guard                                        */
-  int32_t seq_len;       /* n; a multiple of `block`, 2 * block <= n <= 8192 * block (1,048,576)     */
+  int32_t seq_len;       /* n; 2 * block <= n <= 8192 * block (1,048,576); need not be a multiple of
+                            `block`: N_b = ceil(n / block), the last block is partial (Section 4.3)  */
   int32_t n_q_heads;     /* H_q                                                                      */
   int32_t n_kv_heads;    /* H_kv; H_q % H_kv == 0 and H_q / H_kv <= 16                               */
   int32_t head_dim;      /* 128 only                                                                 */

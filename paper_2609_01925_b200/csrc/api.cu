@@ -74,11 +74,13 @@ int validate(const crisp_params* p, Dims* d) {
       !std::isfinite(p->gamma) || !(p->softmax_scale >= 0.f) || !std::isfinite(p->softmax_scale))
     return CRISP_ERR_INVALID_ARG;
   if (p->head_dim != kHeadDim || p->block != kBlock) return CRISP_ERR_UNSUPPORTED;
-  if (p->seq_len % kBlock != 0 || p->seq_len < 2 * kBlock) return CRISP_ERR_UNSUPPORTED;
+  if (p->seq_len < 2 * kBlock) return CRISP_ERR_UNSUPPORTED;
   if (p->n_q_heads / p->n_kv_heads > kMaxGroup) return CRISP_ERR_UNSUPPORTED;
-  if (p->seq_len / kBlock > 8192) return CRISP_ERR_UNSUPPORTED;  // N_b limit of the selection kernels (1M tokens)
+  if (p->seq_len > 8192 * kBlock) return CRISP_ERR_UNSUPPORTED;  // N_b limit of the selection kernels (1M tokens)
   d->n = p->seq_len;
-  d->nb = p->seq_len / kBlock;
+  d->nb = (p->seq_len + kBlock - 1) / kBlock;
+  d->nfull = p->seq_len / kBlock;
+  d->rho = p->seq_len % kBlock;
   d->hq = p->n_q_heads;
   d->hkv = p->n_kv_heads;
   d->group = d->hq / d->hkv;

@@ -18,7 +18,9 @@ constexpr float kLog2e = 1.4426950408889634f;
 // Validated, derived problem sizes passed to kernels by value.
 struct Dims {
   int n;          // seq_len
-  int nb;         // N_b = n / B
+  int nb;         // N_b = ceil(n / B); the last block holds n - (N_b - 1) B tokens
+  int nfull;      // floor(n / B)
+  int rho;        // n mod B (0 when every block is full)
   int hq, hkv, group;
   int w_sink, w_local;
   int n_sink_tiles;    // key tiles intersecting [0, w_sink)

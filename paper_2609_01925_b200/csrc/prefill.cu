@@ -564,6 +564,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       tc_fence_after_sync();
       const float inv = 1.0f / l_run;
       const size_t token = static_cast<size_t>(m_t) * kBlock + r;
+      const bool in_range = token < static_cast<size_t>(d.n);  // the last block may be partial
       __nv_bfloat16* orow = a.o + (token * d.hq + it.h) * kHeadDim;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
@@ -571,6 +572,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         tmem_ld_x32(o_addr + c * 32, ov);
         tmem_ld_wait();
         uint4* dst = reinterpret_cast<uint4*>(orow + c * 32);
+        if (in_range)
 #pragma unroll
         for (int g = 0; g < 4; ++g) {
           uint4 val;
@@ -581,7 +583,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           dst[g] = val;
         }
       }
-      if (a.lse) a.lse[static_cast<size_t>(it.h) * d.n + token] = m_used * 0.6931471805599453f + logf(l_run);
+      if (a.lse && in_range) a.lse[static_cast<size_t>(it.h) * d.n + token] = m_used * 0.6931471805599453f + logf(l_run);
       tc_fence_before_sync();
     }
   }

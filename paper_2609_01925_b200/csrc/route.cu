@@ -27,6 +27,7 @@ struct RoutePtrs {
   float* pm;       // [hq][nb][128] tile-local max of the scaled logits (base-2 units)
   float* plo;      // [hq][nb][128] sum of 2^(x - max) over entries with key offset <= row
   float* pup;      // [hq][nb][128] ... over entries with key offset > row
+  float* phi;      // [hq][nb][128] third band, only when n is not a multiple of 128 (see proxy_partials_kernel)
   float* panc;     // [hq][slots][128] ... over anchor keys of the tile
   float* cm;       // [hq][n_chunks][128] chunk max
   float* cl;       // [hq][n_chunks][128] chunk sum relative to chunk max
@@ -34,6 +35,7 @@ struct RoutePtrs {
   float* row_invl; // [hq][128] 1 / global row sum
   float* slo;      // [hq][nb] mass (over rows) on/below the tile diagonal
   float* sup;      // [hq][nb] mass above the tile diagonal
+  float* shi;      // [hq][nb] mass of the third band (ragged n only)
   int n_chunks;
 };
 
@@ -118,7 +120,14 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   } else {
     // ---- one thread per proxy row
     const int i = tid;
-    const bool last_tile = (J == d.nb - 1);
+    // Offset of proxy row i to local key jl of this tile: o = t_i - j = q * 128 + (rho + i - jl) with
+    // q = nfull - 1 - J and rho = n mod 128.  The entry is visible iff o >= 0 and belongs to the diagonal
+    // band of block offset floor(o / 128), which is q - 1 ("up": jl > i + rho), q ("lo") or q + 1
+    // ("hi": jl <= i + rho - 128, possible only when rho > 0).  A band with a negative offset is invisible.
+    const int qoff = d.nfull - 1 - J;
+    const int a_thr = i + d.rho;          // jl <= a_thr  <=>  not in the "up" band
+    const int b_thr = i + d.rho - kBlock;  // jl <= b_thr  <=>  in the "hi" band
+    const bool vis_up = qoff - 1 >= 0, vis_lo = qoff >= 0;  // "hi" (q + 1 >= 0) is visible whenever it is non-empty
     const int js = min(max(d.w_sink - J * kBlock, 0), kBlock);            // anchor: local key < js
     const int jl = min(max(d.n - d.w_local - J * kBlock, 0), kBlock);     // anchor: local key >= jl
     const bool has_slot = (J < d.n_sink_tiles) || (J >= d.first_local_tile);
@@ -144,26 +153,33 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
           const int j = c * 32 + t;
           const float x = __uint_as_float(r[c][t]) * d.scale_log2;
           r[c][t] = __float_as_uint(x);
-          if (!last_tile || j <= i) mx = fmaxf(mx, x);
+          const bool visible = (j <= b_thr) || (j <= a_thr ? vis_lo : vis_up);
+          if (visible) mx = fmaxf(mx, x);
         }
-      float lo = 0.f, up = 0.f, anc = 0.f;
+      // a row may see no key of this tile (ragged n: the tiles around the proxy block): leave a neutral partial
+      const bool any = mx > -INFINITY;
+      if (!any) mx = -1e30f;
+      float lo = 0.f, up = 0.f, hi = 0.f, anc = 0.f;
 #pragma unroll
       for (int c = 0; c < 4; ++c)
 #pragma unroll
         for (int t = 0; t < 32; ++t) {
           const int j = c * 32 + t;
           const float e = ex2(__uint_as_float(r[c][t]) - mx);
-          const bool below = (j <= i);
-          const bool valid = below || !last_tile;
-          lo += below ? e : 0.f;
-          up += (valid && !below) ? e : 0.f;
-          anc += (valid && (j < js || j >= jl)) ? e : 0.f;
+          const bool in_hi = j <= b_thr, in_lo = !in_hi && j <= a_thr, in_up = j > a_thr;
+          const bool visible = in_hi || (in_lo && vis_lo) || (in_up && vis_up);
+          hi += in_hi ? e : 0.f;
+          lo += (in_lo && vis_lo) ? e : 0.f;
+          up += (in_up && vis_up) ? e : 0.f;
+          anc += (visible && (j < js || j >= jl)) ? e : 0.f;
         }
+      if (!any) lo = up = hi = anc = 0.f;
       const int h = kvh * G + g;
       const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
       w.pm[off] = mx;
       w.plo[off] = lo;
       w.pup[off] = up;
+      if (d.rho > 0) w.phi[off] = hi;
       if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
     }
   }
@@ -183,7 +199,7 @@ __global__ void __launch_bounds__(128) row_stats_kernel(const Dims d, const Rout
   for (int J = j0; J < j1; ++J) {
     const size_t off = base + static_cast<size_t>(J) * kBlock;
     const float m = w.pm[off];
-    const float sum = w.plo[off] + w.pup[off];
+    const float sum = w.plo[off] + w.pup[off] + (d.rho > 0 ? w.phi[off] : 0.f);
     const float nm = fmaxf(M, m);
     L = L * ex2(M - nm) + sum * ex2(m - nm);
     M = nm;
@@ -227,19 +243,22 @@ __global__ void __launch_bounds__(128) tile_sums_kernel(const Dims d, const Rout
   const int j0 = chunk * kChunk, j1 = min(j0 + kChunk, d.nb);
   for (int J = j0 + warp; J < j1; J += 4) {
     const size_t base = (static_cast<size_t>(h) * d.nb + J) * kBlock + lane;
-    float lo = 0.f, up = 0.f;
+    float lo = 0.f, up = 0.f, hi = 0.f;
 #pragma unroll
     for (int r = 0; r < 4; ++r) {
       const float wgt = ex2(w.pm[base + 32 * r] - M[r]) * invl[r];
       lo += wgt * w.plo[base + 32 * r];
       up += wgt * w.pup[base + 32 * r];
+      if (d.rho > 0) hi += wgt * w.phi[base + 32 * r];
     }
     lo = warp_sum(lo);
     up = warp_sum(up);
+    hi = warp_sum(hi);
     if (lane == 0) {
       w.slo[static_cast<size_t>(h) * d.nb + J] = lo;
       w.sup[static_cast<size_t>(h) * d.nb + J] = up;
-      p_v[static_cast<size_t>(h) * d.nb + J] = lo + up;
+      w.shi[static_cast<size_t>(h) * d.nb + J] = hi;
+      p_v[static_cast<size_t>(h) * d.nb + J] = (lo + up) + hi;
     }
   }
 }
@@ -250,9 +269,15 @@ __global__ void __launch_bounds__(256) finalize_kernel(const Dims d, const Route
   const int h = blockIdx.x, tid = threadIdx.x;
   const float* slo = w.slo + static_cast<size_t>(h) * d.nb;
   const float* sup = w.sup + static_cast<size_t>(h) * d.nb;
+  const float* shi = w.shi + static_cast<size_t>(h) * d.nb;
+  // band of block offset s: "lo" of tile nfull-1-s, "up" of tile nfull-2-s, "hi" of tile nfull-s
   for (int sidx = tid; sidx < d.nb; sidx += blockDim.x) {
-    const int jlo = d.nb - 1 - sidx, jup = d.nb - 2 - sidx;
-    p_s[static_cast<size_t>(h) * d.nb + sidx] = slo[jlo] + (jup >= 0 ? sup[jup] : 0.f);
+    const int jlo = d.nfull - 1 - sidx, jup = d.nfull - 2 - sidx, jhi = d.nfull - sidx;
+    float v = 0.f;
+    if (jlo >= 0 && jlo < d.nb) v += slo[jlo];
+    if (jup >= 0 && jup < d.nb) v += sup[jup];
+    if (d.rho > 0 && jhi >= 0 && jhi < d.nb) v += shi[jhi];
+    p_s[static_cast<size_t>(h) * d.nb + sidx] = v;
   }
   __shared__ float red[4];
   float acc = 0.f;
@@ -291,6 +316,7 @@ RoutePtrs carve(const Dims& d, void* ws) {
   w.pm = take(part);
   w.plo = take(part);
   w.pup = take(part);
+  w.phi = d.rho > 0 ? take(part) : nullptr;  // third band: only for lengths that are not multiples of 128
   w.panc = take(static_cast<size_t>(d.hq) * d.n_anchor_slots * kBlock);
   w.cm = take(static_cast<size_t>(d.hq) * w.n_chunks * kBlock);
   w.cl = take(static_cast<size_t>(d.hq) * w.n_chunks * kBlock);
@@ -298,6 +324,7 @@ RoutePtrs carve(const Dims& d, void* ws) {
   w.row_invl = take(static_cast<size_t>(d.hq) * kBlock);
   w.slo = take(static_cast<size_t>(d.hq) * d.nb);
   w.sup = take(static_cast<size_t>(d.hq) * d.nb);
+  w.shi = take(static_cast<size_t>(d.hq) * d.nb);
   return w;
 }
 
@@ -305,7 +332,7 @@ RoutePtrs carve(const Dims& d, void* ws) {
 
 size_t route_ws_bytes(const Dims& d) {
   RoutePtrs w = carve(d, nullptr);
-  return reinterpret_cast<size_t>(w.sup) + align_up(static_cast<size_t>(d.hq) * d.nb * sizeof(float), 256);
+  return reinterpret_cast<size_t>(w.shi) + align_up(static_cast<size_t>(d.hq) * d.nb * sizeof(float), 256);
 }
 
 int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c_struct, int32_t* pattern,

@@ -215,8 +215,11 @@ pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is
   const __nv_bfloat162* base = reinterpret_cast<const __nv_bfloat162*>(
       x + (static_cast<size_t>(J) * kBlock + half * 64) * heads * kHeadDim + static_cast<size_t>(h) * kHeadDim);
   float a0 = 0.f, a1 = 0.f;
+  // the last block may hold fewer than 128 tokens: rows at or beyond n are not read
+  const int valid = min(kBlock, d.n - J * kBlock);
+  const int rows = min(max(valid - half * 64, 0), 64);
 #pragma unroll 8
-  for (int t = 0; t < 64; ++t) {
+  for (int t = 0; t < rows; ++t) {
     const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
     a0 += v.x;
     a1 += v.y;
@@ -226,8 +229,9 @@ pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is
   __syncthreads();
   if (half == 0) {
     float* o = out + (static_cast<size_t>(h) * d.nb + J) * kHeadDim;
-    o[2 * pair] = (a0 + other[pair].x) * (1.0f / kBlock);
-    o[2 * pair + 1] = (a1 + other[pair].y) * (1.0f / kBlock);
+    const float inv = 1.0f / static_cast<float>(valid);
+    o[2 * pair] = (a0 + other[pair].x) * inv;
+    o[2 * pair + 1] = (a1 + other[pair].y) * inv;
   }
 }
 

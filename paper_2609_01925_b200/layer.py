@@ -22,7 +22,7 @@ class CrispLayer:
         self.p = params
         self.device = torch.device(device)
         n, hq = params.seq_len, params.n_q_heads
-        self.nb = n // params.block
+        self.nb = -(-n // params.block)
         rws, sws, pws = B.crisp_workspace_bytes(params)
         dev = self.device
         self.route_ws = torch.empty(rws, dtype=torch.uint8, device=dev)

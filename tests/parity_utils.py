@@ -132,7 +132,7 @@ def gpu_matrix(g, h, nb):
 
 def check_lists(g, res, p, heads=None):
     """GPU lists vs oracle lists under the matching rule.  Returns the count of excused blocks."""
-    nb = p.seq_len // p.block
+    nb = -(-p.seq_len // p.block)
     excused_total = 0
     heads = range(len(res)) if heads is None else heads
     for h in heads:

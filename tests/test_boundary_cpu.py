@@ -49,7 +49,8 @@ def test_workspace_sizes_grow_with_the_problem():
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(seq_len=4096 + 64), B.ERR_UNSUPPORTED),        # ragged n
+    (dict(seq_len=255), B.ERR_UNSUPPORTED),              # fewer than two blocks
+    (dict(seq_len=8192 * 128 + 1), B.ERR_UNSUPPORTED),   # more than 8192 blocks
     (dict(seq_len=128), B.ERR_UNSUPPORTED),              # fewer than two blocks
     (dict(head_dim=64), B.ERR_UNSUPPORTED),
     (dict(block=64), B.ERR_UNSUPPORTED),
@@ -73,6 +74,12 @@ def test_invalid_parameters_are_rejected(kw, code):
     with pytest.raises(crisp.CrispError) as e:
         B.crisp_workspace_bytes(p)
     assert e.value.status == code
+
+
+def test_ragged_lengths_are_accepted():
+    for n in (256, 257, 4096 + 64, 8192 * 128 - 5):
+        sizes = B.crisp_workspace_bytes(crisp.make_params(n, 4, 1))
+        assert all(s > 0 for s in sizes)
 
 
 def test_abi_guard_and_null_pointers():

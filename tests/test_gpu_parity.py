@@ -58,6 +58,25 @@ def test_small_and_odd_block_counts(n):
     _full_check(w, per_head=16)
 
 
+@pytest.mark.parametrize("n", [257, 300, 1000, 4096 + 37, 4096 - 1, 2048 + 64])
+def test_ragged_sequence_lengths(n):
+    """n not a multiple of 128: N_b = ceil(n / 128), the last block is partial (Section 4.3)."""
+    pu = _pu()
+    w = synth.tiny(n=n).with_(k_min_blocks=2)
+    g, res = _full_check(w, per_head=64)
+    np.testing.assert_allclose(g["p_v"].sum(1), 1.0, rtol=1e-5)
+    np.testing.assert_allclose(g["p_s"].sum(1), 1.0, rtol=1e-5)
+
+
+def test_ragged_length_gqa_and_selectors():
+    pu = _pu()
+    w = synth.llama_shaped("L8k-r", 8192 + 77, 32).with_(n_q_heads=8, n_kv_heads=2,
+                                                        head_classes=("conc", "diffuse") * 4)
+    _full_check(w, per_head=6)
+    _full_check(w, p=pu.params_of(w, selector=1), per_head=2, dense=False)
+    _full_check(w, p=pu.params_of(w, selector=2, sink_tokens=128), per_head=2, dense=False)
+
+
 def test_paper_window_sizes_and_identity():
     """w_sink = w_local = 128: C_struct equals p_v[0] + p_v[N_b-1] (Section 4.3)."""
     pu = _pu()

@@ -114,7 +114,7 @@ class Workload:
 
     @property
     def n_blocks(self) -> int:
-        return self.seq_len // BLOCK
+        return -(-self.seq_len // BLOCK)
 
     @property
     def group(self) -> int:
