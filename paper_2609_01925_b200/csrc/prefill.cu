@@ -6,17 +6,27 @@
 // of the two blocks' lists; each entry carries two flags saying which tile uses it.
 //
 // Warp roles (384 threads):
-//   warps 0-3  softmax of tile 0 (one thread per query row; TMEM lanes 0-127)
-//   warps 4-7  softmax of tile 1
-//   warp  8    TMA producer (one thread): Q once per item, K and V blocks through one five-slot ring
-//   warp  9    MMA issuer (one thread): S_t = Q_t K^T (SS) and O_t += P_t V (P read from TMEM)
-// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each; P_t (bf16) overwrites the first
-// 64 columns of S_t.  The issuer interleaves the two tiles so that the tensor pipe works on one
-// tile while the other tile's softmax runs.  The online softmax rescales O lazily, only when the
-// running maximum grows by more than 2^8, and does it in place in TMEM.
-// Measured alternatives that were slower and are not kept: one issuing thread per tile (the two tiles
-// fall into phase, both softmax phases collide and the tensor pipe idles: 726 vs 970 TFLOP/s dense);
-// handing P over in two halves; computing part of the exponentials on the FMA pipe (see kPolyEvery).
+//   warps 0-3   softmax of tile 0 (one thread per query row; TMEM lanes 0-127)
+//   warps 4-7   softmax of tile 1
+//   warp  8     TMA producer (one thread): Q once per item, K and V blocks through one five-slot ring
+//   warps 9,10  MMA issuers, one thread per tile: S_t = Q_t K^T (SS) and O_t += P_t V (P read from TMEM)
+// TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each.  Every key block is worked on in two
+// halves of 64 keys (A, B): S_A and S_B are separate MMAs (N = 64) into the two halves of S_t, and P_t (bf16)
+// is written over the columns of S_B.  The columns of S_A are therefore free as soon as the softmax has read
+// both halves, so Q K_A^T of the NEXT step is issued behind P_A V_A, in the middle of the current step, and
+// Q K_B^T behind P_B V_B at its end: the softmax of the next step finds its first half waiting and receives
+// the second while it works on the first.  Neither the softmax nor the tensor pipe waits for a whole step of
+// the other, which a whole-block S (P aliased on it) forces: there the per-tile chain Q K^T -> softmax ->
+// P V -> Q K^T is serial and two tiles cover only about half of the pipe's time.  The price is that an N = 64
+// MMA with both operands in shared memory is bound by operand fetch (58 cycles instead of 32, measured).
+// Each half is one step of the online softmax, which rescales O lazily, only when the running maximum
+// grows by more than 2^8, and does it in place in TMEM.
+// Both issuers see every load of the K/V ring in order and release every slot once, so the ring never runs
+// ahead of either tile; apart from that the two tiles run free of each other.
+// Measured alternatives that were slower and are not kept: a single issuing thread for both tiles (its scalar
+// bookkeeping between bursts, several hundred cycles, is idle pipe time); whole-block steps with one issuer
+// per tile, with and without handing P over in two halves; computing part of the exponentials on the FMA
+// pipe (see kPolyEvery).
 // Every mbarrier wait is bounded; a wait that gives up sets a flag that ends all roles, and the
 // status word reports CRISP_ERR_DEVICE_TIMEOUT.
 #include "common.cuh"
@@ -50,7 +60,8 @@ struct PrefillSmem {
   alignas(1024) uint8_t kv[kStages][2][16384];  // ring of K and V blocks [slot][half]; load 2e is K_e, 2e+1 is V_e
   uint64_t q_full, q_free;
   uint64_t kv_full[kStages], kv_empty[kStages];
-  uint64_t s_full[2], p_ready[2], o_done[2];
+  // per tile and per 64-key half (A = keys 0-63, B = keys 64-127 of the block)
+  uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -123,7 +134,7 @@ struct EntryReader {
 // Register budgets after setmaxnreg.  The CTA's pool is what the launch allocated (384 threads x 168
 // registers); setmaxnreg.inc waits, without a bound, until the pool can serve it, so the budgets of the
 // three warpgroups must never add up to more than the pool.
-constexpr int kRegsSoftmax = 208, kRegsOther = 88, kRegsLaunch = 168;
+constexpr int kRegsSoftmax = 192, kRegsOther = 112, kRegsLaunch = 168;
 static_assert(256 * kRegsSoftmax + 128 * kRegsOther <= 384 * kRegsLaunch, "setmaxnreg budgets exceed the CTA's pool");
 
 template <int N>
@@ -133,13 +144,6 @@ __device__ __forceinline__ void reg_alloc() {
 template <int N>
 __device__ __forceinline__ void reg_dealloc() {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
-}
-
-// Lane 0 polls; the outcome is broadcast so the warp stays converged.
-__device__ __forceinline__ bool mbar_wait_lane0(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane) {
-  int ok = 1;
-  if (lane == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-  return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 // ---- packed fp32x2 arithmetic (two lanes per instruction on the FMA pipe)
@@ -194,19 +198,20 @@ __device__ __forceinline__ void exp2_poly2(uint64_t t2, float& p0, float& p1) {
   p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(r1) << 23));
 }
 
-// Maximum of one row of raw logits; on the diagonal block only keys j <= r are visible.
+// Maximum of 64 raw logits of one row (keys key0 .. key0 + 63 of the block); on the diagonal block only
+// keys j <= r are visible.
 template <bool kDiag>
-__device__ __forceinline__ float row_max(const uint32_t (&x)[4][32], int r) {
+__device__ __forceinline__ float row_max(const uint32_t (&x)[2][32], int r, int key0) {
   float m0 = -INFINITY, m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
 #pragma unroll
-  for (int c = 0; c < 4; ++c)
+  for (int c = 0; c < 2; ++c)
 #pragma unroll
     for (int i = 0; i < 32; i += 8) {
       float a[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         a[u] = __uint_as_float(x[c][i + u]);
-        if (kDiag && (c * 32 + i + u) > r) a[u] = -INFINITY;
+        if (kDiag && (key0 + c * 32 + i + u) > r) a[u] = -INFINITY;
       }
       m0 = max3(m0, a[0], a[1]);
       m1 = max3(m1, a[2], a[3]);
@@ -216,28 +221,25 @@ __device__ __forceinline__ float row_max(const uint32_t (&x)[4][32], int r) {
   return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
 }
 
-// P = 2^(x * scale - m) as bf16 into TMEM (two keys per 32-bit column); returns the fp32 row sum.
+// P = 2^(x * scale - m) for 64 keys as bf16 pairs (two keys per 32-bit word); returns the fp32 row sum.
 // With kPolyEvery > 0 one pair in every kPolyEvery goes through exp2_poly2 (FMA pipe) instead of the MUFU.
-// Measured on B200 (L32k dense): 959 TFLOP/s with 0, 893 with 4, 854 with 2 - the softmax warps are bound
-// by issue slots, not by the MUFU, so the default is 0 (every exponential on the MUFU).
 #ifndef CRISP_POLY_EVERY
 #define CRISP_POLY_EVERY 0
 #endif
 constexpr int kPolyEvery = CRISP_POLY_EVERY;
 template <bool kDiag>
-__device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int r, float scale_log2, float m_used,
-                                                uint32_t s_addr) {
+__device__ __forceinline__ float exp_pack(const uint32_t (&x)[2][32], int r, int key0, float scale_log2, float m_used,
+                                          uint32_t (&pk)[2][16]) {
   const uint64_t scale2 = pack2(scale_log2, scale_log2);
   const uint64_t negm2 = pack2(-m_used, -m_used);
   uint64_t sum_a = pack2(0.f, 0.f), sum_b = pack2(0.f, 0.f);
 #pragma unroll
-  for (int c = 0; c < 4; ++c) {
-    uint32_t pk[16];
+  for (int c = 0; c < 2; ++c) {
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
       const uint64_t t2 = fma2(pack2(__uint_as_float(x[c][2 * i]), __uint_as_float(x[c][2 * i + 1])), scale2, negm2);
       float p0, p1;
-      if (kPolyEvery > 0 && (i % kPolyEvery) == kPolyEvery - 1) {
+      if (kPolyEvery > 0 && (i % (kPolyEvery > 0 ? kPolyEvery : 1)) == kPolyEvery - 1) {
         exp2_poly2(t2, p0, p1);
       } else {
         float t0, t1;
@@ -246,17 +248,16 @@ __device__ __forceinline__ float exp_pack_store(const uint32_t (&x)[4][32], int 
         p1 = ex2(t1);
       }
       if (kDiag) {
-        if (c * 32 + 2 * i > r) p0 = 0.f;
-        if (c * 32 + 2 * i + 1 > r) p1 = 0.f;
+        if (key0 + c * 32 + 2 * i > r) p0 = 0.f;
+        if (key0 + c * 32 + 2 * i + 1 > r) p1 = 0.f;
       }
       if (i & 1) {
         sum_a = add2(sum_a, pack2(p0, p1));
       } else {
         sum_b = add2(sum_b, pack2(p0, p1));
       }
-      pk[i] = pack_bf16(p0, p1);
+      pk[c][i] = pack_bf16(p0, p1);
     }
-    tmem_st_x16(s_addr + c * 16, pk);
   }
   float s0, s1, s2, s3;
   unpack2(sum_a, s0, s1);
@@ -303,16 +304,17 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   if (tid == 0) {
     s.abort_flag = 0;
     mbar_init(&s.q_full, 1);
-    mbar_init(&s.q_free, 1);
+    mbar_init(&s.q_free, 2);  // one arrival per issuer
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&s.kv_full[i], 1);
-      mbar_init(&s.kv_empty[i], 1);
+      mbar_init(&s.kv_empty[i], 2);  // one arrival per issuer, whether or not its tile uses the block
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&s.s_full[i], 1);
-      mbar_init(&s.p_ready[i], 128);
-      mbar_init(&s.o_done[i], 1);
-    }
+    for (int i = 0; i < 2; ++i)
+      for (int h = 0; h < 2; ++h) {
+        mbar_init(&s.s_full[i][h], 1);
+        mbar_init(&s.p_ready[i][h], 128);
+        mbar_init(&s.o_done[i][h], 1);
+      }
     fence_mbar_init();
   }
   if (warp == 8) {
@@ -374,110 +376,163 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       }
     }
     __syncwarp();
-  } else if (warp == 9) {
-    // =============================================================== MMA issuer
+  } else if (warp == 9 || warp == 10) {
+    // =============================================================== MMA issuers, one thread per tile
     reg_dealloc<kRegsOther>();
-    constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 128, false, false);
-    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, false, true);
+    constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 64, false, false);   // S half: 128 x 64
+    constexpr uint32_t idesc_pv = umma_idesc_bf16(128, 128, false, true);   // O: 128 x 128
     if (lane == 0) {
-      uint32_t ecount_base = 0;
-      uint32_t pv_count[2] = {0, 0};  // P-ready phases consumed per tile
+      const int t = warp - 9;
+      const uint32_t flag_t = t == 0 ? kFlag0 : kFlag1;
+      uint32_t ecount_base = 0;  // ring index of the item's first entry
+      uint32_t p_count = 0;      // steps whose P has been consumed (phase of p_ready)
       int it_count = 0;
       bool ok = true;
 
       // Operand descriptors are built once; inside the loops only the 14-bit start-address field moves
       // (a compile-time offset per K step), so issuing an MMA costs two integer adds.
-      const uint64_t q_desc[2] = {umma_desc_sw128(smem_u32(s.q[0][0]), 0, 1024),
-                                  umma_desc_sw128(smem_u32(s.q[1][0]), 0, 1024)};
+      const uint64_t q_desc = umma_desc_sw128(smem_u32(s.q[t][0]), 0, 1024);
       // slot s of the ring starts 32 KB after slot s - 1: +2048 in the descriptor's address field
       const uint64_t k_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 0, 1024);      // K block: K-major B operand
       const uint64_t v_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 16384, 1024);  // V block: MN-major B operand
-      uint32_t k_seen = 0xffffffffu, v_seen = 0xffffffffu;  // loads whose arrival has been observed already
+      const uint32_t s_tm = tm + t * 128, o_tm = tm + 256 + t * 128;
 
-      auto issue_qk = [&](int t, uint32_t ecount, bool last_use, bool last_of_item) {
-        const uint32_t load = 2u * ecount;
-        const int st = load % kStages;
-        if (k_seen != load) {
-          ok = ok && mbar_wait(&s.kv_full[st], (load / kStages) & 1, abort_flag);
-          k_seen = load;
+      // Every issuer observes every load of the ring in order and releases every slot once (a commit
+      // behind the MMAs that read it, a plain arrival for a block only the other tile uses).  A slot is
+      // therefore never refilled before both have seen it, so a phase parity can never be mistaken for
+      // the one two refills earlier or later.
+      uint32_t observed = 0;  // loads [0, observed) have been seen complete by this thread
+      auto wait_next_load = [&]() {
+        ok = ok && mbar_wait(&s.kv_full[observed % kStages], (observed / kStages) & 1, abort_flag);
+        ++observed;
+      };
+      // observe and release the loads in [observed, load_end): blocks of the other tile
+      auto skip_to = [&](uint32_t load_end) {
+        while (observed < load_end && ok) {
+          const int slot = observed % kStages;
+          wait_next_load();
+          if (ok) mbar_arrive(&s.kv_empty[slot]);
         }
-        if (!ok) return;
-        tc_fence_after_sync();
-        const uint64_t ad0 = q_desc[t], bd0 = k_desc0 + static_cast<uint64_t>(st) * 2048u;
-        const uint32_t dst = tm + t * 128;
+      };
+      // One step of this tile: ring index of its entry; whether it is the tile's last step (its diagonal).
+      struct Step {
+        uint32_t ec;
+        bool last;
+      };
+      // S half h (keys 64 h .. 64 h + 63) = Q_t K_h^T: eight K steps of 16 dims, N = 64
+      auto mma_qk_half = [&](const Step& st, int h) {
+        const int slot = (2u * st.ec) % kStages;
+        // key rows 64-127 of the block start 64 x 128 B further into each 64-dim half
+        const uint64_t bd0 = k_desc0 + static_cast<uint64_t>(slot) * 2048u + static_cast<uint64_t>(h) * (8192u >> 4);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           // K step kk: 64-column half kk / 4 (16 KB apart), 32 bytes per step inside the swizzle atom
           constexpr uint32_t kHalf = 16384 >> 4, kStep = 32 >> 4;
           const uint64_t off = static_cast<uint64_t>((kk >> 2) * kHalf + (kk & 3) * kStep);
-          umma_ss(dst, ad0 + off, bd0 + off, idesc_qk, kk > 0);
+          umma_ss(s_tm + h * 64, q_desc + off, bd0 + off, idesc_qk, kk > 0);
         }
-        umma_commit(&s.s_full[t]);
-        if (last_use) umma_commit(&s.kv_empty[st]);
-        if (last_of_item) umma_commit(&s.q_free);
+        umma_commit(&s.s_full[t][h]);
+        if (h == 1) {
+          umma_commit(&s.kv_empty[slot]);
+          if (st.last) umma_commit(&s.q_free);
+        }
       };
-      auto issue_pv = [&](int t, uint32_t ecount, bool last_use, bool first_of_tile) {
-        const uint32_t load = 2u * ecount + 1u;
-        const int st = load % kStages;
-        const uint64_t bd0 = v_desc0 + static_cast<uint64_t>(st) * 2048u;
-        const uint32_t dst = tm + 256 + t * 128, src = tm + t * 128;
-        ok = ok && mbar_wait(&s.p_ready[t], pv_count[t] & 1, abort_flag);
-        if (v_seen != load) {
-          ok = ok && mbar_wait(&s.kv_full[st], (load / kStages) & 1, abort_flag);
-          v_seen = load;
-        }
-        if (!ok) return;
-        ++pv_count[t];
-        tc_fence_after_sync();
+      // O_t += P_h V_h: four steps of 16 keys; P_h (bf16) sits in columns 64 + 32 h .. of the tile's S region
+      auto mma_pv_half = [&](const Step& st, int h, bool first) {
+        const int slot = (2u * st.ec + 1u) % kStages;
+        const uint64_t bd0 = v_desc0 + static_cast<uint64_t>(slot) * 2048u;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
+        for (int k4 = 0; k4 < 4; ++k4) {
+          const int kk = h * 4 + k4;
           // V block as the MN-major B operand: 16 keys per step = two groups of 8 key rows = 2048 B
           const uint64_t off = static_cast<uint64_t>(kk * (2048 >> 4));
-          umma_ts(dst, src + kk * 8, bd0 + off, idesc_pv, (kk > 0 || !first_of_tile) ? 1u : 0u);
+          umma_ts(o_tm, s_tm + 64 + kk * 8, bd0 + off, idesc_pv, (kk > 0 || !first) ? 1u : 0u);
         }
-        umma_commit(&s.o_done[t]);
-        if (last_use) umma_commit(&s.kv_empty[st]);
+        umma_commit(&s.o_done[t][h]);
+        if (h == 1) umma_commit(&s.kv_empty[slot]);
       };
 
       for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x, ++it_count) {
         const Item it = decode_item<kDense>(idx, d, a);
-        EntryStream<kDense> rd;
-        rd.init(it, a);
         ok = mbar_wait(&s.q_full, it_count & 1, abort_flag);
         if (!ok) break;
-        // pending step whose P*V has not been issued yet
-        bool have_prev = false;
-        int prev_t = 0;
-        uint32_t prev_ec = 0;
-        bool prev_last_use = false, prev_first = false;
-        bool seen[2] = {false, false};
-        for (int e = 0; e < it.n_entries && ok; ++e) {
-          const uint32_t ent = rd.get(e);
-          const bool f0 = (ent & kFlag0) != 0, f1 = (ent & kFlag1) != 0;
-          const uint32_t ec = ecount_base + e;
-          for (int t = 0; t < 2; ++t) {
-            if (!(t == 0 ? f0 : f1)) continue;
-            const bool last_use = (t == 1) || !f1;
-            // the last step of an item is the diagonal block of its last tile
-            const bool last_of_item = (e == it.n_entries - 1) && last_use;
-            if (have_prev && prev_t != t) {
-              issue_qk(t, ec, last_use, last_of_item);
-              issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
-            } else if (have_prev) {
-              issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
-              issue_qk(t, ec, last_use, last_of_item);
-            } else {
-              issue_qk(t, ec, last_use, last_of_item);
-            }
-            have_prev = true;
-            prev_t = t;
-            prev_ec = ec;
-            prev_last_use = last_use;
-            prev_first = !seen[t];
-            seen[t] = true;
-          }
+        const uint32_t item_loads_end = 2u * (ecount_base + it.n_entries);
+        if (t == 1 && !it.tile1) {
+          // an item without a second tile: see its loads through and release Q
+          skip_to(item_loads_end);
+          if (ok) mbar_arrive(&s.q_free);
+          ecount_base += it.n_entries;
+          continue;
         }
-        if (have_prev && ok) issue_pv(prev_t, prev_ec, prev_last_use, prev_first);
+        EntryStream<kDense> rd;
+        rd.init(it, a);
+        int e = 0;
+        // next step of this tile: walks the union list (flags only, never waits)
+        auto find_next = [&](Step& st) {
+          while (e < it.n_entries) {
+            const uint32_t ent = rd.get(e);
+            ++e;
+            if (ent & flag_t) {
+              st.ec = ecount_base + e - 1;
+              st.last = static_cast<int>(ent & kColMask) == (t == 0 ? it.m0 : it.m1);
+              return true;
+            }
+          }
+          return false;
+        };
+
+        Step cur, nx;
+        bool have = find_next(cur);
+        if (have) {
+          skip_to(2u * cur.ec);
+          wait_next_load();  // K of the first step
+          if (!ok) break;
+          tc_fence_after_sync();
+          mma_qk_half(cur, 0);
+          mma_qk_half(cur, 1);
+        }
+        // ---- steady state, two bursts per step.  The softmax hands P over in two halves; P lives in the
+        // columns of S half B, so the columns of S half A are free as soon as P_A has been written (the
+        // softmax has read both halves by then): the burst behind P_A is P_A V_A followed by the NEXT step's
+        // Q K_A^T, the burst behind P_B is P_B V_B followed by the next Q K_B^T.  The softmax of the next step
+        // therefore finds its first half waiting and its second half arrives while it works on the first:
+        // neither the softmax nor the tensor pipe waits for a whole step of the other.
+        bool first = true;
+        while (have && ok) {
+          const bool have_nx = find_next(nx);
+          wait_next_load();  // V of this step (the load after its K)
+          // The next K block may be waited for before this step's V is released only if it is at most two
+          // entries ahead (a later one reuses the slot V sits in).
+          const bool early = have_nx && nx.ec <= cur.ec + 2u;
+          if (early) {
+            skip_to(2u * nx.ec);
+            wait_next_load();
+          }
+          ok = ok && mbar_wait(&s.p_ready[t][0], p_count & 1, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          mma_pv_half(cur, 0, first);
+          if (early) mma_qk_half(nx, 0);
+          ok = mbar_wait(&s.p_ready[t][1], p_count & 1, abort_flag);
+          if (!ok) break;
+          ++p_count;
+          tc_fence_after_sync();
+          mma_pv_half(cur, 1, false);
+          if (have_nx) {
+            if (!early) {
+              skip_to(2u * nx.ec);
+              wait_next_load();
+              if (!ok) break;
+              tc_fence_after_sync();
+              mma_qk_half(nx, 0);
+            }
+            mma_qk_half(nx, 1);
+          }
+          first = false;
+          cur = nx;
+          have = have_nx;
+        }
+        skip_to(item_loads_end);  // blocks after this tile's diagonal belong to the other tile
         ecount_base += it.n_entries;
       }
     }
@@ -490,8 +545,20 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t s_addr = tm + lane_addr + t * 128;
     const uint32_t o_addr = tm + lane_addr + 256 + t * 128;
-    uint32_t step_count = 0;  // steps of this tile so far (all items): phase of s_full / o_done
+    uint32_t step_count = 0;  // steps of this tile so far (all items): phase of s_full / p_ready / o_done
     bool ok = true;
+    // In-place rescale of the accumulator by 2^(m_used - m_new); every P*V issued so far must have completed.
+    auto rescale_o = [&](float f) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t ov[32];
+        tmem_ld_x32(o_addr + c * 32, ov);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
+        tmem_st_x32(o_addr + c * 32, ov);
+      }
+    };
     for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
       const Item it = decode_item<kDense>(idx, d, a);
       if (t == 1 && !it.tile1) continue;
@@ -504,62 +571,71 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const uint32_t ent = rd.get(e, it.n_entries, lane);
         if (!(ent & (t == 0 ? kFlag0 : kFlag1))) continue;
         const int J = static_cast<int>(ent & kColMask);
-        ok = mbar_wait_warp(&s.s_full[t], step_count & 1, abort_flag);
+        const bool diag = (J == m_t);
+        const uint32_t ph = step_count & 1;
+        // Each 64-key half is one step of the online softmax.  The rescale decision is taken per warp
+        // (the TMEM accesses are warp-collective): if any row of the warp outgrew its reference maximum by
+        // more than the threshold, every row of the warp moves to its own current maximum.
+        // ---------------- half A: keys 0-63
+        ok = mbar_wait_warp(&s.s_full[t][0], ph, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        uint32_t x[4][32];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld_x32(s_addr + c * 32, x[c]);
+        uint32_t x[2][32];
+        tmem_ld_x32(s_addr, x[0]);
+        tmem_ld_x32(s_addr + 32, x[1]);
         tmem_ld_wait();
-        const bool diag = (J == m_t);
-        float mx;
-        if (diag) {
-          mx = row_max<true>(x, r);
-        } else {
-          mx = row_max<false>(x, r);
-        }
-        mx *= d.scale_log2;
-        // The rescale decision is taken per warp (the TMEM accesses below are warp-collective):
-        // if any row of the warp outgrew its reference maximum by more than the threshold, every row
-        // of the warp moves to its own current maximum.
-        const bool grow = !first && __any_sync(0xffffffffu, mx > m_used + kRescaleThreshold);
+        float mx = (diag ? row_max<true>(x, r, 0) : row_max<false>(x, r, 0)) * d.scale_log2;
         if (first) {
-          m_used = mx;
-        } else if (grow) {
-          // rescale the accumulator in place once every earlier P*V of this tile has completed
-          ok = mbar_wait_warp(&s.o_done[t], (step_count - 1) & 1, abort_flag);
+          m_used = mx;  // key 0 is visible to every row, so this is finite
+        } else if (__any_sync(0xffffffffu, mx > m_used + kRescaleThreshold)) {
+          // the latest P*V issued is the second half of the previous step
+          ok = mbar_wait_warp(&s.o_done[t][1], ph ^ 1u, abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           const float m_new = fmaxf(m_used, mx);
           const float f = ex2(m_used - m_new);
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint32_t ov[32];
-            tmem_ld_x32(o_addr + c * 32, ov);
-            tmem_ld_wait();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
-            tmem_st_x32(o_addr + c * 32, ov);
-          }
+          rescale_o(f);
           l_run *= f;
           m_used = m_new;
         }
-        float sum;
-        if (diag) {
-          sum = exp_pack_store<true>(x, r, d.scale_log2, m_used, s_addr);
-        } else {
-          sum = exp_pack_store<false>(x, r, d.scale_log2, m_used, s_addr);
-        }
-        l_run += sum;
+        uint32_t pk[2][16];
+        l_run += diag ? exp_pack<true>(x, r, 0, d.scale_log2, m_used, pk) : exp_pack<false>(x, r, 0, d.scale_log2, m_used, pk);
+        // ---------------- half B: keys 64-127.  Its logits leave TMEM before P_A goes into their columns.
+        ok = mbar_wait_warp(&s.s_full[t][1], ph, abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        tmem_ld_x32(s_addr + 64, x[0]);
+        tmem_ld_x32(s_addr + 96, x[1]);
+        tmem_ld_wait();
+        tmem_st_x16(s_addr + 64, pk[0]);
+        tmem_st_x16(s_addr + 80, pk[1]);
         tmem_st_wait();
         tc_fence_before_sync();
-        mbar_arrive(&s.p_ready[t]);
+        mbar_arrive(&s.p_ready[t][0]);
+        mx = (diag ? row_max<true>(x, r, 64) : row_max<false>(x, r, 64)) * d.scale_log2;
+        if (__any_sync(0xffffffffu, mx > m_used + kRescaleThreshold)) {
+          // the latest P*V issued is the first half of this step
+          ok = mbar_wait_warp(&s.o_done[t][0], ph, abort_flag);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const float m_new = fmaxf(m_used, mx);
+          const float f = ex2(m_used - m_new);
+          rescale_o(f);
+          l_run *= f;
+          m_used = m_new;
+        }
+        l_run += diag ? exp_pack<true>(x, r, 64, d.scale_log2, m_used, pk) : exp_pack<false>(x, r, 64, d.scale_log2, m_used, pk);
+        tmem_st_x16(s_addr + 96, pk[0]);
+        tmem_st_x16(s_addr + 112, pk[1]);
+        tmem_st_wait();
+        tc_fence_before_sync();
+        mbar_arrive(&s.p_ready[t][1]);
         first = false;
         ++step_count;
       }
       if (!ok) break;
       // ---- epilogue: wait for the last P*V of this tile, normalise, store
-      ok = mbar_wait_warp(&s.o_done[t], (step_count - 1) & 1, abort_flag);
+      ok = mbar_wait_warp(&s.o_done[t][1], (step_count - 1) & 1, abort_flag);
       if (!ok) break;
       tc_fence_after_sync();
       const float inv = 1.0f / l_run;
