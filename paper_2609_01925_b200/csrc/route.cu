@@ -50,6 +50,8 @@ struct ProxySmem {
   int abort_flag;
 };
 
+// kRagged: n is not a multiple of 128 (third band possible); the aligned instantiation drops its predicates.
+template <bool kRagged>
 __global__ void __launch_bounds__(160)
 proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const Dims d, const RoutePtrs w, int* status) {
@@ -145,7 +147,52 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       __syncwarp();
       if (lane == 0) mbar_arrive(&s.bar_s_free[b]);
 
-      float mx = -INFINITY;
+      float mx, lo = 0.f, up = 0.f, hi = 0.f, anc = 0.f;
+      bool any = true;
+      if (!kRagged && vis_up) {
+        // ---- interior tile of an aligned sequence (all but the last tile): every key is visible, and the
+        // band of key jl is decided by jl <= i alone.  Rows of warp w lie in [32 w, 32 w + 31], so a
+        // 32-key chunk c lies wholly on/below the diagonal for c < w and wholly above it for c > w: only
+        // the chunk c == w needs a per-key test.
+        float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int t = 0; t < 32; t += 2) {
+            m0 = fmaxf(m0, __uint_as_float(r[c][t]));
+            m1 = fmaxf(m1, __uint_as_float(r[c][t + 1]));
+          }
+        mx = fmaxf(m0, m1) * d.scale_log2;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float s0 = 0.f, s1 = 0.f, d0 = 0.f, u0 = 0.f;
+#pragma unroll
+          for (int t = 0; t < 32; t += 2) {
+            const float e0 = ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
+            const float e1 = ex2(fmaf(__uint_as_float(r[c][t + 1]), d.scale_log2, -mx));
+            s0 += e0;
+            s1 += e1;
+            if (c == warp) {
+              d0 += (c * 32 + t <= i ? e0 : 0.f) + (c * 32 + t + 1 <= i ? e1 : 0.f);
+              u0 += (c * 32 + t <= i ? 0.f : e0) + (c * 32 + t + 1 <= i ? 0.f : e1);
+            }
+            if (has_slot) {
+              anc += (c * 32 + t < js || c * 32 + t >= jl) ? e0 : 0.f;
+              anc += (c * 32 + t + 1 < js || c * 32 + t + 1 >= jl) ? e1 : 0.f;
+            }
+          }
+          const float sum = s0 + s1;
+          if (c < warp) {
+            lo += sum;
+          } else if (c > warp) {
+            up += sum;
+          } else {
+            lo += d0;
+            up += u0;
+          }
+        }
+      } else {
+      mx = -INFINITY;
 #pragma unroll
       for (int c = 0; c < 4; ++c)
 #pragma unroll
@@ -153,33 +200,33 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
           const int j = c * 32 + t;
           const float x = __uint_as_float(r[c][t]) * d.scale_log2;
           r[c][t] = __float_as_uint(x);
-          const bool visible = (j <= b_thr) || (j <= a_thr ? vis_lo : vis_up);
+          const bool visible = (kRagged && j <= b_thr) || (j <= a_thr ? vis_lo : vis_up);
           if (visible) mx = fmaxf(mx, x);
         }
       // a row may see no key of this tile (ragged n: the tiles around the proxy block): leave a neutral partial
-      const bool any = mx > -INFINITY;
+      any = mx > -INFINITY;
       if (!any) mx = -1e30f;
-      float lo = 0.f, up = 0.f, hi = 0.f, anc = 0.f;
 #pragma unroll
       for (int c = 0; c < 4; ++c)
 #pragma unroll
         for (int t = 0; t < 32; ++t) {
           const int j = c * 32 + t;
           const float e = ex2(__uint_as_float(r[c][t]) - mx);
-          const bool in_hi = j <= b_thr, in_lo = !in_hi && j <= a_thr, in_up = j > a_thr;
+          const bool in_hi = kRagged && j <= b_thr, in_lo = !in_hi && j <= a_thr, in_up = j > a_thr;
           const bool visible = in_hi || (in_lo && vis_lo) || (in_up && vis_up);
           hi += in_hi ? e : 0.f;
           lo += (in_lo && vis_lo) ? e : 0.f;
           up += (in_up && vis_up) ? e : 0.f;
           anc += (visible && (j < js || j >= jl)) ? e : 0.f;
         }
+      }
       if (!any) lo = up = hi = anc = 0.f;
       const int h = kvh * G + g;
       const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
       w.pm[off] = mx;
       w.plo[off] = lo;
       w.pup[off] = up;
-      if (d.rho > 0) w.phi[off] = hi;
+      if (kRagged) w.phi[off] = hi;
       if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
     }
   }
@@ -346,10 +393,10 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   rc = make_tmap_bf16_nhd(&tk, k, d.n, d.hkv);
   if (rc != CRISP_OK) return rc;
   const size_t smem = sizeof(ProxySmem) + 1024;
-  CRISP_CUDA_TRY(cudaFuncSetAttribute(proxy_partials_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      static_cast<int>(smem)),
+  auto* proxy = d.rho > 0 ? proxy_partials_kernel<true> : proxy_partials_kernel<false>;
+  CRISP_CUDA_TRY(cudaFuncSetAttribute(proxy, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)),
                  "route: smem attribute");
-  proxy_partials_kernel<<<dim3(d.nb, d.hkv), 160, smem, stream>>>(tq, tk, d, w, status);
+  proxy<<<dim3(d.nb, d.hkv), 160, smem, stream>>>(tq, tk, d, w, status);
   row_stats_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w);
   row_final_kernel<<<d.hq, 128, 0, stream>>>(d, w);
   tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v);
