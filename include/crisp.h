@@ -162,7 +162,11 @@ int crisp_sparse_prefill(const crisp_params* p, const void* q, const void* k, co
                          const int64_t* row_ptr, const int32_t* col_idx, void* ws, size_t ws_bytes, void* o,
                          float* lse, void* cuda_stream);
 
-/* Dense causal attention: crisp_sparse_prefill with every causal block listed (the baseline of Section 5). */
+/*
+ * Dense causal attention: crisp_sparse_prefill with every causal block listed (the baseline of Section 5).
+ * Unlike the routed calls it accepts every seq_len from 1 to 8192 * block (sink_tokens and local_tokens are
+ * not read); crisp_workspace_bytes reports route_ws = select_ws = 0 for seq_len < 2 * block.
+ */
 int crisp_dense_prefill(const crisp_params* p, const void* q, const void* k, const void* v, void* ws,
                         size_t ws_bytes, void* o, float* lse, void* cuda_stream);
 
@@ -195,6 +199,39 @@ int crisp_forward(const crisp_params* p, const void* q, const void* k, const voi
                   size_t prefill_ws_bytes, float* c_struct, int32_t* pattern, float* p_v, float* p_s,
                   int64_t* row_ptr, int32_t* col_idx, int64_t capacity, int64_t* nnz_needed, void* o, float* lse,
                   int32_t dense_below_tokens, void* cuda_stream);
+
+/*
+ * A batch of independent sequences of different lengths, packed token-major (Algorithm 1 is defined per
+ * sequence and per head; the paper's experiments use batch size 1, so the packing is this library's).
+ * cu_seqlens is a HOST array of batch + 1 non-decreasing token offsets with cu_seqlens[0] = 0; sequence b holds
+ * tokens cu_seqlens[b] .. cu_seqlens[b+1] - 1 of q, k, v, o; p->seq_len is ignored.  Every sequence is processed
+ * exactly as crisp_forward would process it alone (same kernels, same results bit for bit), one after the other
+ * on the stream; the three workspaces are reused and must be large enough for the longest sequence
+ * (crisp_workspace_bytes with seq_len = that length).  A sequence shorter than max(dense_below_tokens, 2 * block)
+ * gets dense attention (a sequence needs two blocks to be routed); an empty sequence is skipped.
+ * With L_b the length of sequence b, N_b,b = ceil(L_b / block) and blk_off[b] = sum of N_b,b' over b' < b:
+ *   c_struct, pattern  [batch][H_q]
+ *   p_v, p_s           sequence b at element H_q * blk_off[b], laid out [H_q][N_b,b]
+ *   row_ptr            sequence b at element H_q * (blk_off[b] + b), laid out [H_q][N_b,b + 1]; its values index
+ *                      the sequence's own segment of col_idx
+ *   col_idx            sequence b owns elements col_off[b] .. col_off[b+1] - 1, where
+ *                      col_off[b] = floor(capacity * (causal blocks of the routed sequences before b) /
+ *                      (causal blocks of all routed sequences)); capacity >= H_q * that total always suffices
+ *   nnz_needed         [batch] (device), written for routed sequences only
+ *   device_status      optional [batch][2] i32 (device): the status words of the selection stage
+ *                      (CRISP_ERR_CAPACITY when the sequence's share of col_idx was too small; its rows of o are
+ *                      then left untouched) and of the attention stage (CRISP_ERR_DEVICE_TIMEOUT), 0 when fine
+ *   lse                optional; sequence b at element H_q * cu_seqlens[b], laid out [H_q][L_b]
+ * crisp_varlen_layout returns blk_off and col_off (HOST arrays of batch + 1 int64) by the same rule, without
+ * touching the GPU.  Entries of the outputs that belong to dense or empty sequences are not written.
+ */
+int crisp_varlen_layout(const crisp_params* p, const int64_t* cu_seqlens, int32_t batch, int64_t capacity,
+                        int32_t dense_below_tokens, int64_t* blk_off, int64_t* col_off);
+int crisp_forward_varlen(const crisp_params* p, const int64_t* cu_seqlens, int32_t batch, const void* q, const void* k,
+                         const void* v, void* route_ws, size_t route_ws_bytes, void* select_ws, size_t select_ws_bytes,
+                         void* prefill_ws, size_t prefill_ws_bytes, float* c_struct, int32_t* pattern, float* p_v,
+                         float* p_s, int64_t* row_ptr, int32_t* col_idx, int64_t capacity, int64_t* nnz_needed,
+                         int32_t* device_status, void* o, float* lse, int32_t dense_below_tokens, void* cuda_stream);
 
 /*
  * Synchronises `cuda_stream`, reads the status word at the start of `ws`, clears it and returns it

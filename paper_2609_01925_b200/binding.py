@@ -27,7 +27,8 @@ PATTERN_PE, PATTERN_VS = 0, 1
 EXPORTS = (
     "crisp_version", "crisp_status_string", "crisp_last_cuda_error", "crisp_workspace_bytes",
     "crisp_route", "crisp_route_static", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
-    "crisp_poll_device_status", "crisp_forward", "crisp_route_jsd",
+    "crisp_poll_device_status", "crisp_forward", "crisp_route_jsd", "crisp_varlen_layout",
+    "crisp_forward_varlen",
 )
 
 
@@ -98,6 +99,11 @@ def load() -> ctypes.CDLL:
     lib.crisp_forward.restype = ctypes.c_int
     lib.crisp_forward.argtypes = [P, vp, vp, vp, vp, sz, vp, sz, vp, sz, vp, vp, vp, vp, vp, vp, i64, vp, vp, vp,
                                   ctypes.c_int32, vp]
+    lib.crisp_varlen_layout.restype = ctypes.c_int
+    lib.crisp_varlen_layout.argtypes = [P, vp, ctypes.c_int32, i64, ctypes.c_int32, vp, vp]
+    lib.crisp_forward_varlen.restype = ctypes.c_int
+    lib.crisp_forward_varlen.argtypes = [P, vp, ctypes.c_int32, vp, vp, vp, vp, sz, vp, sz, vp, sz, vp, vp, vp, vp,
+                                         vp, vp, i64, vp, vp, vp, vp, ctypes.c_int32, vp]
     lib.crisp_poll_device_status.restype = ctypes.c_int
     lib.crisp_poll_device_status.argtypes = [vp, vp]
     _lib = lib
@@ -186,6 +192,35 @@ def crisp_forward(p, q, k, v, route_ws, select_ws, prefill_ws, c_struct, pattern
                                 _ptr(c_struct), _ptr(pattern), _ptr(p_v), _ptr(p_s), _ptr(row_ptr),
                                 _ptr(col_idx), int(capacity), _ptr(nnz_needed), _ptr(o), _ptr(lse),
                                 int(dense_below_tokens), _stream(stream))
+
+
+def _host_i64(values):
+    arr = (ctypes.c_int64 * len(values))(*[int(x) for x in values])
+    return arr
+
+
+def crisp_varlen_layout(p, cu_seqlens, capacity, dense_below_tokens=0):
+    """(blk_off, col_off) of a packed batch: where each sequence's outputs live (see include/crisp.h)."""
+    batch = len(cu_seqlens) - 1
+    cu = _host_i64(cu_seqlens)
+    blk, col = (ctypes.c_int64 * (batch + 1))(), (ctypes.c_int64 * (batch + 1))()
+    rc = load().crisp_varlen_layout(ctypes.byref(p), cu, batch, int(capacity), int(dense_below_tokens), blk, col)
+    if rc != OK:
+        raise CrispError(rc, "crisp_varlen_layout")
+    return list(blk), list(col)
+
+
+def crisp_forward_varlen(p, cu_seqlens, q, k, v, route_ws, select_ws, prefill_ws, c_struct, pattern, p_v, p_s,
+                         row_ptr, col_idx, capacity, nnz_needed, device_status, o, lse=None, dense_below_tokens=0,
+                         stream=None) -> int:
+    """cu_seqlens: a host sequence of batch + 1 token offsets (list, tuple or CPU tensor)."""
+    cu = _host_i64([int(x) for x in cu_seqlens])
+    return load().crisp_forward_varlen(ctypes.byref(p), cu, len(cu) - 1, _ptr(q), _ptr(k), _ptr(v), _ptr(route_ws),
+                                       _nbytes(route_ws), _ptr(select_ws), _nbytes(select_ws), _ptr(prefill_ws),
+                                       _nbytes(prefill_ws), _ptr(c_struct), _ptr(pattern), _ptr(p_v), _ptr(p_s),
+                                       _ptr(row_ptr), _ptr(col_idx), int(capacity), _ptr(nnz_needed),
+                                       _ptr(device_status), _ptr(o), _ptr(lse), int(dense_below_tokens),
+                                       _stream(stream))
 
 
 def crisp_poll_device_status(ws, stream=None) -> int:

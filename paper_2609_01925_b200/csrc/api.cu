@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "common.cuh"
 
@@ -60,13 +61,18 @@ int make_tmap_bf16_nhd(CUtensorMap* out, const void* base, int n, int heads, int
   return CRISP_OK;
 }
 
-int validate(const crisp_params* p, Dims* d) {
+// dense_only: the call runs dense attention alone, which is defined for every length >= 1 and reads none of
+// the routing parameters' relation to the length.
+int validate(const crisp_params* p, Dims* d, bool dense_only) {
   if (!p) return CRISP_ERR_INVALID_ARG;
   if (p->struct_size != static_cast<int32_t>(sizeof(crisp_params))) return CRISP_ERR_INVALID_ARG;
   if (p->seq_len <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0) return CRISP_ERR_INVALID_ARG;
   if (p->n_q_heads % p->n_kv_heads != 0) return CRISP_ERR_INVALID_ARG;
-  if (p->sink_tokens < 1 || p->sink_tokens > p->seq_len) return CRISP_ERR_INVALID_ARG;
-  if (p->local_tokens < 1 || p->local_tokens > p->seq_len) return CRISP_ERR_INVALID_ARG;
+  // fewer than two blocks cannot be routed; said before the windows are compared with the length
+  if (!dense_only && p->seq_len < 2 * kBlock && p->head_dim == kHeadDim && p->block == kBlock)
+    return CRISP_ERR_UNSUPPORTED;
+  if (p->sink_tokens < 1 || (!dense_only && p->sink_tokens > p->seq_len)) return CRISP_ERR_INVALID_ARG;
+  if (p->local_tokens < 1 || (!dense_only && p->local_tokens > p->seq_len)) return CRISP_ERR_INVALID_ARG;
   if (p->k_min_blocks < 0) return CRISP_ERR_INVALID_ARG;
   if (p->selector < 0 || p->selector > 2) return CRISP_ERR_INVALID_ARG;
   if (p->force_pattern < 0 || p->force_pattern > 2) return CRISP_ERR_INVALID_ARG;
@@ -74,7 +80,7 @@ int validate(const crisp_params* p, Dims* d) {
       !std::isfinite(p->gamma) || !(p->softmax_scale >= 0.f) || !std::isfinite(p->softmax_scale))
     return CRISP_ERR_INVALID_ARG;
   if (p->head_dim != kHeadDim || p->block != kBlock) return CRISP_ERR_UNSUPPORTED;
-  if (p->seq_len < 2 * kBlock) return CRISP_ERR_UNSUPPORTED;
+  if (!dense_only && p->seq_len < 2 * kBlock) return CRISP_ERR_UNSUPPORTED;
   if (p->n_q_heads / p->n_kv_heads > kMaxGroup) return CRISP_ERR_UNSUPPORTED;
   if (p->seq_len > 8192 * kBlock) return CRISP_ERR_UNSUPPORTED;  // N_b limit of the selection kernels (1M tokens)
   d->n = p->seq_len;
@@ -84,8 +90,8 @@ int validate(const crisp_params* p, Dims* d) {
   d->hq = p->n_q_heads;
   d->hkv = p->n_kv_heads;
   d->group = d->hq / d->hkv;
-  d->w_sink = p->sink_tokens;
-  d->w_local = p->local_tokens;
+  d->w_sink = p->sink_tokens < p->seq_len ? p->sink_tokens : p->seq_len;
+  d->w_local = p->local_tokens < p->seq_len ? p->local_tokens : p->seq_len;
   d->n_sink_tiles = (d->w_sink + kBlock - 1) / kBlock;
   if (d->n_sink_tiles > d->nb) d->n_sink_tiles = d->nb;
   int fl = (d->n - d->w_local) / kBlock;
@@ -129,6 +135,15 @@ const char* crisp_last_cuda_error(void) { return g_cuda_error; }
 
 int crisp_workspace_bytes(const crisp_params* p, size_t* route_ws, size_t* select_ws, size_t* prefill_ws) {
   Dims d;
+  if (p && p->seq_len > 0 && p->seq_len < 2 * kBlock) {
+    // too short to be routed: only dense attention applies, and only its workspace is needed
+    const int rc_dense = validate(p, &d, /*dense_only=*/true);
+    if (rc_dense != CRISP_OK) return rc_dense;
+    if (route_ws) *route_ws = 0;
+    if (select_ws) *select_ws = 0;
+    if (prefill_ws) *prefill_ws = prefill_ws_bytes(d);
+    return CRISP_OK;
+  }
   int rc = validate(p, &d);
   if (rc != CRISP_OK) return rc;
   if (route_ws) *route_ws = route_ws_bytes(d);
@@ -188,7 +203,7 @@ int crisp_sparse_prefill(const crisp_params* p, const void* q, const void* k, co
 int crisp_dense_prefill(const crisp_params* p, const void* q, const void* k, const void* v, void* ws,
                         size_t ws_bytes, void* o, float* lse, void* cuda_stream) {
   Dims d;
-  int rc = validate(p, &d);
+  int rc = validate(p, &d, /*dense_only=*/true);
   if (rc != CRISP_OK) return rc;
   if (!q || !k || !v || !ws || !o) return CRISP_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return CRISP_ERR_INVALID_ARG;
@@ -214,13 +229,14 @@ int crisp_forward(const crisp_params* p, const void* q, const void* k, const voi
                   int64_t* row_ptr, int32_t* col_idx, int64_t capacity, int64_t* nnz_needed, void* o, float* lse,
                   int32_t dense_below_tokens, void* cuda_stream) {
   Dims d;
-  int rc = validate(p, &d);
+  const bool gated = p && p->seq_len < dense_below_tokens;
+  int rc = validate(p, &d, gated);
   if (rc != CRISP_OK) return rc;
   if (!q || !k || !v || !o || !prefill_ws) return CRISP_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return CRISP_ERR_INVALID_ARG;
   if (!aligned16(prefill_ws) || prefill_ws_bytes_ < prefill_ws_bytes(d)) return CRISP_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (d.n < dense_below_tokens) {
+  if (gated) {
     // short prompt: routing and selection would cost more than they save
     return launch_prefill(d, q, k, v, nullptr, nullptr, prefill_ws, o, lse, st);
   }
@@ -235,6 +251,125 @@ int crisp_forward(const crisp_params* p, const void* q, const void* k, const voi
   if (rc != CRISP_OK) return rc;
   // the status word of the selection stage gates the attention kernels: lists that did not fit are never read
   return launch_prefill(d, q, k, v, row_ptr, col_idx, prefill_ws, o, lse, st, static_cast<const int*>(select_ws));
+}
+
+namespace {
+// Is sequence length `len` of a packed batch routed (true) or sent to dense attention (false)?
+bool varlen_routed(int64_t len, int32_t dense_below_tokens) {
+  return len >= 2 * kBlock && len >= dense_below_tokens;
+}
+}  // namespace
+
+int crisp_varlen_layout(const crisp_params* p, const int64_t* cu_seqlens, int32_t batch, int64_t capacity,
+                        int32_t dense_below_tokens, int64_t* blk_off, int64_t* col_off) {
+  if (!p || !cu_seqlens || batch < 0 || capacity < 0 || !blk_off || !col_off) return CRISP_ERR_INVALID_ARG;
+  if (p->n_q_heads <= 0) return CRISP_ERR_INVALID_ARG;
+  if (cu_seqlens[0] != 0) return CRISP_ERR_INVALID_ARG;
+  // causal blocks of the routed sequences: the shares of col_idx
+  unsigned __int128 total = 0;
+  blk_off[0] = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int64_t len = cu_seqlens[b + 1] - cu_seqlens[b];
+    if (len < 0 || len > 8192LL * kBlock) return len < 0 ? CRISP_ERR_INVALID_ARG : CRISP_ERR_UNSUPPORTED;
+    const int64_t nb = (len + kBlock - 1) / kBlock;
+    blk_off[b + 1] = blk_off[b] + nb;
+    if (varlen_routed(len, dense_below_tokens)) total += static_cast<unsigned __int128>(nb) * (nb + 1) / 2;
+  }
+  unsigned __int128 run = 0;
+  col_off[0] = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int64_t len = cu_seqlens[b + 1] - cu_seqlens[b];
+    const int64_t nb = (len + kBlock - 1) / kBlock;
+    if (varlen_routed(len, dense_below_tokens)) run += static_cast<unsigned __int128>(nb) * (nb + 1) / 2;
+    col_off[b + 1] = total == 0 ? 0 : static_cast<int64_t>(static_cast<unsigned __int128>(capacity) * run / total);
+  }
+  return CRISP_OK;
+}
+
+int crisp_forward_varlen(const crisp_params* p, const int64_t* cu_seqlens, int32_t batch, const void* q, const void* k,
+                         const void* v, void* route_ws, size_t route_ws_bytes_, void* select_ws,
+                         size_t select_ws_bytes_, void* prefill_ws, size_t prefill_ws_bytes_, float* c_struct,
+                         int32_t* pattern, float* p_v, float* p_s, int64_t* row_ptr, int32_t* col_idx, int64_t capacity,
+                         int64_t* nnz_needed, int32_t* device_status, void* o, float* lse, int32_t dense_below_tokens,
+                         void* cuda_stream) {
+  if (!p || !cu_seqlens || batch < 0) return CRISP_ERR_INVALID_ARG;
+  if (p->struct_size != static_cast<int32_t>(sizeof(crisp_params))) return CRISP_ERR_INVALID_ARG;
+  if (batch == 0) return CRISP_OK;
+  if (!q || !k || !v || !o || !prefill_ws) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return CRISP_ERR_INVALID_ARG;
+  if (capacity < 0 || (capacity > 0 && !col_idx)) return CRISP_ERR_INVALID_ARG;
+  std::vector<int64_t> blk_off, col_off;
+  std::vector<Dims> dims;
+  try {
+    blk_off.resize(static_cast<size_t>(batch) + 1);
+    col_off.resize(static_cast<size_t>(batch) + 1);
+    dims.resize(static_cast<size_t>(batch));
+  } catch (...) {
+    return CRISP_ERR_INVALID_ARG;  // a batch too large to describe on the host
+  }
+  int rc = crisp_varlen_layout(p, cu_seqlens, batch, capacity, dense_below_tokens, blk_off.data(), col_off.data());
+  if (rc != CRISP_OK) return rc;
+
+  // ---- first pass: every sequence's parameters and workspace needs, before anything is enqueued
+  bool any_routed = false;
+  for (int b = 0; b < batch; ++b) {
+    const int64_t len = cu_seqlens[b + 1] - cu_seqlens[b];
+    if (len == 0) continue;
+    crisp_params pb = *p;
+    pb.seq_len = static_cast<int32_t>(len);
+    const bool routed = varlen_routed(len, dense_below_tokens);
+    rc = validate(&pb, &dims[b], !routed);
+    if (rc != CRISP_OK) return rc;
+    if (!aligned16(prefill_ws) || prefill_ws_bytes_ < prefill_ws_bytes(dims[b])) return CRISP_ERR_WORKSPACE;
+    if (routed) {
+      any_routed = true;
+      if (!route_ws || !select_ws) return CRISP_ERR_INVALID_ARG;
+      if (!aligned16(route_ws) || route_ws_bytes_ < route_ws_bytes(dims[b])) return CRISP_ERR_WORKSPACE;
+      if (!aligned16(select_ws) || select_ws_bytes_ < select_ws_bytes(dims[b])) return CRISP_ERR_WORKSPACE;
+    }
+  }
+  if (any_routed && (!c_struct || !pattern || !p_v || !p_s || !row_ptr || !nnz_needed)) return CRISP_ERR_INVALID_ARG;
+
+  // ---- second pass: one sequence after the other on the stream; the workspaces are reused in stream order
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t hq = static_cast<size_t>(p->n_q_heads), hkv = static_cast<size_t>(p->n_kv_heads);
+  for (int b = 0; b < batch; ++b) {
+    const int64_t t0 = cu_seqlens[b], len = cu_seqlens[b + 1] - t0;
+    if (device_status)
+      CRISP_CUDA_TRY(cudaMemsetAsync(device_status + 2 * b, 0, 2 * sizeof(int32_t), st), "forward_varlen: clear status");
+    if (len == 0) continue;
+    const Dims& d = dims[b];
+    const char* qb = static_cast<const char*>(q) + static_cast<size_t>(t0) * hq * kHeadDim * 2;
+    const char* kb = static_cast<const char*>(k) + static_cast<size_t>(t0) * hkv * kHeadDim * 2;
+    const char* vb = static_cast<const char*>(v) + static_cast<size_t>(t0) * hkv * kHeadDim * 2;
+    char* ob = static_cast<char*>(o) + static_cast<size_t>(t0) * hq * kHeadDim * 2;
+    float* lb = lse ? lse + static_cast<size_t>(t0) * hq : nullptr;
+    if (!varlen_routed(len, dense_below_tokens)) {
+      rc = launch_prefill(d, qb, kb, vb, nullptr, nullptr, prefill_ws, ob, lb, st);
+      if (rc != CRISP_OK) return rc;
+    } else {
+      float* cs = c_struct + static_cast<size_t>(b) * hq;
+      int32_t* pat = pattern + static_cast<size_t>(b) * hq;
+      float* pv = p_v + static_cast<size_t>(blk_off[b]) * hq;
+      float* ps = p_s + static_cast<size_t>(blk_off[b]) * hq;
+      int64_t* rp = row_ptr + (static_cast<size_t>(blk_off[b]) + b) * hq;
+      int32_t* ci = col_idx ? col_idx + col_off[b] : nullptr;
+      const int64_t cap = col_off[b + 1] - col_off[b];
+      rc = launch_route(d, qb, kb, route_ws, cs, pat, pv, ps, st);
+      if (rc != CRISP_OK) return rc;
+      rc = launch_select(d, qb, kb, pat, pv, ps, select_ws, rp, ci, cap, nnz_needed + b, st);
+      if (rc != CRISP_OK) return rc;
+      rc = launch_prefill(d, qb, kb, vb, rp, ci, prefill_ws, ob, lb, st, static_cast<const int*>(select_ws));
+      if (rc != CRISP_OK) return rc;
+      if (device_status)
+        CRISP_CUDA_TRY(cudaMemcpyAsync(device_status + 2 * b, select_ws, sizeof(int32_t), cudaMemcpyDeviceToDevice, st),
+                       "forward_varlen: selection status");
+    }
+    if (device_status)
+      CRISP_CUDA_TRY(cudaMemcpyAsync(device_status + 2 * b + 1, prefill_ws, sizeof(int32_t), cudaMemcpyDeviceToDevice, st),
+                     "forward_varlen: attention status");
+  }
+  return CRISP_OK;
 }
 
 int crisp_poll_device_status(void* ws, void* cuda_stream) {

@@ -32,7 +32,7 @@ struct Dims {
   float scale_log2; // scale * log2(e)
 };
 
-int validate(const crisp_params* p, Dims* d);
+int validate(const crisp_params* p, Dims* d, bool dense_only = false);
 void set_cuda_error(cudaError_t e, const char* where);
 void set_cu_error(const char* msg);
 

@@ -49,9 +49,8 @@ def test_workspace_sizes_grow_with_the_problem():
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(seq_len=255), B.ERR_UNSUPPORTED),              # fewer than two blocks
     (dict(seq_len=8192 * 128 + 1), B.ERR_UNSUPPORTED),   # more than 8192 blocks
-    (dict(seq_len=128), B.ERR_UNSUPPORTED),              # fewer than two blocks
+    (dict(seq_len=0), B.ERR_INVALID_ARG),
     (dict(head_dim=64), B.ERR_UNSUPPORTED),
     (dict(block=64), B.ERR_UNSUPPORTED),
     (dict(n_q_heads=6, n_kv_heads=4), B.ERR_INVALID_ARG),
@@ -74,6 +73,50 @@ def test_invalid_parameters_are_rejected(kw, code):
     with pytest.raises(crisp.CrispError) as e:
         B.crisp_workspace_bytes(p)
     assert e.value.status == code
+
+
+@pytest.mark.parametrize("n", [1, 100, 128, 255])
+def test_lengths_below_two_blocks_are_dense_only(n):
+    """Routing needs two blocks (the noise floor divides by N_b - 2 and the proxy block needs a predecessor);
+    dense attention does not: the workspace query says so, and the routed entry points refuse the length
+    before they look at any pointer."""
+    import ctypes
+    p = crisp.make_params(n, 4, 1, sink_tokens=4, local_tokens=128)
+    route_ws, select_ws, prefill_ws = B.crisp_workspace_bytes(p)
+    assert route_ws == 0 and select_ws == 0 and prefill_ws > 0
+    lib = B.load()
+    assert lib.crisp_route(ctypes.byref(p), None, None, None, 0, None, None, None, None, None) == B.ERR_UNSUPPORTED
+    assert lib.crisp_select(ctypes.byref(p), None, None, None, None, None, None, 0, None, None, 0, None,
+                            None) == B.ERR_UNSUPPORTED
+    assert lib.crisp_sparse_prefill(ctypes.byref(p), None, None, None, None, None, None, 0, None, None,
+                                    None) == B.ERR_UNSUPPORTED
+
+
+def test_varlen_layout_rule():
+    """blk_off counts blocks of every sequence; col_off splits the capacity in proportion to the causal block
+    counts of the routed sequences (dense and empty ones get nothing), with floor rounding."""
+    p = crisp.make_params(4096, 4, 2, sink_tokens=4)
+    lens = [300, 0, 1000, 128, 70, 2112]
+    cu = [0]
+    for x in lens:
+        cu.append(cu[-1] + x)
+    nb = [(x + 127) // 128 for x in lens]
+    causal = [b * (b + 1) // 2 if x >= 256 else 0 for x, b in zip(lens, nb)]
+    capacity = 4 * sum(causal) + 3
+    blk, col = B.crisp_varlen_layout(p, cu, capacity)
+    assert blk == [sum(nb[:i]) for i in range(len(lens) + 1)]
+    assert col == [capacity * sum(causal[:i]) // sum(causal) for i in range(len(lens) + 1)]
+    assert col[-1] == capacity and all(b >= a for a, b in zip(col, col[1:]))
+    # the gate moves short sequences to dense: they lose their share
+    blk2, col2 = B.crisp_varlen_layout(p, cu, capacity, dense_below_tokens=512)
+    causal2 = [c if x >= 512 else 0 for c, x in zip(causal, lens)]
+    assert blk2 == blk and col2 == [capacity * sum(causal2[:i]) // sum(causal2) for i in range(len(lens) + 1)]
+    # nothing routed: every share is empty
+    assert B.crisp_varlen_layout(p, [0, 100, 200], 1000)[1] == [0, 0, 0]
+    with pytest.raises(crisp.CrispError):
+        B.crisp_varlen_layout(p, [0, 300, 200], 1000)      # decreasing offsets
+    with pytest.raises(crisp.CrispError):
+        B.crisp_varlen_layout(p, [5, 300], 1000)           # must start at 0
 
 
 def test_ragged_lengths_are_accepted():
