@@ -293,6 +293,13 @@ struct EntryStream {
   }
 };
 
+// Position (in the cost-sorted order) of the item a CTA takes in round `rnd`.  Odd rounds run backwards:
+// with costs falling along the order, CTA 0 would otherwise get the most expensive item of every round.
+__device__ __forceinline__ int item_pos(int rnd) {
+  const int c = (rnd & 1) ? static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x);
+  return rnd * static_cast<int>(gridDim.x) + c;
+}
+
 template <bool kDense>
 __global__ void __launch_bounds__(384, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -341,9 +348,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
     if (lane == 0) {
       uint32_t ecount = 0;
-      int it_count = 0;
       bool ok = true;
-      for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x, ++it_count) {
+      for (int rnd = 0; rnd * static_cast<int>(gridDim.x) < n_items && ok; ++rnd) {
+        const int idx = item_pos(rnd);
+        if (idx >= n_items) break;  // only in the last, partial round
+        const int it_count = rnd;
         const Item it = decode_item<kDense>(idx, d, a);
         EntryStream<kDense> rd;
         rd.init(it, a);
@@ -386,7 +395,6 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const uint32_t flag_t = t == 0 ? kFlag0 : kFlag1;
       uint32_t ecount_base = 0;  // ring index of the item's first entry
       uint32_t p_count = 0;      // steps whose P has been consumed (phase of p_ready)
-      int it_count = 0;
       bool ok = true;
 
       // Operand descriptors are built once; inside the loops only the 14-bit start-address field moves
@@ -452,7 +460,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (h == 1) umma_commit(&s.kv_empty[slot]);
       };
 
-      for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x, ++it_count) {
+      for (int rnd = 0; rnd * static_cast<int>(gridDim.x) < n_items && ok; ++rnd) {
+        const int idx = item_pos(rnd);
+        if (idx >= n_items) break;  // only in the last, partial round
+        const int it_count = rnd;
         const Item it = decode_item<kDense>(idx, d, a);
         ok = mbar_wait(&s.q_full, it_count & 1, abort_flag);
         if (!ok) break;
@@ -559,7 +570,9 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         tmem_st_x32(o_addr + c * 32, ov);
       }
     };
-    for (int idx = blockIdx.x; idx < n_items && ok; idx += gridDim.x) {
+    for (int rnd = 0; rnd * static_cast<int>(gridDim.x) < n_items && ok; ++rnd) {
+      const int idx = item_pos(rnd);
+      if (idx >= n_items) break;  // only in the last, partial round
       const Item it = decode_item<kDense>(idx, d, a);
       if (t == 1 && !it.tile1) continue;
       EntryReader<kDense> rd;
