@@ -176,10 +176,6 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
               d0 += (c * 32 + t <= i ? e0 : 0.f) + (c * 32 + t + 1 <= i ? e1 : 0.f);
               u0 += (c * 32 + t <= i ? 0.f : e0) + (c * 32 + t + 1 <= i ? 0.f : e1);
             }
-            if (has_slot) {
-              anc += (c * 32 + t < js || c * 32 + t >= jl) ? e0 : 0.f;
-              anc += (c * 32 + t + 1 < js || c * 32 + t + 1 >= jl) ? e1 : 0.f;
-            }
           }
           const float sum = s0 + s1;
           if (c < warp) {
@@ -190,6 +186,16 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             lo += d0;
             up += u0;
           }
+        }
+        if (has_slot) {
+          // the few tiles that hold anchor keys (sinks, the local window) take a second pass for their sum
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int t = 0; t < 32; ++t) {
+              const int j = c * 32 + t;
+              if (j < js || j >= jl) anc += ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
+            }
         }
       } else {
       mx = -INFINITY;

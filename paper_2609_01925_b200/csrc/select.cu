@@ -218,11 +218,20 @@ pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is
   // the last block may hold fewer than 128 tokens: rows at or beyond n are not read
   const int valid = min(kBlock, d.n - J * kBlock);
   const int rows = min(max(valid - half * 64, 0), 64);
-#pragma unroll 8
-  for (int t = 0; t < rows; ++t) {
-    const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
-    a0 += v.x;
-    a1 += v.y;
+  if (rows == 64) {
+    // full half block: a fixed trip count keeps all 64 loads of a thread in flight
+#pragma unroll
+    for (int t = 0; t < 64; ++t) {
+      const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
+      a0 += v.x;
+      a1 += v.y;
+    }
+  } else {
+    for (int t = 0; t < rows; ++t) {
+      const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
+      a0 += v.x;
+      a1 += v.y;
+    }
   }
   __shared__ float2 other[64];
   if (half == 1) other[pair] = make_float2(a0, a1);
