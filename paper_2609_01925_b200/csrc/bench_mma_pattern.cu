@@ -1,6 +1,7 @@
 // Stand-alone micro-benchmark of the attention kernel's MMA issue pattern in isolation: one thread per CTA issues
 // 8 SS MMAs (S = Q K^T, both operands in shared memory) and 8 TS MMAs (O += P V, A in TMEM) per step, optionally
-// with the commits and with background bulk copies into shared memory.  Build and run on a B200:
+// with the commits and with background bulk copies into shared memory; then the time of a single MMA
+// instruction for a range of shapes.  Build and run on a B200:
 //   nvcc -gencode arch=compute_100a,code=sm_100a -O2 -std=c++17 -o bench_mma_pattern bench_mma_pattern.cu && ./bench_mma_pattern
 #include <cstdio>
 #include <cuda_runtime.h>
@@ -57,6 +58,46 @@ __global__ void __launch_bounds__(128) mix(int mode, int iters, const uint8_t* g
   tc_fence_before_sync(); __syncthreads();
   if (warp == 0) tmem_dealloc(tm, 512);
 }
+// ---- time of one MMA instruction as a function of its shape: 8192 back-to-back MMAs of one shape per CTA
+struct SweepSmem { alignas(1024) uint8_t a[2][16384]; alignas(1024) uint8_t b[4][16384]; uint64_t bar; uint32_t tmem_base; int abort_flag; };
+template <int N, int TS, int M = 128>
+__global__ void __launch_bounds__(128) shape_sweep(int iters, long long* out) {
+  extern __shared__ uint8_t raw[];
+  SweepSmem& s = *reinterpret_cast<SweepSmem*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5;
+  for (int i = tid; i < (int)(6 * 16384) / 4; i += 128) reinterpret_cast<uint32_t*>(&s)[i] = 0;
+  if (tid == 0) { s.abort_flag = 0; mbar_init(&s.bar, 1); fence_mbar_init(); }
+  if (warp == 0) { tmem_alloc(&s.tmem_base, 512); tmem_relinquish(); }
+  fence_proxy_async_smem(); tc_fence_before_sync(); __syncthreads(); tc_fence_after_sync();
+  const uint32_t tm = s.tmem_base;
+  if (tid == 0) {
+    const uint32_t idesc = umma_idesc_bf16(M, N, false, TS ? true : false);
+    const uint64_t ad0 = umma_desc_sw128(smem_u32(s.a[0]), 0, 1024), bd0 = umma_desc_sw128(smem_u32(s.b[0]), TS ? 16384 : 0, 1024);
+    long long t0 = clock64();
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+      for (int kk = 0; kk < 8; ++kk) {
+        const uint64_t off = (uint64_t)((kk >> 2) * 1024 + (kk & 3) * 2);
+        if (TS) umma_ts(tm + 256, tm + kk * 8, bd0 + (uint64_t)(kk * 128), idesc, 1);
+        else umma_ss(tm + (it & 1) * 256, ad0 + off, bd0 + off, idesc, kk > 0);
+      }
+    }
+    umma_commit(&s.bar);
+    mbar_wait(&s.bar, 0, &s.abort_flag);
+    long long t2 = clock64();
+    if (blockIdx.x == 0) out[0] = t2 - t0;
+  }
+  tc_fence_before_sync(); __syncthreads();
+  if (warp == 0) tmem_dealloc(tm, 512);
+}
+template <int N, int TS, int M = 128> void run_shape(long long* d) {
+  size_t smem = sizeof(SweepSmem) + 1024;
+  cudaFuncSetAttribute(shape_sweep<N, TS, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  shape_sweep<N, TS, M><<<148, 128, smem>>>(1024, d);
+  cudaError_t e = cudaDeviceSynchronize();
+  long long h; cudaMemcpy(&h, d, 8, cudaMemcpyDeviceToHost);
+  printf("%s M=%d N=%3d K=16: %.1f clk per MMA (math floor %.0f)  %s\n", TS ? "TS" : "SS", M, N, h / 8192.0, N / 2.0, cudaGetErrorString(e));
+}
 int main() {
   long long* d; cudaMalloc(&d, 16);
   uint8_t* g; cudaMalloc(&g, (size_t)4096 * 32768); cudaMemset(g, 0, (size_t)4096 * 32768);
@@ -69,5 +110,9 @@ int main() {
     long long h[2]; cudaMemcpy(h, d, 16, cudaMemcpyDeviceToHost);
     printf("%-46s: %.0f clk per (8 SS + 8 TS) step (ideal 1024)  %s\n", names[mode], h[1] / 1024.0, cudaGetErrorString(e));
   }
+  printf("\ncycles per MMA instruction by shape (SS: both operands in shared memory, TS: A in TMEM)\n");
+  run_shape<32, 0>(d); run_shape<64, 0>(d); run_shape<96, 0>(d); run_shape<128, 0>(d); run_shape<192, 0>(d); run_shape<256, 0>(d);
+  run_shape<32, 1>(d); run_shape<64, 1>(d); run_shape<128, 1>(d); run_shape<256, 1>(d);
+  run_shape<64, 0, 64>(d); run_shape<128, 0, 64>(d); run_shape<128, 1, 64>(d);
   return 0;
 }
