@@ -23,6 +23,26 @@ namespace {
 
 constexpr int kChunk = 16;  // key tiles per CTA in the merge kernels
 
+// ---- packed fp32x2 arithmetic (two values per instruction on the FMA pipe)
+__device__ __forceinline__ uint64_t pack2f(float lo, float hi) {
+  uint64_t v;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+  return v;
+}
+__device__ __forceinline__ void unpack2f(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2f(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2f(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 struct RoutePtrs {
   float* pm;       // [hq][nb][128] tile-local max of the scaled logits (base-2 units)
   float* plo;      // [hq][nb][128] sum of 2^(x - max) over entries with key offset <= row
@@ -39,207 +59,265 @@ struct RoutePtrs {
   int n_chunks;
 };
 
+constexpr int kProxyHeads = 4;  // query heads of one KV group handled by one CTA (their proxy queries stay in shared memory)
+
 struct ProxySmem {
-  alignas(1024) uint8_t k[2][16384];      // key tile, two 64-column halves, 128-byte swizzle
-  alignas(1024) uint8_t q[2][2][16384];   // [buffer][half] proxy queries of one head
-  uint64_t bar_k;
-  uint64_t bar_q[2];
-  uint64_t bar_s_full[2];
-  uint64_t bar_s_free[2];
+  alignas(1024) uint8_t q[kProxyHeads][2][16384];  // [head][half] proxy queries, resident for the CTA's lifetime
+  alignas(1024) uint8_t k[2][2][16384];            // [buffer][half] key tiles, two 64-column halves, 128-byte swizzle
+  uint64_t bar_q;
+  uint64_t bar_k_full[2], bar_k_free[2];
+  uint64_t bar_s_full[4], bar_s_free[4];
   uint32_t tmem_base;
   int abort_flag;
 };
 
+// Persistent CTAs, one per SM.  A CTA owns up to four query heads of one KV group - their 128 proxy queries
+// are loaded once and stay in shared memory - and walks over every gridDim.x-th key tile: TMA brings the K
+// tile in (two buffers, the load of the tile after next is issued while the current one is worked on), one
+// thread issues a 128 x 128 x 128 tcgen05 MMA per head into one of four TMEM buffers, and two groups of four
+// warps (one thread per proxy row; group 0 takes the even heads, group 1 the odd ones) reduce the logits to the
+// tile partials.  Two warps per scheduler keep the MUFU busy while the other loads its logits from TMEM.
 // kRagged: n is not a multiple of 128 (third band possible); the aligned instantiation drops its predicates.
 template <bool kRagged>
-__global__ void __launch_bounds__(160)
+__global__ void __launch_bounds__(288, 1)
 proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                      const Dims d, const RoutePtrs w, int* status) {
+                      const Dims d, const RoutePtrs w, int* status, int n_head_chunks) {
   extern __shared__ uint8_t smem_raw[];
   ProxySmem& s = *reinterpret_cast<ProxySmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int J = blockIdx.x, kvh = blockIdx.y;
   const int G = d.group;
+  const int kvh = blockIdx.y / n_head_chunks, g0 = (blockIdx.y % n_head_chunks) * kProxyHeads;
+  const int gc = min(kProxyHeads, G - g0);            // heads of this CTA
+  const int stride = gridDim.x;
+  const int n_my_tiles = static_cast<int>(blockIdx.x) < d.nb ? (d.nb - 1 - static_cast<int>(blockIdx.x)) / stride + 1 : 0;
 
   if (tid == 0) {
     s.abort_flag = 0;
-    mbar_init(&s.bar_k, 1);
+    mbar_init(&s.bar_q, 1);
     for (int b = 0; b < 2; ++b) {
-      mbar_init(&s.bar_q[b], 1);
+      mbar_init(&s.bar_k_full[b], 1);
+      mbar_init(&s.bar_k_free[b], 1);
+    }
+    for (int b = 0; b < 4; ++b) {
       mbar_init(&s.bar_s_full[b], 1);
-      mbar_init(&s.bar_s_free[b], 4);
+      mbar_init(&s.bar_s_free[b], 4);  // one arrival per warp of the group that reads the buffer
     }
     fence_mbar_init();
   }
-  if (warp == 4) {
-    tmem_alloc(&s.tmem_base, 256);
+  if (warp == 8) {
+    tmem_alloc(&s.tmem_base, 512);
     tmem_relinquish();
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tm = s.tmem_base;
+  // jobs (tile, head) of group gr per tile: the even heads for group 0, the odd ones for group 1
+  const int jobs0 = (gc + 1) >> 1, jobs1 = gc >> 1;
 
-  if (warp == 4) {
-    if (lane == 0) {
+  if (warp == 8) {
+    if (lane == 0 && n_my_tiles > 0) {
       // ---- producer + MMA issuer
       prefetch_tmap(&tmap_q);
       prefetch_tmap(&tmap_k);
-      mbar_arrive_expect_tx(&s.bar_k, 32768);
-      tma_load_3d(s.k[0], &tmap_k, &s.bar_k, 0, kvh, J * kBlock);
-      tma_load_3d(s.k[1], &tmap_k, &s.bar_k, 64, kvh, J * kBlock);
-      for (int g = 0; g < G && g < 2; ++g) {
-        mbar_arrive_expect_tx(&s.bar_q[g], 32768);
-        tma_load_3d(s.q[g][0], &tmap_q, &s.bar_q[g], 0, kvh * G + g, d.n - kBlock);
-        tma_load_3d(s.q[g][1], &tmap_q, &s.bar_q[g], 64, kvh * G + g, d.n - kBlock);
+      auto load_k = [&](int n) {
+        const int J = blockIdx.x + n * stride, kb = n & 1;
+        mbar_arrive_expect_tx(&s.bar_k_full[kb], 32768);
+        tma_load_3d(s.k[kb][0], &tmap_k, &s.bar_k_full[kb], 0, kvh, J * kBlock);
+        tma_load_3d(s.k[kb][1], &tmap_k, &s.bar_k_full[kb], 64, kvh, J * kBlock);
+      };
+      load_k(0);
+      mbar_arrive_expect_tx(&s.bar_q, 32768u * gc);
+      for (int g = 0; g < gc; ++g) {
+        tma_load_3d(s.q[g][0], &tmap_q, &s.bar_q, 0, kvh * G + g0 + g, d.n - kBlock);
+        tma_load_3d(s.q[g][1], &tmap_q, &s.bar_q, 64, kvh * G + g0 + g, d.n - kBlock);
       }
-      bool ok = mbar_wait(&s.bar_k, 0, &s.abort_flag);
+      if (n_my_tiles > 1) load_k(1);
+      bool ok = mbar_wait(&s.bar_q, 0, &s.abort_flag);
       constexpr uint32_t idesc = umma_idesc_bf16(128, 128, false, false);
-      for (int g = 0; g < G && ok; ++g) {
-        const int b = g & 1, use = g >> 1;
-        ok = ok && mbar_wait(&s.bar_q[b], use & 1, &s.abort_flag);
-        if (use > 0) ok = ok && mbar_wait(&s.bar_s_free[b], (use - 1) & 1, &s.abort_flag);
-        if (!ok) break;
-        tc_fence_after_sync();
-#pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t ad = umma_desc_sw128(smem_u32(s.q[b][kk >> 2]) + (kk & 3) * 32, 0, 1024);
-          const uint64_t bd = umma_desc_sw128(smem_u32(s.k[kk >> 2]) + (kk & 3) * 32, 0, 1024);
-          umma_ss(tm + b * 128, ad, bd, idesc, kk > 0);
-        }
-        umma_commit(&s.bar_s_full[b]);
-        if (g + 2 < G) {
-          // the query buffer is free again once this MMA has read it
-          ok = ok && mbar_wait(&s.bar_s_full[b], use & 1, &s.abort_flag);
+      const uint64_t q_desc0 = umma_desc_sw128(smem_u32(s.q[0][0]), 0, 1024);
+      const uint64_t k_desc0 = umma_desc_sw128(smem_u32(s.k[0][0]), 0, 1024);
+      for (int n = 0; n < n_my_tiles && ok; ++n) {
+        const int kb = n & 1;
+        ok = mbar_wait(&s.bar_k_full[kb], (n >> 1) & 1, &s.abort_flag);
+        for (int g = 0; g < gc && ok; ++g) {
+          const int gr = g & 1;
+          const int job = n * (gr ? jobs1 : jobs0) + (g >> 1);  // running job number of the group
+          const int buf = gr * 2 + (job & 1), use = job >> 1;
+          if (use > 0) ok = mbar_wait(&s.bar_s_free[buf], (use - 1) & 1, &s.abort_flag);
           if (!ok) break;
-          mbar_arrive_expect_tx(&s.bar_q[b], 32768);
-          tma_load_3d(s.q[b][0], &tmap_q, &s.bar_q[b], 0, kvh * G + g + 2, d.n - kBlock);
-          tma_load_3d(s.q[b][1], &tmap_q, &s.bar_q[b], 64, kvh * G + g + 2, d.n - kBlock);
+          tc_fence_after_sync();
+          // descriptors: only the 14-bit start-address field moves (head: +32 KB, buffer: +32 KB, K step kk:
+          // 16 KB per 64-dim half, 32 B per step inside the swizzle atom), so an MMA costs two integer adds
+          const uint64_t ad0 = q_desc0 + static_cast<uint64_t>(g) * 2048u, bd0 = k_desc0 + static_cast<uint64_t>(kb) * 2048u;
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            constexpr uint32_t kHalf = 16384 >> 4, kStep = 32 >> 4;
+            const uint64_t off = static_cast<uint64_t>((kk >> 2) * kHalf + (kk & 3) * kStep);
+            umma_ss(tm + buf * 128, ad0 + off, bd0 + off, idesc, kk > 0);
+          }
+          umma_commit(&s.bar_s_full[buf]);
+          // As early in this tile as the pipe allows, refill the other buffer (the previous tile's, whose MMAs
+          // were issued a whole tile ago) with the next tile, so its latency hides behind this tile's work.
+          if (g == 0 && n >= 1 && n + 1 < n_my_tiles) {
+            ok = mbar_wait(&s.bar_k_free[kb ^ 1], ((n - 1) >> 1) & 1, &s.abort_flag);
+            if (ok) load_k(n + 1);
+          }
         }
+        if (!ok) break;
+        umma_commit(&s.bar_k_free[kb]);  // the K buffer is free once this tile's MMAs have read it
       }
     }
     __syncwarp();
   } else {
-    // ---- one thread per proxy row
-    const int i = tid;
-    // Offset of proxy row i to local key jl of this tile: o = t_i - j = q * 128 + (rho + i - jl) with
+    // ---- one thread per proxy row; group 0 = warps 0-3, group 1 = warps 4-7
+    const int gr = warp >> 2;
+    const int i = tid & 127;
+    const int wq = warp & 3;  // warp within the group = TMEM sub-partition = rows 32 wq .. 32 wq + 31
+    // Offset of proxy row i to local key jl of a tile: o = t_i - j = q * 128 + (rho + i - jl) with
     // q = nfull - 1 - J and rho = n mod 128.  The entry is visible iff o >= 0 and belongs to the diagonal
     // band of block offset floor(o / 128), which is q - 1 ("up": jl > i + rho), q ("lo") or q + 1
     // ("hi": jl <= i + rho - 128, possible only when rho > 0).  A band with a negative offset is invisible.
-    const int qoff = d.nfull - 1 - J;
-    const int a_thr = i + d.rho;          // jl <= a_thr  <=>  not in the "up" band
+    const int a_thr = i + d.rho;           // jl <= a_thr  <=>  not in the "up" band
     const int b_thr = i + d.rho - kBlock;  // jl <= b_thr  <=>  in the "hi" band
-    const bool vis_up = qoff - 1 >= 0, vis_lo = qoff >= 0;  // "hi" (q + 1 >= 0) is visible whenever it is non-empty
-    const int js = min(max(d.w_sink - J * kBlock, 0), kBlock);            // anchor: local key < js
-    const int jl = min(max(d.n - d.w_local - J * kBlock, 0), kBlock);     // anchor: local key >= jl
-    const bool has_slot = (J < d.n_sink_tiles) || (J >= d.first_local_tile);
-    const int slot = (J < d.n_sink_tiles) ? J : d.n_sink_tiles + (J - d.first_local_tile);
-    const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
-    for (int g = 0; g < G; ++g) {
-      const int b = g & 1, use = g >> 1;
-      if (!mbar_wait(&s.bar_s_full[b], use & 1, &s.abort_flag)) break;
-      tc_fence_after_sync();
-      uint32_t r[4][32];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld_x32(tm + lane_addr + b * 128 + c * 32, r[c]);
-      tmem_ld_wait();
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s.bar_s_free[b]);
-
-      float mx, lo = 0.f, up = 0.f, hi = 0.f, anc = 0.f;
-      bool any = true;
-      if (!kRagged && vis_up) {
-        // ---- interior tile of an aligned sequence (all but the last tile): every key is visible, and the
-        // band of key jl is decided by jl <= i alone.  Rows of warp w lie in [32 w, 32 w + 31], so a
-        // 32-key chunk c lies wholly on/below the diagonal for c < w and wholly above it for c > w: only
-        // the chunk c == w needs a per-key test.
-        float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int t = 0; t < 32; t += 2) {
-            m0 = fmaxf(m0, __uint_as_float(r[c][t]));
-            m1 = fmaxf(m1, __uint_as_float(r[c][t + 1]));
-          }
-        mx = fmaxf(m0, m1) * d.scale_log2;
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          float s0 = 0.f, s1 = 0.f, d0 = 0.f, u0 = 0.f;
-#pragma unroll
-          for (int t = 0; t < 32; t += 2) {
-            const float e0 = ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
-            const float e1 = ex2(fmaf(__uint_as_float(r[c][t + 1]), d.scale_log2, -mx));
-            s0 += e0;
-            s1 += e1;
-            if (c == warp) {
-              d0 += (c * 32 + t <= i ? e0 : 0.f) + (c * 32 + t + 1 <= i ? e1 : 0.f);
-              u0 += (c * 32 + t <= i ? 0.f : e0) + (c * 32 + t + 1 <= i ? 0.f : e1);
-            }
-          }
-          const float sum = s0 + s1;
-          if (c < warp) {
-            lo += sum;
-          } else if (c > warp) {
-            up += sum;
-          } else {
-            lo += d0;
-            up += u0;
-          }
+    const uint32_t lane_addr = static_cast<uint32_t>(wq * 32) << 16;
+    const int my_jobs = gr ? jobs1 : jobs0;
+    int job = 0;
+    bool ok = true;
+    for (int n = 0; n < n_my_tiles && ok; ++n) {
+      const int J = blockIdx.x + n * stride;
+      const int qoff = d.nfull - 1 - J;
+      const bool vis_up = qoff - 1 >= 0, vis_lo = qoff >= 0;  // "hi" (q + 1 >= 0) is visible whenever it is non-empty
+      const int js = min(max(d.w_sink - J * kBlock, 0), kBlock);         // anchor: local key < js
+      const int jl = min(max(d.n - d.w_local - J * kBlock, 0), kBlock);  // anchor: local key >= jl
+      const bool has_slot = (J < d.n_sink_tiles) || (J >= d.first_local_tile);
+      const int slot = (J < d.n_sink_tiles) ? J : d.n_sink_tiles + (J - d.first_local_tile);
+      for (int gj = 0; gj < my_jobs; ++gj, ++job) {
+        const int g = 2 * gj + gr;
+        const int buf = gr * 2 + (job & 1), use = job >> 1;
+        if (!mbar_wait(&s.bar_s_full[buf], use & 1, &s.abort_flag)) {
+          ok = false;
+          break;
         }
-        if (has_slot) {
-          // the few tiles that hold anchor keys (sinks, the local window) take a second pass for their sum
+        tc_fence_after_sync();
+        uint32_t r[4][32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld_x32(tm + lane_addr + buf * 128 + c * 32, r[c]);
+        tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s.bar_s_free[buf]);
+
+        float mx, lo = 0.f, up = 0.f, hi = 0.f, anc = 0.f;
+        bool any = true;
+        if (!kRagged && vis_up) {
+          // ---- interior tile of an aligned sequence (all but the last tile): every key is visible, and the
+          // band of key jl is decided by jl <= i alone.  Rows of warp w lie in [32 w, 32 w + 31], so a
+          // 32-key chunk c lies wholly on/below the diagonal for c < w and wholly above it for c > w: only
+          // the chunk c == w needs a per-key test.
+          float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int t = 0; t < 32; ++t) {
-              const int j = c * 32 + t;
-              if (j < js || j >= jl) anc += ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
+            for (int t = 0; t < 32; t += 2) {
+              m0 = fmaxf(m0, __uint_as_float(r[c][t]));
+              m1 = fmaxf(m1, __uint_as_float(r[c][t + 1]));
             }
+          mx = fmaxf(m0, m1) * d.scale_log2;
+          const uint64_t scale2 = pack2f(d.scale_log2, d.scale_log2), negm2 = pack2f(-mx, -mx);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            uint64_t sa = pack2f(0.f, 0.f), sb = pack2f(0.f, 0.f);
+            if (c != wq) {
+              // the whole chunk lies in one band: packed fp32x2 arithmetic, no per-key test
+#pragma unroll
+              for (int t = 0; t < 32; t += 4) {
+                float a0, a1, b0, b1;
+                unpack2f(fma2f(pack2f(__uint_as_float(r[c][t]), __uint_as_float(r[c][t + 1])), scale2, negm2), a0, a1);
+                unpack2f(fma2f(pack2f(__uint_as_float(r[c][t + 2]), __uint_as_float(r[c][t + 3])), scale2, negm2), b0, b1);
+                sa = add2f(sa, pack2f(ex2(a0), ex2(a1)));
+                sb = add2f(sb, pack2f(ex2(b0), ex2(b1)));
+              }
+              float x0, x1, y0, y1;
+              unpack2f(sa, x0, x1);
+              unpack2f(sb, y0, y1);
+              const float sum = (x0 + x1) + (y0 + y1);
+              if (c < wq) {
+                lo += sum;
+              } else {
+                up += sum;
+              }
+            } else {
+              // the chunk the diagonal crosses: key 32 c + t is on/below it iff t <= i - 32 c
+              const int il = i - 32 * c;
+              float d0 = 0.f, d1 = 0.f, u0 = 0.f, u1 = 0.f;
+#pragma unroll
+              for (int t = 0; t < 32; t += 2) {
+                const float e0 = ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
+                const float e1 = ex2(fmaf(__uint_as_float(r[c][t + 1]), d.scale_log2, -mx));
+                d0 += t <= il ? e0 : 0.f;
+                u0 += t <= il ? 0.f : e0;
+                d1 += t + 1 <= il ? e1 : 0.f;
+                u1 += t + 1 <= il ? 0.f : e1;
+              }
+              lo += d0 + d1;
+              up += u0 + u1;
+            }
+          }
+          if (has_slot) {
+            // the few tiles that hold anchor keys (sinks, the local window) take a second pass for their sum
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+              for (int t = 0; t < 32; ++t) {
+                const int j = c * 32 + t;
+                if (j < js || j >= jl) anc += ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
+              }
+          }
+        } else {
+        mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int t = 0; t < 32; ++t) {
+            const int j = c * 32 + t;
+            const float x = __uint_as_float(r[c][t]) * d.scale_log2;
+            r[c][t] = __float_as_uint(x);
+            const bool visible = (kRagged && j <= b_thr) || (j <= a_thr ? vis_lo : vis_up);
+            if (visible) mx = fmaxf(mx, x);
+          }
+        // a row may see no key of this tile (ragged n: the tiles around the proxy block): leave a neutral partial
+        any = mx > -INFINITY;
+        if (!any) mx = -1e30f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int t = 0; t < 32; ++t) {
+            const int j = c * 32 + t;
+            const float e = ex2(__uint_as_float(r[c][t]) - mx);
+            const bool in_hi = kRagged && j <= b_thr, in_lo = !in_hi && j <= a_thr, in_up = j > a_thr;
+            const bool visible = in_hi || (in_lo && vis_lo) || (in_up && vis_up);
+            hi += in_hi ? e : 0.f;
+            lo += (in_lo && vis_lo) ? e : 0.f;
+            up += (in_up && vis_up) ? e : 0.f;
+            anc += (visible && (j < js || j >= jl)) ? e : 0.f;
+          }
         }
-      } else {
-      mx = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-#pragma unroll
-        for (int t = 0; t < 32; ++t) {
-          const int j = c * 32 + t;
-          const float x = __uint_as_float(r[c][t]) * d.scale_log2;
-          r[c][t] = __float_as_uint(x);
-          const bool visible = (kRagged && j <= b_thr) || (j <= a_thr ? vis_lo : vis_up);
-          if (visible) mx = fmaxf(mx, x);
-        }
-      // a row may see no key of this tile (ragged n: the tiles around the proxy block): leave a neutral partial
-      any = mx > -INFINITY;
-      if (!any) mx = -1e30f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c)
-#pragma unroll
-        for (int t = 0; t < 32; ++t) {
-          const int j = c * 32 + t;
-          const float e = ex2(__uint_as_float(r[c][t]) - mx);
-          const bool in_hi = kRagged && j <= b_thr, in_lo = !in_hi && j <= a_thr, in_up = j > a_thr;
-          const bool visible = in_hi || (in_lo && vis_lo) || (in_up && vis_up);
-          hi += in_hi ? e : 0.f;
-          lo += (in_lo && vis_lo) ? e : 0.f;
-          up += (in_up && vis_up) ? e : 0.f;
-          anc += (visible && (j < js || j >= jl)) ? e : 0.f;
-        }
+        if (!any) lo = up = hi = anc = 0.f;
+        const int h = kvh * G + g0 + g;
+        const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
+        w.pm[off] = mx;
+        w.plo[off] = lo;
+        w.pup[off] = up;
+        if (kRagged) w.phi[off] = hi;
+        if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
       }
-      if (!any) lo = up = hi = anc = 0.f;
-      const int h = kvh * G + g;
-      const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
-      w.pm[off] = mx;
-      w.plo[off] = lo;
-      w.pup[off] = up;
-      if (kRagged) w.phi[off] = hi;
-      if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
     }
   }
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0 && s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
-  if (warp == 4) tmem_dealloc(tm, 256);
+  if (warp == 8) tmem_dealloc(tm, 512);
 }
 
 // Per (head, chunk of tiles): running max and sum of every proxy row over the chunk's tiles.
@@ -402,7 +480,17 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   auto* proxy = d.rho > 0 ? proxy_partials_kernel<true> : proxy_partials_kernel<false>;
   CRISP_CUDA_TRY(cudaFuncSetAttribute(proxy, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)),
                  "route: smem attribute");
-  proxy<<<dim3(d.nb, d.hkv), 160, smem, stream>>>(tq, tk, d, w, status);
+  // one CTA per SM: the (KV head, chunk of four query heads) groups share the SMs evenly, each group's CTAs
+  // split its key tiles
+  int dev = 0, n_sm = 0;
+  CRISP_CUDA_TRY(cudaGetDevice(&dev), "route: current device");
+  CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "route: SM count");
+  const int n_head_chunks = (d.group + kProxyHeads - 1) / kProxyHeads;
+  const int groups = d.hkv * n_head_chunks;
+  int slices = n_sm / groups;
+  if (slices < 1) slices = 1;
+  if (slices > d.nb) slices = d.nb;
+  proxy<<<dim3(slices, groups), 288, smem, stream>>>(tq, tk, d, w, status, n_head_chunks);
   row_stats_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w);
   row_final_kernel<<<d.hq, 128, 0, stream>>>(d, w);
   tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v);
