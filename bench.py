@@ -170,6 +170,9 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="L512k", choices=list(synth.CONFIGS))
+    ap.add_argument("--seq-len", type=int, default=0,
+                    help="instead of a named workload: the Llama-shaped recipe (32/8 heads) at this many tokens "
+                         "(context-length sweeps)")
     ap.add_argument("--impl", default="crisp", choices=["crisp", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -180,6 +183,8 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     w = synth.CONFIGS[args.workload]
+    if args.seq_len > 0:
+        w = synth.llama_shaped(f"Llama-shaped-{args.seq_len}", args.seq_len, n_columns=max(16, args.seq_len // 2048))
     config = {"workload": f"{w.name}: n={w.seq_len}, H_q/H_kv={w.n_q_heads}/{w.n_kv_heads}, d=128, B=128, "
                           f"alpha={w.alpha}, tau={w.tau}, gamma={w.gamma}, w_sink={w.sink_tokens}, "
                           f"w_local={w.local_tokens}, k_min={w.k_min_blocks}",
