@@ -50,6 +50,38 @@ int make_tmap_bf16_nhd(CUtensorMap* out, const void* base, int n, int heads, int
     }                                            \
   } while (0)
 
+#ifdef __CUDACC__
+// Exclusive prefix sum over the 1024 threads of a block, in thread order (warp shuffles, then the 32 warp
+// totals).  `scratch` holds 33 values; `*total` (optional) receives the sum of all threads.  Every thread of
+// the block must call it; it contains two __syncthreads and leaves `scratch` reusable after the second.
+__device__ __forceinline__ long long block_exclusive_scan_1024(long long v, long long* scratch, long long* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  long long incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  __syncthreads();  // scratch may still be read from a previous call
+  if (lane == 31) scratch[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const long long wt = scratch[lane];
+    long long wi = wt;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const long long t = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += t;
+    }
+    scratch[lane] = wi - wt;
+    if (lane == 31) scratch[32] = wi;
+  }
+  __syncthreads();
+  if (total) *total = scratch[32];
+  return scratch[warp] + (incl - v);
+}
+#endif
+
 // stage launchers (each enqueues on `stream` and returns a crisp_status)
 int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c_struct, int32_t* pattern,
                  float* p_v, float* p_s, cudaStream_t stream);

@@ -752,16 +752,13 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
 // run at the same time on the same K/V blocks (L2 reuse); sorting by cost inside a group lets the
 // round-robin assignment balance heads with long lists (PE) against heads with short ones (VS).
 __global__ void __launch_bounds__(1024) sched_scan_kernel(int* __restrict__ cost_hist, int n_bins) {
-  __shared__ int seg_tot[1024];
+  __shared__ long long scratch[33];
   const int tid = threadIdx.x;
   const int seg = (n_bins + 1023) / 1024;
   const int b0 = min(tid * seg, n_bins), b1 = min(b0 + seg, n_bins);
   int local = 0;
   for (int i = b0; i < b1; ++i) local += cost_hist[i];
-  seg_tot[tid] = local;
-  __syncthreads();
-  int run = 0;
-  for (int t = 0; t < tid; ++t) run += seg_tot[t];
+  int run = static_cast<int>(block_exclusive_scan_1024(local, scratch, nullptr));
   for (int i = b0; i < b1; ++i) {
     const int c = cost_hist[i];
     cost_hist[i] = run;  // first position of this key in the sorted order

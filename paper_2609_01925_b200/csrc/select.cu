@@ -391,11 +391,12 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
     }
 }
 
-// One warp per head walks the bins from the largest values down, 32 bins at a time, until the mass
-// reaches gamma.
-__global__ void __launch_bounds__(32)
+// One CTA per head: the bins are read once, in parallel (two per thread, largest values first), an exclusive
+// block scan gives the mass above every bin, and the first non-empty bin at which the mass reaches gamma
+// is the one the cut falls into.
+__global__ void __launch_bounds__(1024)
 pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int level) {
-  const int h = blockIdx.x, lane = threadIdx.x;
+  const int h = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (pattern[h] != CRISP_PATTERN_PE) return;
   const int nbins = level == 2 ? kL2Bins : 2048;
   const int off = level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins);
@@ -412,39 +413,58 @@ pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtr
   }
   const double gd = static_cast<double>(d.gamma) * static_cast<double>(kMassScale);
   const unsigned long long gamma = gd >= 1.8e19 ? 0xffffffffffffffffull : static_cast<unsigned long long>(gd);
-  int found = -1;
-  unsigned long long above = c.mass_above;
-  unsigned int found_count = 0;
-  for (int top = nbins - 1; top >= 0 && found < 0; top -= 32) {
-    const int b = top - lane;
-    const unsigned long long mine = b >= 0 ? gm[b] : 0ull;
-    const unsigned int mycnt = b >= 0 ? gc[b] : 0u;
-    unsigned long long incl = mine;  // inclusive prefix over lanes = over bins from `top` downwards
+
+  // position p (0 = largest values) is bin nbins - 1 - p; thread t owns positions 2t and 2t + 1
+  const int p0 = 2 * tid, p1 = 2 * tid + 1;
+  const unsigned long long m0 = p0 < nbins ? gm[nbins - 1 - p0] : 0ull, m1 = p1 < nbins ? gm[nbins - 1 - p1] : 0ull;
+  const unsigned int c0 = p0 < nbins ? gc[nbins - 1 - p0] : 0u, c1 = p1 < nbins ? gc[nbins - 1 - p1] : 0u;
+  // exclusive scan of the per-thread sums: warp shuffles, then the 32 warp totals
+  __shared__ unsigned long long warp_tot[32];
+  __shared__ int first_hit;
+  __shared__ unsigned long long total_mass;
+  if (tid == 0) first_hit = 0x7fffffff;
+  const unsigned long long mine = m0 + m1;
+  unsigned long long incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    const unsigned long long wt = warp_tot[lane];
+    unsigned long long wi = wt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += t;
+      const unsigned long long t = __shfl_up_sync(0xffffffffu, wi, o);
+      if (lane >= o) wi += t;
     }
-    const bool hit = mycnt != 0u && (above + incl >= gamma);
-    const unsigned int mask = __ballot_sync(0xffffffffu, hit);
-    if (mask) {
-      const int l = __ffs(mask) - 1;
-      found = top - l;
-      above += __shfl_sync(0xffffffffu, incl - mine, l);
-      found_count = __shfl_sync(0xffffffffu, mycnt, l);
-    } else {
-      above += __shfl_sync(0xffffffffu, incl, 31);
-    }
+    warp_tot[lane] = wi - wt;  // mass of the warps before this one
+    if (lane == 31) total_mass = wi;
   }
-  if (lane != 0) return;
-  if (found < 0) {
-    // the target exceeds the total mass (gamma >= 1 or rounding): keep every causal entry
-    c.cutkey = 0u;
-    c.take = -1;
-    c.mass_above = above;
-    w.cut[h] = c;
+  __syncthreads();
+  const unsigned long long before0 = c.mass_above + warp_tot[warp] + (incl - mine);  // mass above position p0
+  const unsigned long long before1 = before0 + m0;
+  const bool hit0 = c0 != 0u && before0 + m0 >= gamma, hit1 = c1 != 0u && before1 + m1 >= gamma;
+  if (hit0 || hit1) atomicMin(&first_hit, hit0 ? p0 : p1);
+  __syncthreads();
+  const int fp = first_hit;
+  if (fp == 0x7fffffff) {
+    if (tid == 0) {
+      // the target exceeds the total mass (gamma >= 1 or rounding): keep every causal entry
+      c.cutkey = 0u;
+      c.take = -1;
+      c.mass_above += total_mass;
+      w.cut[h] = c;
+    }
     return;
   }
+  if (fp != p0 && fp != p1) return;
+  // the thread that owns the bin of the cut finishes the level
+  const int found = nbins - 1 - fp;
+  const unsigned long long above = fp == p0 ? before0 : before1;
+  const unsigned int found_count = fp == p0 ? c0 : c1;
   c.mass_above = above;
   const int shift = level == 0 ? 20 : (level == 1 ? 9 : 0);
   c.prefix |= static_cast<unsigned int>(found) << shift;
@@ -497,16 +517,13 @@ __global__ void __launch_bounds__(1024)
 pe_take_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
   const int h = blockIdx.x, tid = threadIdx.x;
   if (pattern[h] != CRISP_PATTERN_PE) return;
-  __shared__ long long seg_tot[1024];
+  __shared__ long long scratch[33];
   const int seg = (d.nb + 1023) / 1024;
   const int b0 = min(tid * seg, d.nb), b1 = min(b0 + seg, d.nb);
   const size_t base = static_cast<size_t>(h) * d.nb;
   long long local = 0;
   for (int m = b0; m < b1; ++m) local += w.n_eq[base + m];
-  seg_tot[tid] = local;
-  __syncthreads();
-  long long before = 0;
-  for (int t = 0; t < tid; ++t) before += seg_tot[t];
+  long long before = block_exclusive_scan_1024(local, scratch, nullptr);
   const CutState c = w.cut[h];
   for (int m = b0; m < b1; ++m) {
     const int eq = w.n_eq[base + m];
@@ -567,24 +584,35 @@ scan_rows_kernel(const Dims d, const SelectPtrs w, int64_t* __restrict__ row_ptr
                  int64_t* __restrict__ nnz_needed, int* status) {
   const int tid = threadIdx.x;
   const long long total_rows = static_cast<long long>(d.hq) * d.nb;
-  const long long seg = (total_rows + 1023) / 1024;
-  const long long b0 = min(tid * seg, total_rows), b1 = min(b0 + seg, total_rows);
-  __shared__ long long seg_tot[1024];
-  long long local = 0;
-  for (long long r = b0; r < b1; ++r) local += w.counts[r];
-  seg_tot[tid] = local;
-  __syncthreads();
-  long long run = 0;
-  for (int t = 0; t < tid; ++t) run += seg_tot[t];
-  for (long long r = b0; r < b1; ++r) {
-    const int h = static_cast<int>(r / d.nb), m = static_cast<int>(r % d.nb);
-    row_ptr[static_cast<size_t>(h) * (d.nb + 1) + m] = run;
-    run += w.counts[r];
-    if (m == d.nb - 1) row_ptr[static_cast<size_t>(h) * (d.nb + 1) + d.nb] = run;
+  __shared__ long long scratch[33];
+  long long carry = 0;
+  // 4096 consecutive rows per pass, four per thread (coalesced), scanned across the block
+  for (long long base = 0; base < total_rows; base += 4096) {
+    const long long r0 = base + 4 * tid;
+    int c[4];
+    long long local = 0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      c[u] = r0 + u < total_rows ? w.counts[r0 + u] : 0;
+      local += c[u];
+    }
+    long long pass_total;
+    long long run = carry + block_exclusive_scan_1024(local, scratch, &pass_total);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const long long r = r0 + u;
+      if (r < total_rows) {
+        const int h = static_cast<int>(r / d.nb), m = static_cast<int>(r % d.nb);
+        row_ptr[static_cast<size_t>(h) * (d.nb + 1) + m] = run;
+        run += c[u];
+        if (m == d.nb - 1) row_ptr[static_cast<size_t>(h) * (d.nb + 1) + d.nb] = run;
+      }
+    }
+    carry += pass_total;
   }
-  if (tid == 1023) {
-    *nnz_needed = run;
-    if (run > capacity) atomicExch(status, CRISP_ERR_CAPACITY);
+  if (tid == 0) {
+    *nnz_needed = carry;
+    if (carry > capacity) atomicExch(status, CRISP_ERR_CAPACITY);
   }
 }
 
@@ -708,7 +736,7 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   const int hist_ctas = d.nb < 128 ? d.nb : 128;
   for (int level = 0; level < 3; ++level) {
     pe_hist_kernel<<<dim3(hist_ctas, d.hq), 256, 0, stream>>>(d, pattern, w, level);
-    pe_cut_kernel<<<d.hq, 32, 0, stream>>>(d, pattern, w, level);
+    pe_cut_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w, level);
   }
   pe_row_stats_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w);
   pe_take_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w);
