@@ -284,7 +284,12 @@ def main():
     layer.poll()
     clocks = sampler.stop()
 
-    ms_per_step = max_over_ranks(total_ms / args.steps, dist, dev)
+    # A step's time runs from its first launch to its last kernel's end (CUDA events on the launching stream).
+    # Without an L2 flush the steps are back to back and this equals the bracket around all K steps; with a
+    # flush (small workloads) it leaves the flush kernel between two steps out of the path's time.
+    step_ms = [e[0].elapsed_time(e[3]) for e in recs]
+    per_step = total_ms / args.steps if flush is None else sum(step_ms) / len(step_ms)
+    ms_per_step = max_over_ranks(per_step, dist, dev)
     med = {kk: statistics.median(vv) for kk, vv in stage_ms.items()}
     dense = statistics.median(dense_ms)
     sparse_tflops = nnz * FLOP_PER_BLOCK / (med["sparse_prefill"] * 1e-3) / 1e12
