@@ -653,21 +653,27 @@ fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs 
     const float* row = w.amat + (static_cast<size_t>(h) * d.nb + m) * d.nb;
     const int take = w.take[static_cast<size_t>(h) * d.nb + m];
     int ties_seen = 0;
-    for (int J0 = 0; J0 <= m; J0 += 32) {
-      const int J = J0 + lane;
-      bool gt = false, eq = false;
-      if (J <= m) {
-        const unsigned int key = __float_as_uint(row[J]);
-        gt = key > c.cutkey;
-        eq = key == c.cutkey;
+    // 128 columns per pass: the four loads of a lane are issued before the (serial) bookkeeping of the pass
+    for (int J0 = 0; J0 <= m; J0 += 128) {
+      unsigned int key[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int J = J0 + 32 * u + lane;
+        key[u] = J <= m ? __float_as_uint(row[J]) : 0u;
       }
-      const uint32_t eqmask = __ballot_sync(0xffffffffu, eq);
-      const int my_tie = ties_seen + __popc(eqmask & ((1u << lane) - 1u));
-      const bool keep = (J <= m) && (gt || (eq && my_tie < take) || J == 0 || J == m);
-      const uint32_t keepmask = __ballot_sync(0xffffffffu, keep);
-      if (keep) out[written + __popc(keepmask & ((1u << lane) - 1u))] = J;
-      written += __popc(keepmask);
-      ties_seen += __popc(eqmask);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int J = J0 + 32 * u + lane;
+        const bool in = J <= m;
+        const bool gt = in && key[u] > c.cutkey, eq = in && key[u] == c.cutkey;
+        const uint32_t eqmask = __ballot_sync(0xffffffffu, eq);
+        const int my_tie = ties_seen + __popc(eqmask & ((1u << lane) - 1u));
+        const bool keep = in && (gt || (eq && my_tie < take) || J == 0 || J == m);
+        const uint32_t keepmask = __ballot_sync(0xffffffffu, keep);
+        if (keep) out[written + __popc(keepmask & ((1u << lane) - 1u))] = J;
+        written += __popc(keepmask);
+        ties_seen += __popc(eqmask);
+      }
     }
   }
 }
