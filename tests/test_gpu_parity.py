@@ -152,6 +152,17 @@ def test_qwen_shape_reduced():
     _full_check(w, per_head=4)
 
 
+@pytest.mark.parametrize("hq,hkv", [(3, 3), (4, 2), (6, 2), (5, 1), (9, 1), (16, 1)])
+def test_group_sizes(hq, hkv):
+    """Query heads per KV head from 1 to 16: the proxy kernel handles them in chunks of four, two reduction
+    groups taking the even and the odd heads of a chunk; the attention kernel shares K/V blocks per KV head."""
+    pu = _pu()
+    classes = tuple(("conc", "diffuse")[h % 2] for h in range(hq))
+    w = synth.llama_shaped("groups", 2048 + 128, 16).with_(n_q_heads=hq, n_kv_heads=hkv, head_classes=classes,
+                                                          k_min_blocks=2)
+    _full_check(w, per_head=4, dense=False)
+
+
 def test_iid_inputs_custom_scale():
     pu = _pu()
     import paper_2609_01925_b200 as crisp
