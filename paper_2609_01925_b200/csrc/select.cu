@@ -14,8 +14,10 @@
 //     lengths (`count_vs_kernel`), one scan gives row_ptr (`scan_rows_kernel`), a second pass writes the
 //     ascending column lists (`fill_kernel`).  No atomics touch the lists, so they are reproducible.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace crisp {
+using namespace sm100;
 
 namespace {
 
@@ -38,6 +40,8 @@ struct SelectPtrs {
   uint32_t* selsr;  // [hq][words + 2] reversed slash bitmap: bit x = S_s contains N_b-1-x
   float* kbar;      // [hkv][nb][128]
   float* qbar;      // [hq][nb][128]
+  __nv_bfloat16* ksplit;  // [3][nb][hkv][128] block means of K as three bf16 terms (hi + mid + lo = the fp32 mean)
+  __nv_bfloat16* qsplit;  // [3][nb][hq][128]  the same for Q
   float* amat;      // [hq][nb][nb] pooled map (row m uses columns 0..m)
   unsigned int* hcount;  // [hq][kHistStride]
   unsigned long long* hmass;  // [hq][kHistStride] fixed-point mass per bin
@@ -195,7 +199,7 @@ select_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const float*
 // Block means of one [128 tokens, 128 dims] tile per CTA.  x is [n, heads, 128] bf16.
 __global__ void __launch_bounds__(128)
 pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is_query,
-            const int32_t* __restrict__ pattern, float* __restrict__ out) {
+            const int32_t* __restrict__ pattern, float* __restrict__ out, __nv_bfloat16* __restrict__ split) {
   const int J = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
   if (pattern == nullptr) {
     // comparison router: every head's block means are wanted
@@ -234,56 +238,123 @@ pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is
   if (half == 0) {
     float* o = out + (static_cast<size_t>(h) * d.nb + J) * kHeadDim;
     const float inv = 1.0f / static_cast<float>(valid);
-    o[2 * pair] = (a0 + other[pair].x) * inv;
-    o[2 * pair + 1] = (a1 + other[pair].y) * inv;
+    const float m0 = (a0 + other[pair].x) * inv, m1 = (a1 + other[pair].y) * inv;
+    o[2 * pair] = m0;
+    o[2 * pair + 1] = m1;
+    if (split != nullptr) {
+      // mean = hi + mid + lo with three bf16 terms (the remainders are exact in fp32): the pooled logits are
+      // then a sum of bf16 tensor-core products that reproduces the fp32 product to ~2^-24
+      float r0 = m0, r1 = m1;
+#pragma unroll
+      for (int pl = 0; pl < 3; ++pl) {
+        const __nv_bfloat162 t = __floats2bfloat162_rn(r0, r1);
+        reinterpret_cast<__nv_bfloat162*>(split + ((static_cast<size_t>(pl) * d.nb + J) * heads + h) * kHeadDim)[pair] = t;
+        r0 -= __low2float(t);
+        r1 -= __high2float(t);
+      }
+    }
   }
 }
 
-// Pooled logits Z[m, J] = qbar[m] . kbar[J] * scale_log2 for a 64 x 64 tile (fp32 FMA, no tensor
-// cores: the selection compares these values, so they keep full fp32 precision).
-__global__ void __launch_bounds__(256)
-pe_logits_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+// Pooled logits Z[m, J] = qbar[m] . kbar[J] * scale_log2, one 128 x 128 tile of (query block, key block) pairs per
+// CTA, on the tensor cores.  The selection compares these values, so bf16 operands alone would not do: each fp32
+// block mean is split into three bf16 terms (pool_kernel), and the six products hi*hi, hi*mid, mid*hi, mid*mid,
+// hi*lo, lo*hi - accumulated in fp32 in TMEM, smallest first - reproduce the fp32 dot product to ~2^-24.
+struct LogitsMaps {
+  CUtensorMap q[3], k[3];
+};
+struct LogitsSmem {
+  alignas(1024) uint8_t a[3][2][16384];  // [term][64-dim half] 128 block means of Q, 128-byte swizzle
+  alignas(1024) uint8_t b[3][2][16384];  // the same for K
+  uint64_t bar_in, bar_mma;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(160)
+pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const int32_t* __restrict__ pattern,
+                 const SelectPtrs w, int* status) {
   const int jt = blockIdx.x, mt = blockIdx.y, h = blockIdx.z;
   if (jt > mt || pattern[h] != CRISP_PATTERN_PE) return;
-  __shared__ float qs[64][33];
-  __shared__ float ks[64][33];
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
-  const float* qb = w.qbar + (static_cast<size_t>(h) * d.nb + mt * 64) * kHeadDim;
-  const float* kb = w.kbar + (static_cast<size_t>(h / d.group) * d.nb + jt * 64) * kHeadDim;
-  const int mrows = min(64, d.nb - mt * 64), jrows = min(64, d.nb - jt * 64);
-  float acc[4][4] = {};
-  for (int c0 = 0; c0 < kHeadDim; c0 += 32) {
-    for (int idx = tid; idx < 64 * 32; idx += 256) {
-      const int r = idx >> 5, c = idx & 31;
-      qs[r][c] = r < mrows ? qb[static_cast<size_t>(r) * kHeadDim + c0 + c] : 0.f;
-      ks[r][c] = r < jrows ? kb[static_cast<size_t>(r) * kHeadDim + c0 + c] : 0.f;
-    }
-    __syncthreads();
-#pragma unroll 8
-    for (int c = 0; c < 32; ++c) {
-      float a[4], b[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) a[i] = qs[ty + 16 * i][c];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) b[j] = ks[tx + 16 * j][c];
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-    }
-    __syncthreads();
+  extern __shared__ uint8_t smem_raw[];
+  LogitsSmem& s = *reinterpret_cast<LogitsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    s.abort_flag = 0;
+    mbar_init(&s.bar_in, 1);
+    mbar_init(&s.bar_mma, 1);
+    fence_mbar_init();
   }
-  float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
+  if (warp == 4) {
+    tmem_alloc(&s.tmem_base, 128);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tm = s.tmem_base;
+  bool ok = true;
+  if (warp == 4) {
+    if (lane == 0) {
+      mbar_arrive_expect_tx(&s.bar_in, 6u * 32768u);
+      for (int pl = 0; pl < 3; ++pl) {
+        tma_load_3d(s.a[pl][0], &maps.q[pl], &s.bar_in, 0, h, mt * kBlock);
+        tma_load_3d(s.a[pl][1], &maps.q[pl], &s.bar_in, 64, h, mt * kBlock);
+        tma_load_3d(s.b[pl][0], &maps.k[pl], &s.bar_in, 0, h / d.group, jt * kBlock);
+        tma_load_3d(s.b[pl][1], &maps.k[pl], &s.bar_in, 64, h / d.group, jt * kBlock);
+      }
+      ok = mbar_wait(&s.bar_in, 0, &s.abort_flag);
+      if (ok) {
+        tc_fence_after_sync();
+        constexpr uint32_t idesc = umma_idesc_bf16(128, 128, false, false);
+        // (term of Q, term of K), smallest products first
+        const int pa[6] = {2, 0, 1, 1, 0, 0}, pb[6] = {0, 2, 1, 0, 1, 0};
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int m = mt * 64 + ty + 16 * i;
-    if (m >= d.nb) continue;
+        for (int t = 0; t < 6; ++t)
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int J = jt * 64 + tx + 16 * j;
-      if (J <= m) am[static_cast<size_t>(m) * d.nb + J] = acc[i][j] * d.scale_log2;
+          for (int kk = 0; kk < 8; ++kk) {
+            const uint64_t ad = umma_desc_sw128(smem_u32(s.a[pa[t]][kk >> 2]) + (kk & 3) * 32, 0, 1024);
+            const uint64_t bd = umma_desc_sw128(smem_u32(s.b[pb[t]][kk >> 2]) + (kk & 3) * 32, 0, 1024);
+            umma_ss(tm, ad, bd, idesc, (t > 0 || kk > 0) ? 1u : 0u);
+          }
+        umma_commit(&s.bar_mma);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ---- one thread per row of the tile: scale, then through shared memory so that the rows go out coalesced
+    ok = mbar_wait(&s.bar_mma, 0, &s.abort_flag);
+    float* stage = reinterpret_cast<float*>(s.a);  // 128 x 129 floats over the operand tiles, which are dead now
+    if (ok) {
+      tc_fence_after_sync();
+      const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t r[32];
+        tmem_ld_x32(tm + lane_addr + c * 32, r);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) stage[tid * 129 + c * 32 + i] = __uint_as_float(r[i]) * d.scale_log2;
+      }
+    }
+    named_bar_sync(1, 128);
+    if (ok) {
+      float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
+      for (int rr = warp; rr < kBlock; rr += 4) {
+        const int m = mt * kBlock + rr;
+        if (m >= d.nb) break;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const int J = jt * kBlock + c * 32 + lane;
+          if (J <= m) am[static_cast<size_t>(m) * d.nb + J] = stage[rr * 129 + c * 32 + lane];
+        }
+      }
     }
   }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
+  if (warp == 4) tmem_dealloc(tm, 128);
 }
 
 // Row softmax over J <= m, divided by N_b (= the total of the pooled map).
@@ -687,6 +758,8 @@ SelectPtrs carve(const Dims& d, void* ws, size_t* total) {
   w.selsr = static_cast<uint32_t*>(take(sizeof(uint32_t) * d.hq * (w.words + 2)));
   w.kbar = static_cast<float*>(take(sizeof(float) * d.hkv * d.nb * kHeadDim));
   w.qbar = static_cast<float*>(take(sizeof(float) * static_cast<size_t>(d.hq) * d.nb * kHeadDim));
+  w.ksplit = static_cast<__nv_bfloat16*>(take(sizeof(__nv_bfloat16) * 3 * static_cast<size_t>(d.hkv) * d.nb * kHeadDim));
+  w.qsplit = static_cast<__nv_bfloat16*>(take(sizeof(__nv_bfloat16) * 3 * static_cast<size_t>(d.hq) * d.nb * kHeadDim));
   w.amat = static_cast<float*>(take(sizeof(float) * static_cast<size_t>(d.hq) * d.nb * d.nb));
   w.hcount = static_cast<unsigned int*>(take(sizeof(unsigned int) * d.hq * kHistStride));
   w.hmass = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * d.hq * kHistStride));
@@ -729,10 +802,23 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   // PE heads (every kernel returns at once for heads routed to VS)
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
-  pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, kb, d.hkv, 0, pattern, w.kbar);
-  pool_kernel<<<dim3(d.nb, d.hq), 128, 0, stream>>>(d, qb, d.hq, 1, pattern, w.qbar);
-  const int nt = (d.nb + 63) / 64;
-  pe_logits_kernel<<<dim3(nt, nt, d.hq), 256, 0, stream>>>(d, pattern, w);
+  pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, kb, d.hkv, 0, pattern, w.kbar, w.ksplit);
+  pool_kernel<<<dim3(d.nb, d.hq), 128, 0, stream>>>(d, qb, d.hq, 1, pattern, w.qbar, w.qsplit);
+  {
+    LogitsMaps maps;
+    for (int pl = 0; pl < 3; ++pl) {
+      int rc = make_tmap_bf16_nhd(&maps.q[pl], w.qsplit + static_cast<size_t>(pl) * d.nb * d.hq * kHeadDim, d.nb, d.hq);
+      if (rc != CRISP_OK) return rc;
+      rc = make_tmap_bf16_nhd(&maps.k[pl], w.ksplit + static_cast<size_t>(pl) * d.nb * d.hkv * kHeadDim, d.nb, d.hkv);
+      if (rc != CRISP_OK) return rc;
+    }
+    const size_t smem = sizeof(LogitsSmem) + 1024;
+    CRISP_CUDA_TRY(cudaFuncSetAttribute(pe_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(smem)),
+                   "select: smem attribute");
+    const int nt = (d.nb + kBlock - 1) / kBlock;
+    pe_logits_kernel<<<dim3(nt, nt, d.hq), 160, smem, stream>>>(maps, d, pattern, w, status);
+  }
   pe_normalise_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w);
   const int hist_ctas = d.nb < 128 ? d.nb : 128;
   for (int level = 0; level < 3; ++level) {
@@ -839,7 +925,7 @@ int launch_route_jsd(const Dims& d, const void* q, const void* k, const float* p
   SelectPtrs w = carve(d, ws, &total);
   CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "route_jsd: clear status");
   pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, static_cast<const __nv_bfloat16*>(k), d.hkv, 0, nullptr,
-                                                     w.kbar);
+                                                     w.kbar, nullptr);
   jsd_kernel<<<d.hq, 256, sizeof(float) * d.nb, stream>>>(d, static_cast<const __nv_bfloat16*>(q), w.kbar, p_v,
                                                          tau_jsd, jsd, pattern);
   CRISP_CUDA_TRY(cudaGetLastError(), "route_jsd: launch");
