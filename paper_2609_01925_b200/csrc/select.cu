@@ -413,36 +413,47 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   const float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
   for (int m = blockIdx.x; m < d.nb; m += gridDim.x) {
     const float* row = am + static_cast<size_t>(m) * d.nb;
-    for (int J0 = 0; J0 <= m; J0 += 256) {
-      const int J = J0 + tid;
-      int bin = -1;
-      unsigned long long fixed = 0ull;
-      if (J <= m) {
-        const float v = row[J];
-        int b;
-        if (key_in_level(__float_as_uint(v), prefix, level, &b)) {
-          bin = b;
-          fixed = __float2ull_rn(v * kMassScale);
-        }
+    // 1024 entries per pass: the four loads of a thread are issued before any of them is binned
+    for (int J0 = 0; J0 <= m; J0 += 1024) {
+      float vals[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int J = J0 + 256 * u + tid;
+        vals[u] = J <= m ? row[J] : 0.f;
       }
-      // Level 0: neighbouring entries of a flat map fall into a handful of bins: lanes with the same bin elect a
-      // leader and add their counts and masses (three 20-bit limbs, summed exactly) in one atomic each.
-      if (level > 0) {
-        // lower levels: the 11 / 9 bits below the fixed prefix spread the entries over many bins
-        if (bin >= 0) {
-          atomicAdd(&cnt[bin], 1u);
-          atomicAdd(&mass[bin], fixed);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int J = J0 + 256 * u + tid;
+        if (J0 + 256 * u > m) break;  // uniform: the whole chunk lies beyond the row
+        int bin = -1;
+        unsigned long long fixed = 0ull;
+        if (J <= m) {
+          const float v = vals[u];
+          int b;
+          if (key_in_level(__float_as_uint(v), prefix, level, &b)) {
+            bin = b;
+            fixed = __float2ull_rn(v * kMassScale);
+          }
         }
-        continue;
-      }
-      const unsigned int peers = __match_any_sync(0xffffffffu, bin);
-      const unsigned int l0 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed & 0xFFFFFull));
-      const unsigned int l1 = __reduce_add_sync(peers, static_cast<unsigned int>((fixed >> 20) & 0xFFFFFull));
-      const unsigned int l2 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed >> 40));
-      if (bin >= 0 && (tid & 31) == __ffs(peers) - 1) {
-        atomicAdd(&cnt[bin], static_cast<unsigned int>(__popc(peers)));
-        atomicAdd(&mass[bin], static_cast<unsigned long long>(l0) + (static_cast<unsigned long long>(l1) << 20) +
-                                  (static_cast<unsigned long long>(l2) << 40));
+        // Level 0: neighbouring entries of a flat map fall into a handful of bins: lanes with the same bin elect a
+        // leader and add their counts and masses (three 20-bit limbs, summed exactly) in one atomic each.
+        if (level > 0) {
+          // lower levels: the 11 / 9 bits below the fixed prefix spread the entries over many bins
+          if (bin >= 0) {
+            atomicAdd(&cnt[bin], 1u);
+            atomicAdd(&mass[bin], fixed);
+          }
+          continue;
+        }
+        const unsigned int peers = __match_any_sync(0xffffffffu, bin);
+        const unsigned int l0 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed & 0xFFFFFull));
+        const unsigned int l1 = __reduce_add_sync(peers, static_cast<unsigned int>((fixed >> 20) & 0xFFFFFull));
+        const unsigned int l2 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed >> 40));
+        if (bin >= 0 && (tid & 31) == __ffs(peers) - 1) {
+          atomicAdd(&cnt[bin], static_cast<unsigned int>(__popc(peers)));
+          atomicAdd(&mass[bin], static_cast<unsigned long long>(l0) + (static_cast<unsigned long long>(l1) << 20) +
+                                    (static_cast<unsigned long long>(l2) << 40));
+        }
       }
     }
   }
