@@ -704,42 +704,49 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   __syncwarp();
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int64_t s0 = rp[m0], e0 = rp[m0 + 1];
-  for (int64_t i = s0 + lane; i < e0; i += 32) {
-    const int c = col_idx[i];
-    atomicOr(&b0[c >> 5], 1u << (c & 31));
-  }
+  // four loads per lane in flight before the bitmap updates
+  auto mark = [&](uint32_t* bits, int64_t from, int64_t to) {
+    for (int64_t i0 = from; i0 < to; i0 += 128) {
+      int c[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int64_t i = i0 + 32 * u + lane;
+        c[u] = i < to ? col_idx[i] : -1;
+      }
+      // the lists are sorted, so the 32 entries of a load fall into one or two words: lanes with the same word
+      // combine their bits and one of them updates the bitmap
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int wd = c[u] >= 0 ? (c[u] >> 5) : -1;
+        const unsigned int peers = __match_any_sync(0xffffffffu, wd);
+        const uint32_t mine = c[u] >= 0 ? (1u << (c[u] & 31)) : 0u;
+        const uint32_t all = __reduce_or_sync(peers, mine);
+        if (wd >= 0 && lane == __ffs(peers) - 1) atomicOr(&bits[wd], all);
+      }
+    }
+  };
+  mark(b0, s0, e0);
   int64_t e1 = e0;
   if (m1 < d.nb) {
     e1 = rp[m1 + 1];
-    for (int64_t i = e0 + lane; i < e1; i += 32) {
-      const int c = col_idx[i];
-      atomicOr(&b1[c >> 5], 1u << (c & 31));
-    }
+    mark(b1, e0, e1);
   }
   __syncwarp();
   int32_t* out = merged + s0;
   int written = 0;
-  for (int w0 = 0; w0 < words; w0 += 32) {
-    const int wd = w0 + lane;
-    const uint32_t x0 = wd < words ? b0[wd] : 0u, x1 = wd < words ? b1[wd] : 0u;
-    uint32_t un = x0 | x1;
-    const int c = __popc(un);
-    int incl = c;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int tmp = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += tmp;
+  // one 32-block word per step, lane b owning bit b: the entries of a word go out as one contiguous store
+  const int last_word = min(words - 1, (m1 < d.nb ? m1 : m0) >> 5);
+  for (int wd = 0; wd <= last_word; ++wd) {
+    const uint32_t x0 = b0[wd], x1 = b1[wd];  // broadcast reads
+    const uint32_t un = x0 | x1;
+    if (un == 0u) continue;
+    if ((un >> lane) & 1u) {
+      uint32_t ent = static_cast<uint32_t>(wd * 32 + lane);
+      if ((x0 >> lane) & 1u) ent |= kFlag0;
+      if ((x1 >> lane) & 1u) ent |= kFlag1;
+      out[written + __popc(un & ((1u << lane) - 1u))] = static_cast<int32_t>(ent);
     }
-    int pos = written + incl - c;
-    while (un) {
-      const int b = __ffs(un) - 1;
-      un &= un - 1;
-      uint32_t ent = static_cast<uint32_t>(wd * 32 + b);
-      if ((x0 >> b) & 1u) ent |= kFlag0;
-      if ((x1 >> b) & 1u) ent |= kFlag1;
-      out[pos++] = static_cast<int32_t>(ent);
-    }
-    written += __shfl_sync(0xffffffffu, incl, 31);
+    written += __popc(un);
   }
   if (lane == 0) {
     item_len[h * n_pairs + u] = written;

@@ -717,11 +717,13 @@ fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs 
         const int t = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += t;
       }
-      int pos = written + incl - c;
-      while (bits) {
-        const int b = __ffs(bits) - 1;
-        bits &= bits - 1;
-        out[pos++] = wd * 32 + b;
+      // emit word by word, lane b owning bit b: the entries of a word go out as one contiguous store
+      const int nw = min(32, nwords - w0);
+      for (int k = 0; k < nw; ++k) {
+        const uint32_t wbits = __shfl_sync(0xffffffffu, bits, k);
+        if (wbits == 0u) continue;
+        const int base = written + __shfl_sync(0xffffffffu, incl - c, k);
+        if ((wbits >> lane) & 1u) out[base + __popc(wbits & ((1u << lane) - 1u))] = (w0 + k) * 32 + lane;
       }
       written += __shfl_sync(0xffffffffu, incl, 31);
     }
