@@ -53,6 +53,7 @@ struct PrefillArgs {
   int n_items;
   int group_kv;            // 1: schedule one KV head at a time (K/V larger than L2), 0: one global order
   const int* gate;         // optional device word: when non-zero the lists are invalid and nothing is done
+  int* next_item;          // device counter (zero at launch): position of the next item nobody has taken yet
 };
 
 struct PrefillSmem {
@@ -62,6 +63,10 @@ struct PrefillSmem {
   uint64_t kv_full[kStages], kv_empty[kStages];
   // per tile and per 64-key half (A = keys 0-63, B = keys 64-127 of the block)
   uint64_t s_full[2][2], p_ready[2][2], o_done[2][2];
+  // items are handed out dynamically: the producer takes the next position from a device counter and passes
+  // it to the other roles through a four-slot queue
+  uint64_t itm_full[4], itm_empty[4];
+  int item_q[4];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -293,13 +298,8 @@ struct EntryStream {
   }
 };
 
-// Position (in the cost-sorted order) of the item a CTA takes in round `rnd`.  Odd rounds run backwards:
-// with costs falling along the order, CTA 0 would otherwise get the most expensive item of every round.
-__device__ __forceinline__ int item_pos(int rnd) {
-  const int c = (rnd & 1) ? static_cast<int>(gridDim.x) - 1 - static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x);
-  return rnd * static_cast<int>(gridDim.x) + c;
-}
-
+// Items are taken in cost-sorted order by whichever CTA is free next (a device counter), so CTAs that run
+// slower - the per-step time differs by a few per cent between SMs - simply take fewer of them.
 template <bool kDense>
 __global__ void __launch_bounds__(384, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
@@ -315,6 +315,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     for (int i = 0; i < kStages; ++i) {
       mbar_init(&s.kv_full[i], 1);
       mbar_init(&s.kv_empty[i], 2);  // one arrival per issuer, whether or not its tile uses the block
+    }
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(&s.itm_full[i], 1);
+      mbar_init(&s.itm_empty[i], 10);  // two issuers and eight softmax warps
     }
     for (int i = 0; i < 2; ++i)
       for (int h = 0; h < 2; ++h) {
@@ -349,10 +353,15 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     if (lane == 0) {
       uint32_t ecount = 0;
       bool ok = true;
-      for (int rnd = 0; rnd * static_cast<int>(gridDim.x) < n_items && ok; ++rnd) {
-        const int idx = item_pos(rnd);
-        if (idx >= n_items) break;  // only in the last, partial round
-        const int it_count = rnd;
+      for (int it_count = 0; ok; ++it_count) {
+        const int qslot = it_count & 3;
+        if (it_count >= 4) ok = mbar_wait(&s.itm_empty[qslot], ((it_count >> 2) - 1) & 1, abort_flag);
+        if (!ok) break;
+        int idx = n_items > 0 ? atomicAdd(a.next_item, 1) : -1;
+        if (idx >= n_items) idx = -1;  // no more work: the others leave when they read this
+        s.item_q[qslot] = idx;
+        mbar_arrive(&s.itm_full[qslot]);
+        if (idx < 0) break;
         const Item it = decode_item<kDense>(idx, d, a);
         EntryStream<kDense> rd;
         rd.init(it, a);
@@ -460,10 +469,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         if (h == 1) umma_commit(&s.kv_empty[slot]);
       };
 
-      for (int rnd = 0; rnd * static_cast<int>(gridDim.x) < n_items && ok; ++rnd) {
-        const int idx = item_pos(rnd);
-        if (idx >= n_items) break;  // only in the last, partial round
-        const int it_count = rnd;
+      for (int it_count = 0; ok; ++it_count) {
+        const int qslot = it_count & 3;
+        ok = mbar_wait(&s.itm_full[qslot], (it_count >> 2) & 1, abort_flag);
+        if (!ok) break;
+        const int idx = *reinterpret_cast<volatile int*>(&s.item_q[qslot]);
+        mbar_arrive(&s.itm_empty[qslot]);
+        if (idx < 0) break;
         const Item it = decode_item<kDense>(idx, d, a);
         ok = mbar_wait(&s.q_full, it_count & 1, abort_flag);
         if (!ok) break;
@@ -570,9 +582,14 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         tmem_st_x32(o_addr + c * 32, ov);
       }
     };
-    for (int rnd = 0; rnd * static_cast<int>(gridDim.x) < n_items && ok; ++rnd) {
-      const int idx = item_pos(rnd);
-      if (idx >= n_items) break;  // only in the last, partial round
+    for (int it_count = 0; ok; ++it_count) {
+      const int qslot = it_count & 3;
+      ok = mbar_wait_warp(&s.itm_full[qslot], (it_count >> 2) & 1, abort_flag);
+      if (!ok) break;
+      const int idx = *reinterpret_cast<volatile int*>(&s.item_q[qslot]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s.itm_empty[qslot]);
+      if (idx < 0) break;
       const Item it = decode_item<kDense>(idx, d, a);
       if (t == 1 && !it.tile1) continue;
       EntryReader<kDense> rd;
@@ -845,6 +862,7 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   a.lse = lse;
   a.status = static_cast<int*>(ws);
   a.gate = gate;
+  a.next_item = static_cast<int*>(ws) + 16;  // inside the header that the memset above has just cleared
   // K + V of all KV heads against the 126 MB L2: group the schedule by KV head only when they do not fit
   a.group_kv = (static_cast<size_t>(d.n) * d.hkv * kHeadDim * 2 * 2 > (256u << 20)) ? 1 : 0;
 
