@@ -863,8 +863,8 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   a.status = static_cast<int*>(ws);
   a.gate = gate;
   a.next_item = static_cast<int*>(ws) + 16;  // inside the header that the memset above has just cleared
-  // K + V of all KV heads against the 126 MB L2: group the schedule by KV head only when they do not fit
-  a.group_kv = (static_cast<size_t>(d.n) * d.hkv * kHeadDim * 2 * 2 > (256u << 20)) ? 1 : 0;
+  // the schedule walks one KV head at a time, so the CTAs running at one moment stream the same K/V blocks
+  a.group_kv = 1;
 
   int dev = 0, n_sm = 0;
   CRISP_CUDA_TRY(cudaGetDevice(&dev), "prefill: device");
