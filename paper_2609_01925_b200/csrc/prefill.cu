@@ -863,13 +863,16 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   a.status = static_cast<int*>(ws);
   a.gate = gate;
   a.next_item = static_cast<int*>(ws) + 16;  // inside the header that the memset above has just cleared
-  // the schedule walks one KV head at a time, so the CTAs running at one moment stream the same K/V blocks
-  a.group_kv = 1;
+  // The schedule walks one KV head at a time, so the CTAs running at one moment stream the same K/V blocks.
+  // Problems of only a few items per SM are ordered by cost alone instead: their K/V fit L2 anyway, and
+  // the longest items of every head should start first.
+  a.group_kv = 0;  // set below, once the SM count is known
 
   int dev = 0, n_sm = 0;
   CRISP_CUDA_TRY(cudaGetDevice(&dev), "prefill: device");
   CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "prefill: SM count");
   const int grid = a.n_items < n_sm ? a.n_items : n_sm;
+  a.group_kv = a.n_items >= 16 * n_sm ? 1 : 0;
   const size_t smem = sizeof(PrefillSmem) + 1024;
   if (dense) {
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
