@@ -23,6 +23,9 @@
 // grows by more than 2^8, and does it in place in TMEM.
 // Both issuers see every load of the K/V ring in order and release every slot once, so the ring never runs
 // ahead of either tile; apart from that the two tiles run free of each other.
+// Work items are handed out dynamically: the producer takes the next position of the cost-sorted order from
+// a device counter and passes it to the other roles through a four-slot queue, which balances the load and
+// keeps the CTAs that run at the same time on the same K/V blocks (they share them through L2).
 // Measured alternatives that were slower and are not kept: a single issuing thread for both tiles (its scalar
 // bookkeeping between bursts, several hundred cycles, is idle pipe time); whole-block steps with one issuer
 // per tile, with and without handing P over in two halves; computing part of the exponentials on the FMA
