@@ -54,7 +54,7 @@ struct PrefillArgs {
   int* status;
   int n_pairs;
   int n_items;
-  int group_kv;            // 1: schedule one KV head at a time (K/V larger than L2), 0: one global order
+  int group_kv;            // 1: schedule one KV head at a time, 0: one global order by cost (small problems)
   const int* gate;         // optional device word: when non-zero the lists are invalid and nothing is done
   int* next_item;          // device counter (zero at launch): position of the next item nobody has taken yet
 };
@@ -777,7 +777,7 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
 
 // Counting sort of the items by (KV head, decreasing cost).  Grouping by KV head keeps the CTAs that
 // run at the same time on the same K/V blocks (L2 reuse); sorting by cost inside a group lets the
-// round-robin assignment balance heads with long lists (PE) against heads with short ones (VS).
+// dynamic hand-out start the long lists (PE heads) before the short ones (VS heads).
 __global__ void __launch_bounds__(1024) sched_scan_kernel(int* __restrict__ cost_hist, int n_bins) {
   __shared__ long long scratch[33];
   const int tid = threadIdx.x;
