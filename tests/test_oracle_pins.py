@@ -370,7 +370,59 @@ def test_pooled_map_zero_inputs_closed_form():
     picked_rows = [m for m in range(nb) if sel[m, :m + 1].all()]
     assert picked_rows[:3] == [0, 1, 2]
     assert sel.sum() in (6, 7)                               # 1+2+3 (+1 if 0.5 missed by an ulp)
+    if sel.sum() == 7:
+        assert sel[3, 0] and not sel[3, 1:].any()             # the extra entry is the first of row 3
     assert not sel[4:].any()
+
+
+def test_select_pe_tie_order_is_lower_flat_index_first():
+    """Algorithm 4 on a map whose entries are powers of two, so every running sum is exact.
+
+    Normalised entries: (0,0) = 1/4; (1,0), (1,1), (2,0) = 1/8; the other six = 1/16.  Descending order with
+    ties to the lower flat index m * N_b + J: (0,0) | (1,0) (1,1) (2,0) | (2,1) (2,2) (3,0) (3,1) (3,2) (3,3),
+    running sums 1/4, 3/8, 1/2, 5/8, 11/16, 3/4, ...  gamma = 1/2 ends INSIDE the run of 1/8s after two of
+    its three members; gamma = 0.7 ends inside the run of 1/16s after two of its six.
+    """
+    a = np.zeros((4, 4))
+    a[0, :1] = [1.0]
+    a[1, :2] = [0.5, 0.5]
+    a[2, :3] = [0.5, 0.25, 0.25]
+    a[3, :4] = [0.25, 0.25, 0.25, 0.25]
+    sel, cut = orc.select_pe(a, 0.5)
+    assert sorted(map(tuple, np.argwhere(sel).tolist())) == [(0, 0), (1, 0), (1, 1)]   # (2,0) ties but comes later
+    assert cut == 0.125
+    sel, cut = orc.select_pe(a, 0.7)
+    assert sorted(map(tuple, np.argwhere(sel).tolist())) == [(0, 0), (1, 0), (1, 1), (2, 0), (2, 1), (2, 2)]
+    assert cut == 0.0625
+    # one entry more of the same tie run as soon as gamma passes the running sum
+    sel, _ = orc.select_pe(a, 0.76)
+    assert sel[3, 0] and not sel[3, 1:].any() and sel.sum() == 7
+    # the expansion adds the forced blocks {0, m} to rows the cut left empty
+    cols = orc.expand_pe(orc.select_pe(a, 0.5)[0])
+    assert [c.tolist() for c in cols] == [[0], [0, 1], [0, 2], [0, 3]]
+
+
+def test_head_pipeline_two_blocks_keeps_every_causal_block():
+    """N_b = 2: mu_d = r_d / (N_b - 2) is undefined, and both blocks are the always-retained first and last
+    block of Algorithm 3 line 12, so every causal block is kept whatever the pattern or selector."""
+    r_ = rng(31)
+    n, d = 2 * B, 16
+    q, k, v = r_.normal(size=(n, d)), r_.normal(size=(n, d)), r_.normal(size=(n, d))
+    for force in (0, 1, 2):
+        for selector in (0, 1, 2):
+            res = orc.head_pipeline(q, k, block=B, sink_tokens=4, local_tokens=B, force_pattern=force,
+                                    selector=selector, k_min_blocks=0, alpha=50.0, gamma=1e-6)
+            assert [c.tolist() for c in res["cols"]] == [[0], [0, 1]]
+            assert abs(res["p_v"].sum() - 1) < 1e-12 and abs(res["p_s"].sum() - 1) < 1e-12
+            # slash offset 0 = the diagonal band of the last block, offset 1 = everything older
+            a = orc.proxy_attention(q, k, B)
+            band0 = sum(a[i, B + i - o] for i in range(B) for o in range(B) if B + i - o >= 0 and o <= B + i) / B
+            assert abs(res["p_s"][0] - band0) < 1e-12
+    # Eq. 1 over those lists is dense causal attention
+    o, _ = orc.sparse_attention_head(q, k, v, res["cols"], B)
+    want = torch.nn.functional.scaled_dot_product_attention(
+        torch.tensor(q)[None, None], torch.tensor(k)[None, None], torch.tensor(v)[None, None], is_causal=True)[0, 0]
+    assert np.abs(o - want.numpy()).max() < 1e-12
 
 
 def test_pooled_map_bruteforce():
