@@ -19,8 +19,9 @@
  *   - `cuda_stream` is a cudaStream_t (NULL = legacy default stream).  Calls only enqueue work on that
  *     stream and return; they never synchronise, except crisp_poll_device_status.
  *   - The return value is a crisp_status.  Host-side argument errors are reported immediately and
- *     nothing is launched.  Device-side conditions (capacity overflow, a bounded wait that gave up) are
- *     recorded in the first word of the workspace and read back with crisp_poll_device_status.
+ *     nothing is launched.  Device-side conditions (capacity overflow, a bounded wait that gave up, index
+ *     lists that break their rules) are recorded in the first word of the workspace and read back with
+ *     crisp_poll_device_status.
  *   - Nothing throws, exits, traps or spins without a bound.
  *   - The library needs a CUDA device of compute capability 10.0; there is no CPU fallback.
  */
@@ -41,7 +42,8 @@ typedef enum crisp_status {
   CRISP_ERR_WORKSPACE = -3,      /* workspace too small or misaligned                                */
   CRISP_ERR_CAPACITY = -4,       /* col_idx capacity too small for the selected blocks               */
   CRISP_ERR_CUDA = -5,           /* a CUDA runtime / driver call failed (see crisp_last_cuda_error)  */
-  CRISP_ERR_DEVICE_TIMEOUT = -6  /* a bounded device-side wait gave up                               */
+  CRISP_ERR_DEVICE_TIMEOUT = -6, /* a bounded device-side wait gave up                               */
+  CRISP_ERR_BAD_LIST = -7        /* row_ptr / col_idx given to crisp_sparse_prefill break the list rules */
 } crisp_status;
 
 /* Pattern labels written by crisp_route (Algorithm 2). */
@@ -114,11 +116,13 @@ int crisp_route(const crisp_params* p, const void* q, const void* k, void* ws, s
  *
  * Limits and rules
  *   - The problem must fit: crisp_workspace_bytes(p).route_ws <= CRISP_ROUTE_STATIC_SCRATCH_BYTES
- *     (4 MiB: for example 8192 tokens with 32 query heads, or 65536 tokens with 4).  Anything larger is
- *     refused with CRISP_ERR_UNSUPPORTED before any work is enqueued, and crisp_last_cuda_error() says
- *     how many bytes would have been needed.
+ *     (4 MiB: for example 8192 tokens with 32 query heads, or 65536 tokens with 4, when seq_len is a
+ *     multiple of `block`; other lengths need about 4/3 of that scratch, so 8191 tokens with 32 heads do not
+ *     fit).  Anything larger is refused with CRISP_ERR_UNSUPPORTED before any work is enqueued, and
+ *     crisp_last_cuda_error() says how many bytes would have been needed.
  *   - The first call on each device looks up the array's device address (with that device current) and
- *     remembers it.  Make that first call during set-up, outside any stream capture.
+ *     remembers it for as long as the device's primary context lives (after cudaDeviceReset the remembered
+ *     address is stale).  Make that first call during set-up, outside any stream capture.
  *   - All calls on one device share the one array.  Nothing of a previous call is ever read back (the
  *     status word is cleared, everything else is rewritten before use), but two calls that overlap in time
  *     on the same GPU - different streams, different threads - overwrite each other's scratch and give
@@ -155,8 +159,12 @@ int crisp_select(const crisp_params* p, const void* q, const void* k, const int3
  * Stage 4 (Eq. 1).  O[t, h, :] = sum_j softmax_j(Q[t,h] . K[j,kv(h)] * scale) V[j,kv(h)] over the keys j <= t
  * of the key blocks listed for query block t / block.  Exact softmax over the kept keys; bf16 inputs,
  * fp32 accumulation, bf16 output.  lse (optional, [H_q, seq_len] f32) receives the natural-log
- * sum-exp of the kept scaled logits.  row_ptr / col_idx as produced by crisp_select (every row must
- * contain its diagonal block).
+ * sum-exp of the kept scaled logits.  row_ptr / col_idx as produced by crisp_select, or built by the caller
+ * to the same rules: row_ptr [H_q, N_b + 1] holds non-negative offsets into col_idx, at most
+ * H_q N_b (N_b + 1) / 2, and col_idx holds at least row_ptr[H_q - 1][N_b] entries; the row of query block m
+ * has between 1 and m + 1 entries, strictly ascending, all in [0, m], the last one m (the diagonal block).
+ * The lists are checked on the device before they are used: if any row breaks a rule, nothing is computed,
+ * O is left untouched and the status word of `ws` becomes CRISP_ERR_BAD_LIST.
  */
 int crisp_sparse_prefill(const crisp_params* p, const void* q, const void* k, const void* v,
                          const int64_t* row_ptr, const int32_t* col_idx, void* ws, size_t ws_bytes, void* o,
@@ -184,8 +192,8 @@ int crisp_route_jsd(const crisp_params* p, const void* q, const void* k, const f
 
 /*
  * Algorithm 1 in one call, with the context-length gate the paper recommends for deployments that serve
- * short prompts (Section 5.3, "Short contexts": routing is a fixed per-head cost that dominates what it
- * saves below some length).
+ * short prompts (Section 5.3, "Short contexts"): below dense_below_tokens the route and select launches take
+ * longer than the skipped blocks would have.
  *   seq_len <  dense_below_tokens : crisp_dense_prefill only; the routing / selection outputs are not
  *                                   written and their pointers (and route_ws, select_ws) may be NULL.
  *   seq_len >= dense_below_tokens : crisp_route, crisp_select, crisp_sparse_prefill, enqueued back to back
@@ -234,8 +242,20 @@ int crisp_forward_varlen(const crisp_params* p, const int64_t* cu_seqlens, int32
                          int32_t* device_status, void* o, float* lse, int32_t dense_below_tokens, void* cuda_stream);
 
 /*
+ * Diagnostic (the paper has no counterpart): exercises the library's failure-reporting path without any
+ * failure.  Enqueues one tiny kernel that waits on a barrier nothing arrives at, with a wait limit of
+ * `limit_ns` nanoseconds (1 .. 10,000,000); the wait runs out, a second role waiting with the normal limit is
+ * released through the shared abort flag, the kernel records CRISP_ERR_DEVICE_TIMEOUT in the status word of
+ * `ws` and returns by itself.  crisp_poll_device_status(ws) then reports that code, and the context stays
+ * usable.  ws: device pointer, 16-byte aligned, at least 256 bytes; bytes 64..79 receive the two roles'
+ * waiting times in nanoseconds (uint64 each).  limit_ns out of range: CRISP_ERR_INVALID_ARG, nothing launched.
+ */
+int crisp_selftest_bounded_wait(void* ws, size_t ws_bytes, int64_t limit_ns, void* cuda_stream);
+
+/*
  * Synchronises `cuda_stream`, reads the status word at the start of `ws`, clears it and returns it
- * (CRISP_OK, CRISP_ERR_CAPACITY or CRISP_ERR_DEVICE_TIMEOUT), or CRISP_ERR_CUDA if the stream failed.
+ * (CRISP_OK, CRISP_ERR_CAPACITY, CRISP_ERR_DEVICE_TIMEOUT or CRISP_ERR_BAD_LIST), or CRISP_ERR_CUDA if the
+ * stream failed.
  */
 int crisp_poll_device_status(void* ws, void* cuda_stream);
 

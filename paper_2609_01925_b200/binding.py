@@ -22,13 +22,14 @@ ERR_WORKSPACE = -3
 ERR_CAPACITY = -4
 ERR_CUDA = -5
 ERR_DEVICE_TIMEOUT = -6
+ERR_BAD_LIST = -7
 PATTERN_PE, PATTERN_VS = 0, 1
 
 EXPORTS = (
     "crisp_version", "crisp_status_string", "crisp_last_cuda_error", "crisp_workspace_bytes",
     "crisp_route", "crisp_route_static", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
     "crisp_poll_device_status", "crisp_forward", "crisp_route_jsd", "crisp_varlen_layout",
-    "crisp_forward_varlen",
+    "crisp_forward_varlen", "crisp_selftest_bounded_wait",
 )
 
 
@@ -104,6 +105,8 @@ def load() -> ctypes.CDLL:
     lib.crisp_forward_varlen.restype = ctypes.c_int
     lib.crisp_forward_varlen.argtypes = [P, vp, ctypes.c_int32, vp, vp, vp, vp, sz, vp, sz, vp, sz, vp, vp, vp, vp,
                                          vp, vp, i64, vp, vp, vp, vp, ctypes.c_int32, vp]
+    lib.crisp_selftest_bounded_wait.restype = ctypes.c_int
+    lib.crisp_selftest_bounded_wait.argtypes = [vp, sz, i64, vp]
     lib.crisp_poll_device_status.restype = ctypes.c_int
     lib.crisp_poll_device_status.argtypes = [vp, vp]
     _lib = lib
@@ -221,6 +224,10 @@ def crisp_forward_varlen(p, cu_seqlens, q, k, v, route_ws, select_ws, prefill_ws
                                        _ptr(row_ptr), _ptr(col_idx), int(capacity), _ptr(nnz_needed),
                                        _ptr(device_status), _ptr(o), _ptr(lse), int(dense_below_tokens),
                                        _stream(stream))
+
+
+def crisp_selftest_bounded_wait(ws, limit_ns, stream=None) -> int:
+    return load().crisp_selftest_bounded_wait(_ptr(ws), _nbytes(ws), int(limit_ns), _stream(stream))
 
 
 def crisp_poll_device_status(ws, stream=None) -> int:

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcrisp.so")
-SOURCES = ["api.cu", "route.cu", "select.cu", "prefill.cu"]
+SOURCES = ["api.cu", "route.cu", "select.cu", "prefill.cu", "selftest.cu"]
 HEADERS = ["common.cuh", "sm100_ptx.cuh", os.path.join("..", "..", "include", "crisp.h")]
 
 

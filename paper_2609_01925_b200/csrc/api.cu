@@ -127,6 +127,7 @@ const char* crisp_status_string(int status) {
     case CRISP_ERR_CAPACITY: return "col_idx capacity too small";
     case CRISP_ERR_CUDA: return "CUDA error";
     case CRISP_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case CRISP_ERR_BAD_LIST: return "index lists break the list rules";
     default: return "unknown status";
   }
 }
@@ -370,6 +371,12 @@ int crisp_forward_varlen(const crisp_params* p, const int64_t* cu_seqlens, int32
                      "forward_varlen: attention status");
   }
   return CRISP_OK;
+}
+
+int crisp_selftest_bounded_wait(void* ws, size_t ws_bytes, int64_t limit_ns, void* cuda_stream) {
+  if (!ws) return CRISP_ERR_INVALID_ARG;
+  if (!aligned16(ws) || ws_bytes < kWsHeader) return CRISP_ERR_WORKSPACE;
+  return launch_selftest_bounded_wait(ws, limit_ns, static_cast<cudaStream_t>(cuda_stream));
 }
 
 int crisp_poll_device_status(void* ws, void* cuda_stream) {

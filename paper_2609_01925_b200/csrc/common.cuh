@@ -98,5 +98,6 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
                    const int32_t* col_idx, void* ws, void* o, float* lse, cudaStream_t stream,
                    const int* gate = nullptr);
 size_t prefill_ws_bytes(const Dims& d);
+int launch_selftest_bounded_wait(void* ws, long long limit_ns, cudaStream_t stream);
 
 }  // namespace crisp

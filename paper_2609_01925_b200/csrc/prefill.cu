@@ -340,7 +340,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   tc_fence_after_sync();
   const uint32_t tm = s.tmem_base;
   volatile int* abort_flag = &s.abort_flag;
-  const int n_items = (a.gate != nullptr && *a.gate != 0) ? 0 : a.n_items;
+  // nothing is done when the selection stage reported an error (gate) or the lists failed validation (status)
+  const int n_items = ((a.gate != nullptr && *a.gate != 0) || (!kDense && *a.status != 0)) ? 0 : a.n_items;
 
   // Register budget: the two softmax warpgroups hold a full 128-column row of S per thread; the third
   // warpgroup (producer, issuer, two idle warps) needs very few registers and gives the rest away.
@@ -710,7 +711,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 __global__ void __launch_bounds__(128)
 merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                    int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
-                   int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate) {
+                   int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate, int* __restrict__ status,
+                   long long merged_capacity) {
   extern __shared__ uint32_t bm[];
   if (gate != nullptr && *gate != 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -724,8 +726,18 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   __syncwarp();
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int64_t s0 = rp[m0], e0 = rp[m0 + 1];
+  const bool has1 = m1 < d.nb;
+  const int64_t e1 = has1 ? rp[m1 + 1] : e0;
+  // The lists may come from the caller, so nothing about them is trusted: a row of query block m must hold
+  // between 1 and m + 1 entries inside the workspace's range, strictly ascending, none above m, the last
+  // one m itself (the diagonal block, which the attention kernel's Q hand-over relies on).  Anything else
+  // marks the launch CRISP_ERR_BAD_LIST; nothing derived from a bad row is written and the attention
+  // kernel, which reads the status word, does no work at all.
+  bool bad = s0 < 0 || e0 - s0 < 1 || e0 - s0 > m0 + 1 || e1 > merged_capacity ||
+             (has1 && (e1 - e0 < 1 || e1 - e0 > m1 + 1));
   // four loads per lane in flight before the bitmap updates
-  auto mark = [&](uint32_t* bits, int64_t from, int64_t to) {
+  auto mark = [&](uint32_t* bits, int64_t from, int64_t to, int m) {
+    int prev_last = -1;  // last entry of the previous group of 32
     for (int64_t i0 = from; i0 < to; i0 += 128) {
       int c[4];
 #pragma unroll
@@ -737,19 +749,28 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
       // combine their bits and one of them updates the bitmap
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
-        const int wd = c[u] >= 0 ? (c[u] >> 5) : -1;
+        const int64_t i = i0 + 32 * u + lane;
+        const bool live = i < to;
+        int before = __shfl_up_sync(0xffffffffu, c[u], 1);
+        if (lane == 0) before = prev_last;
+        const bool okc = !live || (c[u] >= 0 && c[u] <= m && c[u] > before && (i + 1 < to || c[u] == m));
+        bad = bad || !okc;
+        prev_last = __shfl_sync(0xffffffffu, c[u], 31);
+        const int wd = (live && okc) ? (c[u] >> 5) : -1;
         const unsigned int peers = __match_any_sync(0xffffffffu, wd);
-        const uint32_t mine = c[u] >= 0 ? (1u << (c[u] & 31)) : 0u;
+        const uint32_t mine = wd >= 0 ? (1u << (c[u] & 31)) : 0u;
         const uint32_t all = __reduce_or_sync(peers, mine);
         if (wd >= 0 && lane == __ffs(peers) - 1) atomicOr(&bits[wd], all);
       }
     }
   };
-  mark(b0, s0, e0);
-  int64_t e1 = e0;
-  if (m1 < d.nb) {
-    e1 = rp[m1 + 1];
-    mark(b1, e0, e1);
+  if (!bad) {
+    mark(b0, s0, e0, m0);
+    if (has1) mark(b1, e0, e1, m1);
+  }
+  if (__any_sync(0xffffffffu, bad)) {
+    if (lane == 0) atomicExch(status, CRISP_ERR_BAD_LIST);
+    return;
   }
   __syncwarp();
   int32_t* out = merged + s0;
@@ -796,9 +817,10 @@ __global__ void __launch_bounds__(1024) sched_scan_kernel(int* __restrict__ cost
 __global__ void __launch_bounds__(256)
 sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, int* __restrict__ cost_hist,
                      int* __restrict__ order, int n_pairs, int n_cost, int group_kv,
-                     const int* __restrict__ gate) {
+                     const int* __restrict__ gate, const int* __restrict__ status) {
   const int u = blockIdx.x * blockDim.x + threadIdx.x, h = blockIdx.y;
   if (u >= n_pairs || (gate != nullptr && *gate != 0)) return;
+  if (*status != 0) return;  // a list failed validation: its row lengths cannot be trusted as histogram keys
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int m0 = 2 * u, mend = min(2 * u + 2, d.nb);
   const int cost = static_cast<int>(rp[mend] - rp[m0]);
@@ -886,10 +908,12 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
     const int words = (d.nb + 31) / 32;
     CRISP_CUDA_TRY(cudaMemsetAsync(w.cost_hist, 0, sizeof(int) * w.n_bins, stream), "prefill: clear histogram");
     merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
-        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate);
+        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate, a.status,
+        static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2);
     sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins);
     sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, 0, stream>>>(d, row_ptr, w.cost_hist,
-                                                                               w.order, a.n_pairs, w.n_cost, a.group_kv, gate);
+                                                                               w.order, a.n_pairs, w.n_cost, a.group_kv, gate,
+                                                                               a.status);
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");

@@ -26,7 +26,7 @@ def test_version_and_status_strings():
     assert crisp.crisp_version() >= 100
     assert B.status_string(B.OK) == "ok"
     for code in (B.ERR_INVALID_ARG, B.ERR_UNSUPPORTED, B.ERR_WORKSPACE, B.ERR_CAPACITY, B.ERR_CUDA,
-                 B.ERR_DEVICE_TIMEOUT):
+                 B.ERR_DEVICE_TIMEOUT, B.ERR_BAD_LIST):
         assert B.status_string(code) not in ("ok", "unknown status")
     assert B.status_string(12345) == "unknown status"
 

@@ -38,7 +38,9 @@ def test_static_route_matches_route_on_two_calls_in_a_row():
     dev = torch.device("cuda")
     cases = [synth.tiny(n=2048),
              synth.llama_shaped("L8k", 8192, 32).with_(n_q_heads=8, n_kv_heads=2,
-                                                       head_classes=("conc", "diffuse") * 4)]
+                                                       head_classes=("conc", "diffuse") * 4),
+             synth.tiny(n=2048 + 37),                      # a length that is not a multiple of the block
+             synth.llama_shaped("L8k-32", 8192, 32)]       # 32 heads x 8192 tokens: just inside the 4 MiB
     for w in cases:                               # the second case reuses the array after the first
         q, k, _ = synth.make_qkv(w, device=dev)
         p = crisp.make_params(w.seq_len, w.n_q_heads, w.n_kv_heads, sink_tokens=w.sink_tokens,

@@ -284,6 +284,25 @@ def make_qkv(w: Workload, device="cpu", chunk_tokens: int = 8192):
     return q, k, v
 
 
+def make_qkv_kv_groups(w: Workload, kv_groups, device="cpu", chunk_tokens: int = 8192):
+    """The slice of make_qkv(w) that belongs to the given KV heads: K, V [n, len(kv_groups), 128] and the
+    Q of their query heads [n, G * len(kv_groups), 128] (group-major, as a head-sharded rank stores them).
+    Every element equals the corresponding element of the full tensors."""
+    dev = torch.device(device)
+    n, g = w.seq_len, w.group
+    kv_idx = torch.tensor(list(kv_groups), dtype=torch.int64, device=dev)
+    q_idx = (kv_idx[:, None] * g + torch.arange(g, dtype=torch.int64, device=dev)[None, :]).reshape(-1)
+    q = torch.empty(n, q_idx.numel(), HEAD_DIM, dtype=torch.bfloat16, device=dev)
+    k = torch.empty(n, kv_idx.numel(), HEAD_DIM, dtype=torch.bfloat16, device=dev)
+    v = torch.empty(n, kv_idx.numel(), HEAD_DIM, dtype=torch.bfloat16, device=dev)
+    for t0 in range(0, n, chunk_tokens):
+        t1 = min(n, t0 + chunk_tokens)
+        q[t0:t1] = make_q_chunk(w, t0, t1, dev)[:, q_idx]
+        k[t0:t1] = make_k_chunk(w, t0, t1, dev)[:, kv_idx]
+        v[t0:t1] = make_v_chunk(w, t0, t1, dev)[:, kv_idx]
+    return q, k, v
+
+
 def random_qkv(n: int, n_q_heads: int, n_kv_heads: int, seed: int, device="cpu",
                scale: float = 1.0):
     """Unstructured iid N(0, scale^2) inputs of an arbitrary shape (edge-case tests)."""
