@@ -24,3 +24,28 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+# Lines the parity tests want shown even under `-q` (sample sizes, excused counts, worst errors): they are
+# printed in the terminal summary and, on a GPU machine, appended to gpurun_out/parity_summary.txt.
+_PARITY_LINES = []
+
+
+@pytest.fixture
+def parity_report():
+    return _PARITY_LINES.append
+
+
+def pytest_terminal_summary(terminalreporter):
+    if not _PARITY_LINES:
+        return
+    terminalreporter.section("parity summary")
+    for line in _PARITY_LINES:
+        terminalreporter.write_line(line)
+    try:
+        out = os.path.join(ROOT, "gpurun_out")
+        os.makedirs(out, exist_ok=True)
+        with open(os.path.join(out, "parity_summary.txt"), "a") as f:
+            f.write("\n".join(_PARITY_LINES) + "\n")
+    except OSError:  # pragma: no cover
+        pass

@@ -1,6 +1,6 @@
 """Helpers shared by the GPU parity tests: run the C-ABI stages, run the oracle, compare.
 
-Matching rule (per stage):
+Matching rule (per stage; the list part lives in oracle/matching.py):
   * c_struct, p_v, p_s: floating point, rtol 2e-4 / atol 1e-7 (fp32 accumulation and the hardware
     exp2 approximation against an fp64 oracle).
   * routing labels: identical unless |C_struct - tau| <= 1e-3 * tau.
@@ -8,20 +8,38 @@ Matching rule (per stage):
     value (alpha * mu_d, or the value at the k_min / gamma cut).  With A the set of such blocks, the
     GPU list of every query block must lie between expand(S minus A) and expand(S union A).
     For the cumulative rules the entry right at the cut is also excused when the running sum passes
-    within 1e-6 of gamma (fp32 scores against fp64).  The number of such blocks is returned.
+    within 1e-6 of gamma (fp32 scores against fp64).  Both kinds of excused blocks are counted, apart,
+    and bounded: at most two mass-band entries per direction and head (the rule cannot produce more),
+    and the 1e-3 band may hold at most BAND_LIMIT of a head's candidate blocks.
   * attention output against the oracle's exact attention over the GPU's own lists:
     rel-L2 <= 1e-2 and max-abs <= 2e-2.
+
+The full-size configurations run the oracle in a pool of forked worker processes (one numpy thread each):
+most of the oracle's time at 128k tokens and above goes into single-threaded gathers and element-wise
+passes, so the host's cores are used by working on several heads / query blocks at once.  The workers
+only run numpy on host arrays they inherited; they never touch CUDA.
 """
 from __future__ import annotations
+
+import multiprocessing
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
 import torch
 
 import paper_2609_01925_b200 as crisp
 from oracle import crisp_oracle as orc
+from oracle import matching
 
-REL_BAND = 1e-3
-MASS_BAND = 1e-6
+REL_BAND = matching.REL_BAND
+MASS_BAND = matching.MASS_BAND
+# Largest share of a head's candidate blocks (2 N_b for a VS head, the causal entries for a PE head) that may
+# sit inside the 1e-3 band (observed on the Llama-shaped workloads: at most 0.45 %).  Heads with a flat
+# background - the sink-dominated heads of Q256k, a diffuse head forced to Vertical-Slash - have all their
+# middle blocks within ~1 % of the mean, so several per cent of them lie within 0.1 % of alpha * mu by
+# construction of the rule; tests of such inputs pass a wider limit and say why.
+BAND_LIMIT = 0.02
 
 
 def params_of(w, **over):
@@ -65,6 +83,41 @@ def oracle_kwargs(p):
                 scale=(p.softmax_scale if p.softmax_scale > 0 else None))
 
 
+def _rule_kwargs(p):
+    return dict(selector=p.selector, alpha=p.alpha, gamma=p.gamma, k_min=p.k_min_blocks)
+
+
+class Excused:
+    """Blocks excused by the matching rule, counted per head and per kind."""
+
+    def __init__(self):
+        self.per_head: Dict[int, Tuple[int, int, int]] = {}   # h -> (band, mass, candidates)
+
+    def add(self, h, band, mass, candidates):
+        self.per_head[h] = (int(band), int(mass), int(candidates))
+
+    @property
+    def band(self):
+        return sum(v[0] for v in self.per_head.values())
+
+    @property
+    def mass(self):
+        return sum(v[1] for v in self.per_head.values())
+
+    @property
+    def worst_band_fraction(self):
+        return max((v[0] / max(v[2], 1) for v in self.per_head.values()), default=0.0)
+
+    def __int__(self):
+        return self.band + self.mass
+
+    def __str__(self):
+        return (f"{self.band} within the 1e-3 band (worst head {100 * self.worst_band_fraction:.2f} % of its "
+                f"candidates) + {self.mass} by the 1e-6 mass rule")
+
+    __repr__ = __str__
+
+
 def check_route(g, res, p, heads=None):
     """Returns the number of heads whose label was excused by the band around tau."""
     excused = 0
@@ -80,98 +133,35 @@ def check_route(g, res, p, heads=None):
     return excused
 
 
-def _ambiguous_vs(pd, p, k_d, raw):
-    """Blocks of one direction whose membership may legitimately differ."""
-    nb = pd.shape[0]
-    order = np.argsort(-pd, kind="stable")
-    amb = np.zeros(nb, dtype=bool)
-    if p.selector in (0, 2):
-        mu = orc.noise_floor(pd)[1] if p.selector == 0 else float(np.median(pd[1:nb - 1]))
-        thr = p.alpha * mu
-        amb |= np.abs(pd - thr) <= REL_BAND * thr
-    if p.selector == 1 and raw < nb:
-        # the running sum may reach gamma one entry earlier or later when it passes within 1e-6 of it
-        cs = np.cumsum(pd[order])
-        if cs[raw - 1] - p.gamma <= MASS_BAND:
-            amb[order[raw]] = True
-        if raw >= 2 and p.gamma - cs[raw - 2] <= MASS_BAND:
-            amb[order[raw - 1]] = True
-    if p.selector == 1 or raw < p.k_min_blocks:
-        if k_d < nb:
-            cut = pd[order[k_d - 1]]
-            amb |= np.abs(pd - cut) <= REL_BAND * cut
-            nxt = pd[order[k_d]]
-            amb |= np.abs(pd - nxt) <= REL_BAND * max(nxt, 1e-300)
-    return amb
-
-
-def _rows_to_matrix(cols_per_row, nb):
-    m = np.zeros((nb, nb), dtype=bool)
-    for r, c in enumerate(cols_per_row):
-        m[r, c] = True
-    return m
+def _check_bounds(h, bounds, band_limit):
+    assert max(bounds["mass_per_direction"]) <= 2, (h, "mass rule excused", bounds["mass_per_direction"])
+    frac = bounds["band"] / max(bounds["candidates"], 1)
+    assert frac <= band_limit, (h, f"{bounds['band']} of {bounds['candidates']} candidate blocks in the 1e-3 band")
 
 
 def gpu_matrix(g, h, nb):
-    """Boolean [N_b, N_b] matrix of the GPU lists of head h; also checks order and bounds."""
-    rp = g["row_ptr"][h]
-    cols = g["col_idx"][rp[0]:rp[nb]].astype(np.int64)
-    lens = np.diff(rp)
-    rows = np.repeat(np.arange(nb), lens)
-    assert lens.min() >= 1
-    assert np.all(cols <= rows) and np.all(cols >= 0), (h, "column out of range")
-    same_row = rows[1:] == rows[:-1]
-    assert np.all(np.diff(cols)[same_row] > 0), (h, "not ascending/unique")
-    first = rp[:-1] - rp[0]
-    last = rp[1:] - rp[0] - 1
-    assert np.all(cols[first] == 0) and np.all(cols[last] == np.arange(nb)), (h, "forced blocks missing")
-    m = np.zeros((nb, nb), dtype=bool)
-    m[rows, cols] = True
-    return m
+    """Boolean [N_b, N_b] matrix of the GPU lists of head h; also checks order, bounds and forced blocks."""
+    return matching.lists_to_matrix(g["row_ptr"][h], g["col_idx"], nb)
 
 
-def check_lists(g, res, p, heads=None):
-    """GPU lists vs oracle lists under the matching rule.  Returns the count of excused blocks."""
+def check_lists(g, res, p, heads=None, band_limit=1.0) -> Excused:
+    """GPU lists vs oracle lists under the matching rule.  Returns the excused blocks (int() = their number).
+    The share of a head's blocks inside the 1e-3 band is bounded only on request (band_limit): the small and
+    degenerate cases that call this directly have a handful of candidate blocks, or ties everywhere."""
     nb = -(-p.seq_len // p.block)
-    excused_total = 0
+    out = Excused()
     heads = range(len(res)) if heads is None else heads
     for h in heads:
         r = res[h]
         if r is None or g["pattern"][h] != r["pattern"]:
             continue  # label excused by check_route; lists follow the other branch
-        if nb <= 2:
-            lo = hi = _rows_to_matrix(r["cols"], nb)
-        elif r["pattern"] == orc.VS:
-            amb_v = _ambiguous_vs(r["p_v"], p, r["k_v"], r["raw_v"])
-            amb_s = _ambiguous_vs(r["p_s"], p, r["k_s"], r["raw_s"])
-            sv = np.zeros(nb, bool); sv[r["s_v"]] = True
-            ss = np.zeros(nb, bool); ss[r["s_s"]] = True
-            lo = _rows_to_matrix(orc.expand_vs(np.nonzero(sv & ~amb_v)[0], np.nonzero(ss & ~amb_s)[0], nb), nb)
-            hi = _rows_to_matrix(orc.expand_vs(np.nonzero(sv | amb_v)[0], np.nonzero(ss | amb_s)[0], nb), nb)
-            excused_total += int(amb_v.sum() + amb_s.sum())
-        else:
-            flat = r["a_bar"] / r["a_bar"].sum()
-            cut = r["pe_cut"]
-            tri = np.tril(np.ones((nb, nb), bool))
-            amb = (np.abs(flat - cut) <= REL_BAND * cut) & tri
-            # mass band: the cumulative sum may pass within 1e-6 of gamma, moving the cut by one entry
-            vals = np.where(tri, flat, -1.0).reshape(-1)
-            order = np.argsort(-vals, kind="stable")[:tri.sum()]
-            cs = np.cumsum(vals[order])
-            kstar = int(r["pe_sel"].sum())
-            if kstar < order.size and cs[kstar - 1] - p.gamma <= MASS_BAND:
-                amb.reshape(-1)[order[kstar]] = True
-            if kstar >= 2 and p.gamma - cs[kstar - 2] <= MASS_BAND:
-                amb.reshape(-1)[order[kstar - 1]] = True
-            lo = _rows_to_matrix(orc.expand_pe(r["pe_sel"] & ~amb), nb)
-            hi = _rows_to_matrix(orc.expand_pe(r["pe_sel"] | amb), nb)
-            excused_total += int(amb.sum())
-        got = gpu_matrix(g, h, nb)
-        missing = lo & ~got
-        extra = got & ~hi
-        assert not missing.any(), (h, "missing", np.argwhere(missing)[:8].tolist())
-        assert not extra.any(), (h, "extra", np.argwhere(extra)[:8].tolist())
-    return excused_total
+        bounds = matching.list_bounds(r, nb, **_rule_kwargs(p))
+        _check_bounds(h, bounds, band_limit)
+        missing, extra = matching.compare_lists(gpu_matrix(g, h, nb), bounds)
+        assert not missing, (h, "missing", missing)
+        assert not extra, (h, "extra", extra)
+        out.add(h, bounds["band"], bounds["mass"], bounds["candidates"])
+    return out
 
 
 def check_attention(g, q, k, v, p, samples, key="o", dense=False):
@@ -214,3 +204,143 @@ def sample_blocks(nb, hq, per_head, seed=0, always=()):
                     chosen.add(int(rng.integers(a, b)))
         out += [(h, m) for m in sorted(chosen)]
     return out
+
+
+# ------------------------------------------------------------------------------------------------------
+# The same checks with the oracle spread over a pool of forked worker processes (full-size configurations)
+# ------------------------------------------------------------------------------------------------------
+_CTX: Dict = {}      # set in the parent before the pool forks; read-only in the workers
+_CACHE: Dict = {}    # per worker: the fp32 copies of the head it worked on last
+
+
+def _bf16_bits(t: torch.Tensor) -> np.ndarray:
+    """Zero-copy int16 view of a CPU bf16 tensor (numpy has no bf16)."""
+    return t.contiguous().view(torch.int16).numpy()
+
+
+def _head_f32(name: str, h: int) -> np.ndarray:
+    bits = _CTX[name][:, h]
+    return ((bits.astype(np.uint32) & np.uint32(0xFFFF)) << np.uint32(16)).view(np.float32)
+
+
+def _worker_head(h: int):
+    if _CACHE.get("h") != h:
+        kv = orc.kv_head(h, _CTX["hq"], _CTX["hkv"])
+        _CACHE.clear()
+        _CACHE.update(h=h, q=_head_f32("q", h), k=_head_f32("k", kv), v=_head_f32("v", kv) if "v" in _CTX else None)
+    return _CACHE["q"], _CACHE["k"], _CACHE["v"]
+
+
+def _pool_init():
+    try:
+        from threadpoolctl import threadpool_limits
+        threadpool_limits(1)
+    except Exception:  # pragma: no cover
+        pass
+
+
+def _lists_worker(h: int):
+    """Oracle steps O1-O6 of one head and the comparison of its lists; returns only small results."""
+    qh, kh, _ = _worker_head(h)
+    kw, rule, nb = _CTX["oracle_kw"], _CTX["rule_kw"], _CTX["nb"]
+    r = orc.head_pipeline(qh, kh, **kw)
+    out = dict(h=h, c_struct=r["c_struct"], pattern=r["pattern"], p_v=r["p_v"], p_s=r["p_s"])
+    for key in ("s_v", "s_s", "k_v", "k_s", "raw_v", "raw_s", "pe_cut"):
+        if key in r:
+            out[key] = r[key]
+    if _CTX["pattern"][h] != r["pattern"]:
+        out["skipped"] = True      # the label differs: check_route decides whether that is excused
+        return out
+    bounds = matching.list_bounds(r, nb, **rule)
+    got = matching.lists_to_matrix(_CTX["row_ptr"][h], _CTX["col_idx"], nb)
+    missing, extra = matching.compare_lists(got, bounds)
+    out.update(band=bounds["band"], mass=bounds["mass"], candidates=bounds["candidates"],
+               mass_per_direction=bounds["mass_per_direction"], missing=missing, extra=extra)
+    return out
+
+
+def _attention_worker(task):
+    h, m, cols, got, got_lse = task
+    qh, kh, vh = _worker_head(h)
+    want, want_lse = orc.sparse_attention_block(qh, kh, vh, m, cols, _CTX["block"], _CTX["scale"])
+    err = got - want
+    rel = float(np.linalg.norm(err) / max(np.linalg.norm(want), 1e-30))
+    lse_err = None
+    if got_lse is not None:
+        lse_err = float(np.max(np.abs(got_lse - want_lse) - 1e-3 * np.abs(want_lse)))
+    return h, m, rel, float(np.abs(err).max()), lse_err
+
+
+class OraclePool:
+    """Worker processes that share the host copies of Q, K, V (and the GPU's lists) by fork."""
+
+    def __init__(self, p, qc, kc, vc=None, g=None, workers: Optional[int] = None):
+        _CTX.clear()
+        _CTX.update(q=_bf16_bits(qc), k=_bf16_bits(kc), hq=p.n_q_heads, hkv=p.n_kv_heads, block=p.block,
+                    nb=-(-p.seq_len // p.block), scale=(p.softmax_scale if p.softmax_scale > 0 else None),
+                    oracle_kw=oracle_kwargs(p), rule_kw=_rule_kwargs(p))
+        if vc is not None:
+            _CTX["v"] = _bf16_bits(vc)
+        if g is not None:
+            _CTX.update(pattern=g["pattern"], row_ptr=g["row_ptr"], col_idx=g["col_idx"])
+        n = workers or min(os.cpu_count() or 1, 16)
+        self.pool = multiprocessing.get_context("fork").Pool(n, initializer=_pool_init)
+        self.p = p
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
+        _CTX.clear()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def heads(self, g, heads: Sequence[int], band_limit=BAND_LIMIT):
+        """Routing and lists of `heads` against the oracle.  Returns (per-head oracle results (small parts
+        only), excused labels, Excused)."""
+        p = self.p
+        # heads routed to pooled estimation cost ten times more: start them first
+        order = sorted(heads, key=lambda h: (g["pattern"][h] != orc.PE, h))
+        res: List[Optional[Dict]] = [None] * p.n_q_heads
+        for out in self.pool.imap_unordered(_lists_worker, order):
+            res[out["h"]] = out
+        labels = check_route(g, res, p, heads=heads)
+        exc = Excused()
+        for h in heads:
+            r = res[h]
+            if r.get("skipped"):
+                continue
+            _check_bounds(h, r, band_limit)
+            assert not r["missing"], (h, "missing", r["missing"])
+            assert not r["extra"], (h, "extra", r["extra"])
+            exc.add(h, r["band"], r["mass"], r["candidates"])
+        return res, labels, exc
+
+    def attention(self, g, samples, fetch_block, lse=None, dense=False):
+        """Sampled query blocks (h, m) against exact attention over the GPU's lists (or every causal block).
+        fetch_block(h, m) returns the GPU output of the block as float32 [rows, 128]."""
+        B = self.p.block
+        tasks = []
+        for h, m in samples:
+            cols = np.arange(m + 1) if dense else np.asarray(gpu_cols(g, h, m))
+            got = fetch_block(h, m)
+            got_lse = None if lse is None else np.asarray(lse[h, m * B:m * B + got.shape[0]])
+            tasks.append((h, m, cols, got, got_lse))
+        # longest lists first, grouped by head so that a worker converts a head's Q, K, V once per chunk
+        per_head = {}
+        for t in tasks:
+            per_head[t[0]] = per_head.get(t[0], 0) + len(t[2])
+        tasks.sort(key=lambda t: (-per_head[t[0]], t[0], -len(t[2])))
+        worst_rel = worst_abs = 0.0
+        blocks = 0
+        for h, m, rel, mab, lse_err in self.pool.imap_unordered(_attention_worker, tasks, chunksize=2):
+            assert rel <= 1e-2, (h, m, rel)
+            assert mab <= 2e-2, (h, m, mab)
+            assert lse_err is None or lse_err <= 2e-3, (h, m, "lse", lse_err)
+            worst_rel, worst_abs = max(worst_rel, rel), max(worst_abs, mab)
+        for t in tasks:
+            blocks += len(t[2])
+        return worst_rel, worst_abs, blocks

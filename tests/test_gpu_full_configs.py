@@ -1,9 +1,16 @@
 """The five workload configurations at their full sizes, in the launch configuration bench.py times.
 
-Routing (C_struct, labels, p_v, p_s) is checked for every head; the index lists for every VS head and a
-subset of the PE heads (all of them with CRISP_TEST_FULL=1); attention on sampled query blocks against
-the oracle's exact attention over the GPU's own lists (64 per head at 512k with CRISP_TEST_FULL=1,
-fewer by default so that the suite stays within a few minutes of host time).
+For every head: routing (C_struct, label, p_v, p_s) and the index lists against the oracle's steps O1-O6
+(all pooled-estimation heads included).  Attention: sampled query blocks against the oracle's exact
+attention over the GPU's own lists - per head block 0, block N_b - 1, the block with the longest list and
+random ones stratified over the four quartiles of m:
+    L32k   every head, 32 blocks (seed 0; 16 for seeds 1 and 2)
+    L128k  every head, 16 blocks
+    Q256k  every head, 32 blocks
+    L512k  every head, 64 blocks
+With CRISP_TEST_FULL=1 L32k is checked on all of its 256 query blocks per head.
+The oracle runs in a pool of worker processes (tests/parity_utils.py); the whole file takes about five minutes
+on a 16-core host.
 """
 import os
 import time
@@ -33,19 +40,27 @@ def _oracle_heads(qc, kc, p, heads, pu):
     return out
 
 
-def _route_only(qc, kc, p, h):
-    """Oracle steps O1-O3 of one head (cheap at any size)."""
-    hq, hkv = p.n_q_heads, p.n_kv_heads
-    a = orc.proxy_attention(qc[:, h].float().numpy(), kc[:, orc.kv_head(h, hq, hkv)].float().numpy(), p.block)
-    c = orc.c_struct(a, p.sink_tokens, p.local_tokens)
-    p_v, p_s = orc.block_scores(a, p.block)
-    return dict(c_struct=c, pattern=orc.route(c, p.tau), p_v=p_v, p_s=p_s)
+def _one_head_per_group_and_class(w):
+    """The first head of every head class inside every KV group."""
+    seen, heads = set(), []
+    for h, cls in enumerate(w.head_classes):
+        key = (h // w.group, cls)
+        if key not in seen:
+            seen.add(key)
+            heads.append(h)
+    return heads
 
 
-def _config_check(name, pe_heads_default, blocks_default, blocks_full, dense_blocks=2):
+def _block_fetcher(layer):
+    def fetch(h, m):
+        return layer.o[m * 128:(m + 1) * 128, h].float().cpu().numpy()
+    return fetch
+
+
+def _config_check(w, attention_heads, blocks_default, blocks_full, dense_blocks=4, report=None, band_limit=None):
     pu = _pu()
     import paper_2609_01925_b200 as crisp
-    w = synth.CONFIGS[name]
+    name = w.name + (f" seed {w.seed}" if w.seed else "")
     p = pu.params_of(w)
     t0 = time.time()
     q, k, v = synth.make_qkv(w, device="cuda")
@@ -59,64 +74,52 @@ def _config_check(name, pe_heads_default, blocks_default, blocks_full, dense_blo
              col_idx=layer.col_idx[:nnz].cpu().numpy(), nnz=nnz, o=None, lse=layer.lse.cpu().numpy())
     qc, kc, vc = q.cpu(), k.cpu(), v.cpu()
     hq, nb = w.n_q_heads, w.n_blocks
-    # routing for every head
-    labels = 0
-    route_res = [_route_only(qc, kc, p, h) for h in range(hq)]
-    labels = pu.check_route(g, route_res, p)
-    # lists: every VS head, some PE heads
-    vs_heads = [h for h in range(hq) if route_res[h]["pattern"] == orc.VS]
-    pe_heads = [h for h in range(hq) if route_res[h]["pattern"] == orc.PE]
-    if not FULL:
-        pe_heads = pe_heads[:pe_heads_default]
-    res = _oracle_heads(qc, kc, p, vs_heads + pe_heads, pu)
-    excused = pu.check_lists(g, res, p, heads=vs_heads + pe_heads)
-    # attention on sampled query blocks: the output tensor is pulled block by block
-    per_head = blocks_full if FULL else blocks_default
     lens = np.diff(g["row_ptr"], axis=1)
-    heads = range(hq) if FULL else sorted(set(vs_heads[:2] + pe_heads[:2] + [hq - 1]))
-    samples = []
-    for h in heads:
-        longest = int(np.argmax(lens[h]))
-        samples += [s for s in pu.sample_blocks(nb, hq, per_head, seed=h, always=(longest,)) if s[0] == h]
-    o_host = {}
-    for h, m in samples:
-        o_host[(h, m)] = layer.o[m * 128:(m + 1) * 128, h].float().cpu().numpy()
-
-    class _O:
-        def __getitem__(self, idx):
-            rows, h = idx
-            return o_host[(h, rows.start // 128)]
-    g["o"] = _O()
-    rel, mab = pu.check_attention(g, qc, kc, vc, p, samples)
-    # the dense kernel on the same inputs
-    layer.dense_prefill(q, k, v)
-    layer.poll()
-    torch.cuda.synchronize()
-    g["lse_dense"] = layer.lse.cpu().numpy()
-    dense_samples = [(h, m) for h, m in samples if m in (0, nb - 1)][:dense_blocks * 2]
-    for h, m in dense_samples:
-        o_host[(h, m)] = layer.o[m * 128:(m + 1) * 128, h].float().cpu().numpy()
-    g["o_dense"] = g["o"]
-    pu.check_attention(g, qc, kc, vc, p, dense_samples, key="o_dense", dense=True)
+    per_head = blocks_full if FULL else blocks_default
+    heads = list(range(hq)) if (FULL or attention_heads == "all") else _one_head_per_group_and_class(w)
+    with pu.OraclePool(p, qc, kc, vc, g) as pool:
+        # routing and lists: every head
+        res, labels, excused = pool.heads(g, list(range(hq)), band_limit=band_limit or pu.BAND_LIMIT)
+        t_lists = time.time() - t0
+        samples = []
+        for h in heads:
+            longest = int(np.argmax(lens[h]))
+            samples += [s for s in pu.sample_blocks(nb, hq, per_head, seed=h, always=(longest,)) if s[0] == h]
+        rel, mab, blocks = pool.attention(g, samples, _block_fetcher(layer), lse=g["lse"])
+        # the dense kernel on the same inputs: the last block of two heads and two blocks inside
+        layer.dense_prefill(q, k, v)
+        layer.poll()
+        torch.cuda.synchronize()
+        lse_dense = layer.lse.cpu().numpy()
+        picks = [(heads[0], nb - 1), (heads[-1], nb - 1), (heads[len(heads) // 2], nb // 2), (heads[0], 0),
+                 (heads[-1], nb // 3), (heads[1 % len(heads)], 1)][:dense_blocks]
+        drel, dmab, dblocks = pool.attention(g, picks, _block_fetcher(layer), lse=lse_dense, dense=True)
+    n_vs = int((g["pattern"] == orc.VS).sum())
     frac = nnz / (hq * nb * (nb + 1) // 2)
-    print(f"{name}: VS heads {len(vs_heads)}, PE heads checked {len(pe_heads)}, excused labels {labels}, "
-          f"excused blocks {excused}, block fraction {frac:.3f}, {len(samples)} sampled blocks, "
-          f"rel-L2 {rel:.2e}, max-abs {mab:.2e}, {time.time() - t0:.0f} s")
+    line = (f"{name}: lists of all {hq} heads ({n_vs} VS, {hq - n_vs} PE) match; excused labels {labels}; excused "
+            f"blocks: {excused}; block fraction {frac:.3f}; attention on {len(samples)} query blocks "
+            f"({per_head} per head on {len(heads)} heads, {blocks} key blocks): rel-L2 {rel:.2e}, max-abs {mab:.2e}; "
+            f"dense kernel on {len(picks)} query blocks ({dblocks} key blocks): rel-L2 {drel:.2e}, max-abs {dmab:.2e}; "
+            f"{t_lists:.0f} s lists + {time.time() - t0 - t_lists:.0f} s attention")
+    print(line)
+    if report is not None:
+        report(line)
     return layer, g, (q, k, v), (qc, kc, vc), res
 
 
-def test_config_L32k():
-    _config_check("L32k", pe_heads_default=4, blocks_default=6, blocks_full=256)
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_config_L32k(seed, parity_report):
+    w = synth.CONFIGS["L32k"].with_(seed=seed)
+    _config_check(w, "all", blocks_default=32 if seed == 0 else 16, blocks_full=256, report=parity_report)
 
 
-def test_config_L128k_alpha_sweep_and_gamma_selector():
+def test_config_L128k_alpha_sweep_and_gamma_selector(parity_report):
     pu = _pu()
-    import paper_2609_01925_b200 as crisp
-    layer, g, (q, k, v), (qc, kc, vc), res = _config_check("L128k", pe_heads_default=2, blocks_default=4,
-                                                            blocks_full=64)
     w = synth.CONFIGS["L128k"]
+    layer, g, (q, k, v), (qc, kc, vc), res = _config_check(w, "all", blocks_default=16, blocks_full=64,
+                                                            report=parity_report)
     hq, nb = w.n_q_heads, w.n_blocks
-    vs_heads = [h for h in range(hq) if g["pattern"][h] == orc.VS][: (hq if FULL else 4)]
+    vs_heads = [h for h in range(hq) if g["pattern"][h] == orc.VS]
     nnz_by = {}
     for label, over in (("alpha=0.5", dict(alpha=0.5)), ("alpha=2.0", dict(alpha=2.0)),
                         ("gamma=0.95", dict(selector=1))):
@@ -138,20 +141,24 @@ def test_config_L128k_alpha_sweep_and_gamma_selector():
                 s_s, ks_, raw_s = orc.select_noise_floor(r["p_s"], p2.alpha, p2.k_min_blocks)
             res2[h] = dict(r, s_v=s_v, s_s=s_s, k_v=kv_, k_s=ks_, raw_v=raw_v, raw_s=raw_s,
                            cols=orc.expand_vs(s_v, s_s, nb))
-        exc = pu.check_lists(g2, res2, p2, heads=vs_heads)
+        exc = pu.check_lists(g2, res2, p2, heads=vs_heads, band_limit=pu.BAND_LIMIT)
         rows_vs = sum(int(np.diff(g2["row_ptr"][h]).sum()) for h in vs_heads)
         nnz_by[label] = rows_vs
-        print(f"L128k {label}: excused blocks {exc}, listed blocks on {len(vs_heads)} VS heads {rows_vs}")
+        line = f"L128k {label}: lists of all {len(vs_heads)} VS heads match; excused blocks: {exc}; listed blocks {rows_vs}"
+        print(line)
+        parity_report(line)
     base = sum(int(np.diff(g["row_ptr"][h]).sum()) for h in vs_heads)
     assert nnz_by["alpha=2.0"] <= base <= nnz_by["alpha=0.5"]
 
 
-def test_config_Q256k():
-    _config_check("Q256k", pe_heads_default=1, blocks_default=3, blocks_full=64)
+def test_config_Q256k(parity_report):
+    # the sink-dominated heads have a flat background: ~8 % of their blocks lie within 0.1 % of alpha * mu
+    _config_check(synth.CONFIGS["Q256k"], "all", blocks_default=32, blocks_full=64, report=parity_report,
+                  band_limit=0.10)
 
 
-def test_config_L512k():
-    _config_check("L512k", pe_heads_default=1, blocks_default=3, blocks_full=64)
+def test_config_L512k(parity_report):
+    _config_check(synth.CONFIGS["L512k"], "all", blocks_default=64, blocks_full=64, report=parity_report)
 
 
 def test_maximum_block_count_one_million_tokens():
@@ -174,7 +181,9 @@ def test_maximum_block_count_one_million_tokens():
     qc, kc, vc = q.cpu(), k.cpu(), v.cpu()
     res = _oracle_heads(qc, kc, p, [0, 1], pu)
     pu.check_route(g, res, p)
-    excused = pu.check_lists(g, res, p)
+    # head 1 is a diffuse head forced to Vertical-Slash: its block scores are flat, so a third of them lie in
+    # the 1e-3 band around alpha * mu
+    excused = pu.check_lists(g, res, p, band_limit=1.0)
     nb = w.n_blocks
     samples = [(0, 0), (0, nb - 1), (0, 5000), (1, nb - 1), (1, 1234)]
     o_host = {(h, m): layer.o[m * 128:(m + 1) * 128, h].float().cpu().numpy() for h, m in samples}
