@@ -242,6 +242,20 @@ int crisp_forward_varlen(const crisp_params* p, const int64_t* cu_seqlens, int32
                          int32_t* device_status, void* o, float* lse, int32_t dense_below_tokens, void* cuda_stream);
 
 /*
+ * Diagnostic (the paper has no counterpart): per-kernel device times of the stage calls, for benchmarks.
+ * crisp_profile_enable(1) discards earlier records and switches recording on: from then on every kernel the
+ * library launches is bracketed by two CUDA events on the caller's stream (the events are created on first use
+ * and reused; this is host-side bookkeeping, but it is not meant for a production loop - it adds an event pair
+ * per kernel and a process-wide lock).  crisp_profile_enable(0) switches it off and discards the records.
+ * crisp_profile_read waits for the recorded kernels and returns, in launch order, up to max_records records:
+ * names (HOST buffer of names_bytes bytes) receives the kernels' names separated by '\n', ms (HOST array of
+ * max_records floats) their device times in milliseconds; *n_records = how many were returned.  Do not read
+ * while a stream that holds recorded kernels is being captured.
+ */
+int crisp_profile_enable(int on);
+int crisp_profile_read(char* names, size_t names_bytes, float* ms, int32_t max_records, int32_t* n_records);
+
+/*
  * Diagnostic (the paper has no counterpart): exercises the library's failure-reporting path without any
  * failure.  Enqueues one tiny kernel that waits on a barrier nothing arrives at, with a wait limit of
  * `limit_ns` nanoseconds (1 .. 10,000,000); the wait runs out, a second role waiting with the normal limit is

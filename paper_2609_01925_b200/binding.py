@@ -29,7 +29,7 @@ EXPORTS = (
     "crisp_version", "crisp_status_string", "crisp_last_cuda_error", "crisp_workspace_bytes",
     "crisp_route", "crisp_route_static", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
     "crisp_poll_device_status", "crisp_forward", "crisp_route_jsd", "crisp_varlen_layout",
-    "crisp_forward_varlen", "crisp_selftest_bounded_wait",
+    "crisp_forward_varlen", "crisp_selftest_bounded_wait", "crisp_profile_enable", "crisp_profile_read",
 )
 
 
@@ -105,6 +105,11 @@ def load() -> ctypes.CDLL:
     lib.crisp_forward_varlen.restype = ctypes.c_int
     lib.crisp_forward_varlen.argtypes = [P, vp, ctypes.c_int32, vp, vp, vp, vp, sz, vp, sz, vp, sz, vp, vp, vp, vp,
                                          vp, vp, i64, vp, vp, vp, vp, ctypes.c_int32, vp]
+    lib.crisp_profile_enable.restype = ctypes.c_int
+    lib.crisp_profile_enable.argtypes = [ctypes.c_int]
+    lib.crisp_profile_read.restype = ctypes.c_int
+    lib.crisp_profile_read.argtypes = [ctypes.c_char_p, sz, ctypes.POINTER(ctypes.c_float), ctypes.c_int32,
+                                       ctypes.POINTER(ctypes.c_int32)]
     lib.crisp_selftest_bounded_wait.restype = ctypes.c_int
     lib.crisp_selftest_bounded_wait.argtypes = [vp, sz, i64, vp]
     lib.crisp_poll_device_status.restype = ctypes.c_int
@@ -224,6 +229,21 @@ def crisp_forward_varlen(p, cu_seqlens, q, k, v, route_ws, select_ws, prefill_ws
                                        _ptr(row_ptr), _ptr(col_idx), int(capacity), _ptr(nnz_needed),
                                        _ptr(device_status), _ptr(o), _ptr(lse), int(dense_below_tokens),
                                        _stream(stream))
+
+
+def crisp_profile_enable(on: bool) -> int:
+    return load().crisp_profile_enable(1 if on else 0)
+
+
+def crisp_profile_read(max_records: int = 4096):
+    """[(kernel name, milliseconds)] of the kernels launched since crisp_profile_enable(True), in launch order."""
+    names = ctypes.create_string_buffer(64 * max_records)
+    ms = (ctypes.c_float * max_records)()
+    n = ctypes.c_int32(0)
+    rc = load().crisp_profile_read(names, len(names), ms, max_records, ctypes.byref(n))
+    if rc != OK:
+        raise CrispError(rc, "crisp_profile_read")
+    return list(zip(names.value.decode().split("\n")[:n.value], [float(x) for x in ms[:n.value]]))
 
 
 def crisp_selftest_bounded_wait(ws, limit_ns, stream=None) -> int:

@@ -32,6 +32,47 @@ EncodeTiledFn encode_fn() {
 }
 }  // namespace
 
+// ---- optional per-kernel timing
+namespace {
+struct ProfRecord {
+  const char* name;
+  cudaEvent_t begin, end;
+};
+std::mutex g_prof_mutex;
+bool g_prof_on = false;
+std::vector<ProfRecord> g_prof_records;
+std::vector<cudaEvent_t> g_prof_free;  // events of earlier records, reused
+
+cudaEvent_t prof_event() {
+  if (!g_prof_free.empty()) {
+    cudaEvent_t e = g_prof_free.back();
+    g_prof_free.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+  return e;
+}
+}  // namespace
+
+bool prof_enabled() {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  return g_prof_on;
+}
+void prof_begin(const char* name, cudaStream_t stream) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  if (!g_prof_on) return;
+  ProfRecord r{name, prof_event(), prof_event()};
+  if (r.begin) cudaEventRecord(r.begin, stream);
+  g_prof_records.push_back(r);
+}
+void prof_end(cudaStream_t stream) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  if (!g_prof_on || g_prof_records.empty()) return;
+  ProfRecord& r = g_prof_records.back();
+  if (r.end) cudaEventRecord(r.end, stream);
+}
+
 void set_cuda_error(cudaError_t e, const char* where) {
   std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
 }
@@ -370,6 +411,42 @@ int crisp_forward_varlen(const crisp_params* p, const int64_t* cu_seqlens, int32
       CRISP_CUDA_TRY(cudaMemcpyAsync(device_status + 2 * b + 1, prefill_ws, sizeof(int32_t), cudaMemcpyDeviceToDevice, st),
                      "forward_varlen: attention status");
   }
+  return CRISP_OK;
+}
+
+int crisp_profile_enable(int on) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  for (ProfRecord& r : g_prof_records) {
+    if (r.begin) g_prof_free.push_back(r.begin);
+    if (r.end) g_prof_free.push_back(r.end);
+  }
+  g_prof_records.clear();
+  g_prof_on = on != 0;
+  return CRISP_OK;
+}
+
+int crisp_profile_read(char* names, size_t names_bytes, float* ms, int32_t max_records, int32_t* n_records) {
+  if (!n_records || max_records < 0 || (max_records > 0 && (!names || !ms))) return CRISP_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  size_t used = 0;
+  int32_t n = 0;
+  if (names && names_bytes > 0) names[0] = 0;
+  for (const ProfRecord& r : g_prof_records) {
+    if (n >= max_records) break;
+    const size_t len = std::strlen(r.name);
+    if (used + len + 2 > names_bytes) break;
+    float t = -1.f;
+    if (r.begin && r.end) {
+      CRISP_CUDA_TRY(cudaEventSynchronize(r.end), "profile: synchronize");
+      CRISP_CUDA_TRY(cudaEventElapsedTime(&t, r.begin, r.end), "profile: elapsed time");
+    }
+    std::memcpy(names + used, r.name, len);
+    used += len;
+    names[used++] = '\n';
+    names[used] = 0;
+    ms[n++] = t;
+  }
+  *n_records = n;
   return CRISP_OK;
 }
 

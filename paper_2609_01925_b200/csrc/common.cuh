@@ -50,6 +50,28 @@ int make_tmap_bf16_nhd(CUtensorMap* out, const void* base, int n, int heads, int
     }                                            \
   } while (0)
 
+// Optional per-kernel timing (diagnostic, off by default; see crisp_profile_enable): while it is on, every kernel
+// launch of the stage launchers is bracketed by a pair of CUDA events on the caller's stream.
+bool prof_enabled();
+void prof_begin(const char* name, cudaStream_t stream);
+void prof_end(cudaStream_t stream);
+struct ProfScope {
+  cudaStream_t stream;
+  bool on;
+  ProfScope(const char* name, cudaStream_t s) : stream(s), on(prof_enabled()) {
+    if (on) prof_begin(name, stream);
+  }
+  ~ProfScope() {
+    if (on) prof_end(stream);
+  }
+};
+// CRISP_KERNEL("name", stream, kernel<<<grid, block, smem, stream>>>(args));
+#define CRISP_KERNEL(name, stream, ...)          \
+  do {                                           \
+    ::crisp::ProfScope prof_scope__(name, stream); \
+    __VA_ARGS__;                                 \
+  } while (0)
+
 #ifdef __CUDACC__
 // Exclusive prefix sum over the 1024 threads of a block, in thread order (warp shuffles, then the 32 warp
 // totals).  `scratch` holds 33 values; `*total` (optional) receives the sum of all threads.  Every thread of

@@ -903,21 +903,21 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
-    prefill_kernel<true><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a);
+    CRISP_KERNEL("prefill_dense", stream, prefill_kernel<true><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a));
   } else {
     const int words = (d.nb + 31) / 32;
     CRISP_CUDA_TRY(cudaMemsetAsync(w.cost_hist, 0, sizeof(int) * w.n_bins, stream), "prefill: clear histogram");
-    merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
+    CRISP_KERNEL("merge_lists", stream, merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
         d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate, a.status,
-        static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2);
-    sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins);
-    sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, 0, stream>>>(d, row_ptr, w.cost_hist,
+        static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2));
+    CRISP_KERNEL("sched_scan", stream, sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins));
+    CRISP_KERNEL("sched_scatter", stream, sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, 0, stream>>>(d, row_ptr, w.cost_hist,
                                                                                w.order, a.n_pairs, w.n_cost, a.group_kv, gate,
-                                                                               a.status);
+                                                                               a.status));
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
-    prefill_kernel<false><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a);
+    CRISP_KERNEL("prefill_sparse", stream, prefill_kernel<false><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a));
   }
   CRISP_CUDA_TRY(cudaGetLastError(), "prefill: launch");
   return CRISP_OK;

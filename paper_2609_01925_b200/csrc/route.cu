@@ -490,11 +490,11 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   int slices = n_sm / groups;
   if (slices < 1) slices = 1;
   if (slices > d.nb) slices = d.nb;
-  proxy<<<dim3(slices, groups), 288, smem, stream>>>(tq, tk, d, w, status, n_head_chunks);
-  row_stats_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w);
-  row_final_kernel<<<d.hq, 128, 0, stream>>>(d, w);
-  tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v);
-  finalize_kernel<<<d.hq, 256, 0, stream>>>(d, w, p_s, c_struct, pattern);
+  CRISP_KERNEL("proxy", stream, proxy<<<dim3(slices, groups), 288, smem, stream>>>(tq, tk, d, w, status, n_head_chunks));
+  CRISP_KERNEL("row_stats", stream, row_stats_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w));
+  CRISP_KERNEL("row_final", stream, row_final_kernel<<<d.hq, 128, 0, stream>>>(d, w));
+  CRISP_KERNEL("tile_sums", stream, tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v));
+  CRISP_KERNEL("finalize", stream, finalize_kernel<<<d.hq, 256, 0, stream>>>(d, w, p_s, c_struct, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route: launch");
   return CRISP_OK;
 }

@@ -810,13 +810,13 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   CRISP_CUDA_TRY(cudaFuncSetAttribute(select_vs_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       static_cast<int>(vs_smem)),
                  "select: smem attribute");
-  select_vs_kernel<<<dim3(d.hq, 2), 1024, vs_smem, stream>>>(d, pattern, p_v, p_s, w);
+  CRISP_KERNEL("select_vs", stream, select_vs_kernel<<<dim3(d.hq, 2), 1024, vs_smem, stream>>>(d, pattern, p_v, p_s, w));
 
   // PE heads (every kernel returns at once for heads routed to VS)
   const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
   const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
-  pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, kb, d.hkv, 0, pattern, w.kbar, w.ksplit);
-  pool_kernel<<<dim3(d.nb, d.hq), 128, 0, stream>>>(d, qb, d.hq, 1, pattern, w.qbar, w.qsplit);
+  CRISP_KERNEL("pool_k", stream, pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, kb, d.hkv, 0, pattern, w.kbar, w.ksplit));
+  CRISP_KERNEL("pool_q", stream, pool_kernel<<<dim3(d.nb, d.hq), 128, 0, stream>>>(d, qb, d.hq, 1, pattern, w.qbar, w.qsplit));
   {
     LogitsMaps maps;
     for (int pl = 0; pl < 3; ++pl) {
@@ -830,22 +830,22 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
                                         static_cast<int>(smem)),
                    "select: smem attribute");
     const int nt = (d.nb + kBlock - 1) / kBlock;
-    pe_logits_kernel<<<dim3(nt, nt, d.hq), 160, smem, stream>>>(maps, d, pattern, w, status);
+    CRISP_KERNEL("pe_logits", stream, pe_logits_kernel<<<dim3(nt, nt, d.hq), 160, smem, stream>>>(maps, d, pattern, w, status));
   }
-  pe_normalise_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w);
+  CRISP_KERNEL("pe_normalise", stream, pe_normalise_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w));
   const int hist_ctas = d.nb < 128 ? d.nb : 128;
   for (int level = 0; level < 3; ++level) {
-    pe_hist_kernel<<<dim3(hist_ctas, d.hq), 256, 0, stream>>>(d, pattern, w, level);
-    pe_cut_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w, level);
+    CRISP_KERNEL("pe_hist", stream, pe_hist_kernel<<<dim3(hist_ctas, d.hq), 256, 0, stream>>>(d, pattern, w, level));
+    CRISP_KERNEL("pe_cut", stream, pe_cut_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w, level));
   }
-  pe_row_stats_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w);
-  pe_take_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w);
+  CRISP_KERNEL("pe_row_stats", stream, pe_row_stats_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w));
+  CRISP_KERNEL("pe_take", stream, pe_take_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w));
 
   // expansion + compaction
-  count_vs_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w);
-  scan_rows_kernel<<<1, 1024, 0, stream>>>(d, w, row_ptr, capacity, nnz_needed, status);
-  fill_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w, row_ptr, col_idx, capacity,
-                                                              nnz_needed);
+  CRISP_KERNEL("count_vs", stream, count_vs_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w));
+  CRISP_KERNEL("scan_rows", stream, scan_rows_kernel<<<1, 1024, 0, stream>>>(d, w, row_ptr, capacity, nnz_needed, status));
+  CRISP_KERNEL("fill", stream, fill_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w, row_ptr, col_idx, capacity,
+                                                              nnz_needed));
   CRISP_CUDA_TRY(cudaGetLastError(), "select: launch");
   return CRISP_OK;
 }
@@ -937,10 +937,10 @@ int launch_route_jsd(const Dims& d, const void* q, const void* k, const float* p
   size_t total;
   SelectPtrs w = carve(d, ws, &total);
   CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "route_jsd: clear status");
-  pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, static_cast<const __nv_bfloat16*>(k), d.hkv, 0, nullptr,
-                                                     w.kbar, nullptr);
-  jsd_kernel<<<d.hq, 256, sizeof(float) * d.nb, stream>>>(d, static_cast<const __nv_bfloat16*>(q), w.kbar, p_v,
-                                                         tau_jsd, jsd, pattern);
+  CRISP_KERNEL("pool_k", stream, pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, static_cast<const __nv_bfloat16*>(k), d.hkv, 0, nullptr,
+                                                     w.kbar, nullptr));
+  CRISP_KERNEL("jsd", stream, jsd_kernel<<<d.hq, 256, sizeof(float) * d.nb, stream>>>(d, static_cast<const __nv_bfloat16*>(q), w.kbar, p_v,
+                                                         tau_jsd, jsd, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route_jsd: launch");
   return CRISP_OK;
 }

@@ -39,7 +39,7 @@ def test_pool_accepts_oracle_results_and_catches_planted_errors():
 
     samples = pu.sample_blocks(nb, hq, 4, seed=1)
     with pu.OraclePool(p, q, k, v, g, workers=2) as pool:
-        small, labels, exc = pool.heads(g, list(range(hq)))
+        small, labels, exc = pool.heads(g, list(range(hq)), band_limit=1.0)   # 32 blocks: two in the band are 3 %
         assert labels == 0 and set(exc.per_head) == set(range(hq))
         assert [r["pattern"] for r in small] == [r["pattern"] for r in res]
         rel, mab, blocks = pool.attention(g, samples, fetch)
@@ -58,4 +58,4 @@ def test_pool_accepts_oracle_results_and_catches_planted_errors():
     g2["row_ptr"], g2["col_idx"] = orc.cols_to_csr(lists)
     with pu.OraclePool(p, q, k, v, g2, workers=2) as pool:
         with pytest.raises(AssertionError, match="extra"):
-            pool.heads(g2, [h])
+            pool.heads(g2, [h], band_limit=1.0)
