@@ -73,10 +73,13 @@ struct ProfScope {
   } while (0)
 
 #ifdef __CUDACC__
-// Exclusive prefix sum over the 1024 threads of a block, in thread order (warp shuffles, then the 32 warp
-// totals).  `scratch` holds 33 values; `*total` (optional) receives the sum of all threads.  Every thread of
-// the block must call it; it contains two __syncthreads and leaves `scratch` reusable after the second.
-__device__ __forceinline__ long long block_exclusive_scan_1024(long long v, long long* scratch, long long* total) {
+// Exclusive prefix sum over the kThreads threads of a block (a multiple of 32, at most 1024), in thread order
+// (warp shuffles, then the warp totals).  `scratch` holds 33 values; `*total` (optional) receives the sum of all
+// threads.  Every thread of the block must call it; it contains three __syncthreads and leaves `scratch` reusable
+// after the last.
+template <int kThreads>
+__device__ __forceinline__ long long block_exclusive_scan(long long v, long long* scratch, long long* total) {
+  constexpr int kWarps = kThreads / 32;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   long long incl = v;
 #pragma unroll
@@ -88,19 +91,22 @@ __device__ __forceinline__ long long block_exclusive_scan_1024(long long v, long
   if (lane == 31) scratch[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    const long long wt = scratch[lane];
+    const long long wt = lane < kWarps ? scratch[lane] : 0;
     long long wi = wt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const long long t = __shfl_up_sync(0xffffffffu, wi, o);
       if (lane >= o) wi += t;
     }
-    scratch[lane] = wi - wt;
+    if (lane < kWarps) scratch[lane] = wi - wt;
     if (lane == 31) scratch[32] = wi;
   }
   __syncthreads();
   if (total) *total = scratch[32];
   return scratch[warp] + (incl - v);
+}
+__device__ __forceinline__ long long block_exclusive_scan_1024(long long v, long long* scratch, long long* total) {
+  return block_exclusive_scan<1024>(v, scratch, total);
 }
 #endif
 

@@ -708,19 +708,12 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 
 // Union of the lists of query blocks (2u, 2u+1) of one head, with per-tile flags.  One warp per pair;
 // the two lists become bitmaps in shared memory, the union is emitted in ascending order.
-__global__ void __launch_bounds__(128)
-merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                   int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
-                   int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate, int* __restrict__ status,
-                   long long merged_capacity) {
-  extern __shared__ uint32_t bm[];
-  if (gate != nullptr && *gate != 0) return;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
-  const int words = (d.nb + 31) / 32;
-  uint32_t* b0 = bm + static_cast<size_t>(warp) * 2 * words;
-  uint32_t* b1 = b0 + words;
-  if (u >= n_pairs) return;
+__device__ __forceinline__ void merge_pair(const Dims& d, const int64_t* __restrict__ row_ptr,
+                                           const int32_t* __restrict__ col_idx, int32_t* __restrict__ merged,
+                                           int* __restrict__ item_len, int* __restrict__ cost_hist, int n_pairs,
+                                           int n_cost, int group_kv, int* __restrict__ status,
+                                           long long merged_capacity, uint32_t* b0, uint32_t* b1, int words, int u,
+                                           int h, int lane) {
   const int m0 = 2 * u, m1 = 2 * u + 1;
   for (int i = lane; i < 2 * words; i += 32) b0[i] = 0u;
   __syncwarp();
@@ -745,8 +738,6 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
         const int64_t i = i0 + 32 * u + lane;
         c[u] = i < to ? col_idx[i] : -1;
       }
-      // the lists are sorted, so the 32 entries of a load fall into one or two words: lanes with the same word
-      // combine their bits and one of them updates the bitmap
 #pragma unroll
       for (int u = 0; u < 4; ++u) {
         const int64_t i = i0 + 32 * u + lane;
@@ -756,6 +747,8 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
         const bool okc = !live || (c[u] >= 0 && c[u] <= m && c[u] > before && (i + 1 < to || c[u] == m));
         bad = bad || !okc;
         prev_last = __shfl_sync(0xffffffffu, c[u], 31);
+        // the entries ascend, so the 32 of a load fall into one or two words (more in a thin list): lanes with the
+        // same word combine their bits and one of them updates the bitmap
         const int wd = (live && okc) ? (c[u] >> 5) : -1;
         const unsigned int peers = __match_any_sync(0xffffffffu, wd);
         const uint32_t mine = wd >= 0 ? (1u << (c[u] & 31)) : 0u;
@@ -796,6 +789,23 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   }
 }
 
+// One warp per pair of query blocks; each also enters its pair into the histogram of the schedule's sort keys.
+__global__ void __launch_bounds__(128)
+merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                   int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
+                   int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate, int* __restrict__ status,
+                   long long merged_capacity) {
+  extern __shared__ uint32_t bm[];
+  if (gate != nullptr && *gate != 0) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
+  const int words = (d.nb + 31) / 32;
+  uint32_t* b0 = bm + static_cast<size_t>(warp) * 2 * words;
+  if (u < n_pairs)
+    merge_pair(d, row_ptr, col_idx, merged, item_len, cost_hist, n_pairs, n_cost, group_kv, status, merged_capacity,
+               b0, b0 + words, words, u, h, lane);
+}
+
 // Counting sort of the items by (KV head, decreasing cost).  Grouping by KV head keeps the CTAs that
 // run at the same time on the same K/V blocks (L2 reuse); sorting by cost inside a group lets the
 // dynamic hand-out start the long lists (PE heads) before the short ones (VS heads).
@@ -834,6 +844,7 @@ struct PrefillWs {
   int* cost_hist;
   int n_cost;  // distinct cost values (0 .. 2 N_b + 1)
   int n_bins;  // n_cost per KV head
+  size_t zero_bytes;  // header + histogram
   int32_t* merged;
 };
 
@@ -842,14 +853,16 @@ PrefillWs carve(const Dims& d, void* ws, size_t* total) {
   uint8_t* base = static_cast<uint8_t*>(ws);
   size_t off = kWsHeader;
   const int n_pairs = (d.nb + 1) / 2;
-  w.item_len = reinterpret_cast<int*>(base + off);
-  off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
-  w.order = reinterpret_cast<int*>(base + off);
-  off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
+  // the histogram sits directly behind the header: one memset clears both
   w.n_cost = 2 * d.nb + 2;
   w.n_bins = w.n_cost * d.hkv;
   w.cost_hist = reinterpret_cast<int*>(base + off);
   off += align_up(sizeof(int) * static_cast<size_t>(w.n_bins), 256);
+  w.zero_bytes = off;
+  w.item_len = reinterpret_cast<int*>(base + off);
+  off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
+  w.order = reinterpret_cast<int*>(base + off);
+  off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
   w.merged = reinterpret_cast<int32_t*>(base + off);
   off += align_up(sizeof(int32_t) * static_cast<size_t>(d.hq) * d.nb * (static_cast<size_t>(d.nb) + 1) / 2, 256);
   *total = off;
@@ -869,7 +882,8 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   const bool dense = (row_ptr == nullptr);
   size_t total;
   PrefillWs w = carve(d, ws, &total);
-  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "prefill: clear status");
+  // status word, item counter and (sparse) the schedule histogram
+  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, dense ? kWsHeader : w.zero_bytes, stream), "prefill: clear status");
   CUtensorMap tq, tk, tv;
   int rc = make_tmap_bf16_nhd(&tq, q, d.n, d.hq);
   if (rc == CRISP_OK) rc = make_tmap_bf16_nhd(&tk, k, d.n, d.hkv);
@@ -906,8 +920,8 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
     CRISP_KERNEL("prefill_dense", stream, prefill_kernel<true><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a));
   } else {
     const int words = (d.nb + 31) / 32;
-    CRISP_CUDA_TRY(cudaMemsetAsync(w.cost_hist, 0, sizeof(int) * w.n_bins, stream), "prefill: clear histogram");
-    CRISP_KERNEL("merge_lists", stream, merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words, stream>>>(
+    CRISP_KERNEL("merge_lists", stream, merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words,
+                                                       stream>>>(
         d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate, a.status,
         static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2));
     CRISP_KERNEL("sched_scan", stream, sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins));

@@ -7,9 +7,11 @@
 // and the sums of exp(logit - max) over the entries on/below the tile diagonal, above it, and on the
 // anchor keys.  Entries on/below the diagonal of key tile J belong to the diagonal band of block
 // offset N_b-1-J, entries above it to offset N_b-2-J, so these sums are all the later steps need.
-// The small kernels after it merge the partials: per-row global max and sum (`row_stats`,
-// `row_final`), per-tile masses across rows with warp-shuffle reductions (`tile_sums`) and the final
-// p_v, p_s, C_struct and routing label (`finalize`).  All reductions run in a fixed order.
+// Every row thread also carries the running maximum and sum of its row over the tiles its CTA visits; the
+// last CTA of a KV group to finish merges these per-CTA statistics into the global row maximum and
+// 1 / row sum.  One more kernel (`tile_sums_kernel`) turns the partials into per-tile masses across rows
+// with warp-shuffle reductions, and the last of its CTAs to finish a head adds up p_s and C_struct and
+// sets the routing label.  All reductions run in a fixed order.
 #include <cstdio>
 #include <mutex>
 
@@ -49,14 +51,18 @@ struct RoutePtrs {
   float* pup;      // [hq][nb][128] ... over entries with key offset > row
   float* phi;      // [hq][nb][128] third band, only when n is not a multiple of 128 (see proxy_partials_kernel)
   float* panc;     // [hq][slots][128] ... over anchor keys of the tile
-  float* cm;       // [hq][n_chunks][128] chunk max
-  float* cl;       // [hq][n_chunks][128] chunk sum relative to chunk max
+  float* cm;       // [hq][n_slices][128] row maximum over the tiles one proxy CTA visited
+  float* cl;       // [hq][n_slices][128] row sum relative to that maximum
   float* row_m;    // [hq][128] global row max
   float* row_invl; // [hq][128] 1 / global row sum
   float* slo;      // [hq][nb] mass (over rows) on/below the tile diagonal
   float* sup;      // [hq][nb] mass above the tile diagonal
   float* shi;      // [hq][nb] mass of the third band (ragged n only)
-  int n_chunks;
+  int* group_done; // [proxy grid.y] CTAs of a (KV head, head chunk) group that finished (zeroed per call)
+  int* head_done;  // [hq] CTAs of tile_sums that finished a head (zeroed per call)
+  size_t zero_bytes;  // header + counters
+  int n_chunks;    // chunks of kChunk key tiles (tile_sums)
+  int n_slices;    // proxy CTAs per group = entries of cm / cl per (head, row)
 };
 
 constexpr int kProxyHeads = 4;  // query heads of one KV group handled by one CTA (their proxy queries stay in shared memory)
@@ -69,6 +75,7 @@ struct ProxySmem {
   uint64_t bar_s_full[4], bar_s_free[4];
   uint32_t tmem_base;
   int abort_flag;
+  int is_last;
 };
 
 // Persistent CTAs, one per SM.  A CTA owns up to four query heads of one KV group - their 128 proxy queries
@@ -184,6 +191,8 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     const int my_jobs = gr ? jobs1 : jobs0;
     int job = 0;
     bool ok = true;
+    // running maximum and sum of this row over the CTA's tiles, per head of the group (two at most)
+    float run_m[2] = {-INFINITY, -INFINITY}, run_l[2] = {0.f, 0.f};
     for (int n = 0; n < n_my_tiles && ok; ++n) {
       const int J = blockIdx.x + n * stride;
       const int qoff = d.nfull - 1 - J;
@@ -304,6 +313,12 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
           }
         }
         if (!any) lo = up = hi = anc = 0.f;
+        {
+          const float sum = lo + up + hi;
+          const float nm = fmaxf(run_m[gj & 1], mx);
+          run_l[gj & 1] = run_l[gj & 1] * ex2(run_m[gj & 1] - nm) + sum * ex2(mx - nm);
+          run_m[gj & 1] = nm;
+        }
         const int h = kvh * G + g0 + g;
         const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
         w.pm[off] = mx;
@@ -313,46 +328,40 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
       }
     }
+    // this CTA's share of the row statistics
+    for (int gj = 0; gj < my_jobs; ++gj) {
+      const int h = kvh * G + g0 + 2 * gj + gr;
+      const size_t o = (static_cast<size_t>(h) * w.n_slices + blockIdx.x) * kBlock + i;
+      w.cm[o] = run_m[gj];
+      w.cl[o] = run_l[gj];
+    }
   }
   tc_fence_before_sync();
+  __threadfence();
   __syncthreads();
-  if (tid == 0 && s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
+  if (tid == 0) {
+    if (s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
+    s.is_last = atomicAdd(&w.group_done[blockIdx.y], 1) == static_cast<int>(gridDim.x) - 1;
+  }
   if (warp == 8) tmem_dealloc(tm, 512);
-}
-
-// Per (head, chunk of tiles): running max and sum of every proxy row over the chunk's tiles.
-__global__ void __launch_bounds__(128) row_stats_kernel(const Dims d, const RoutePtrs w) {
-  const int h = blockIdx.y, chunk = blockIdx.x, i = threadIdx.x;
-  const int j0 = chunk * kChunk, j1 = min(j0 + kChunk, d.nb);
-  float M = -INFINITY, L = 0.f;
-  const size_t base = static_cast<size_t>(h) * d.nb * kBlock + i;
-#pragma unroll 4
-  for (int J = j0; J < j1; ++J) {
-    const size_t off = base + static_cast<size_t>(J) * kBlock;
-    const float m = w.pm[off];
-    const float sum = w.plo[off] + w.pup[off] + (d.rho > 0 ? w.phi[off] : 0.f);
-    const float nm = fmaxf(M, m);
-    L = L * ex2(M - nm) + sum * ex2(m - nm);
-    M = nm;
+  __syncthreads();
+  if (!s.is_last) return;
+  // The last CTA of the group to finish merges the per-CTA statistics (written by other CTAs: read from L2)
+  // into the global row maximum and 1 / row sum of the group's heads.
+  __threadfence();
+  for (int item = tid; item < gc * kBlock; item += blockDim.x) {
+    const int h = kvh * G + g0 + item / kBlock, i = item % kBlock;
+    float M = -INFINITY, L = 0.f;
+    for (int c = 0; c < static_cast<int>(gridDim.x); ++c) {
+      const size_t o = (static_cast<size_t>(h) * w.n_slices + c) * kBlock + i;
+      const float m = __ldcg(w.cm + o), l = __ldcg(w.cl + o);
+      const float nm = fmaxf(M, m);
+      L = L * ex2(M - nm) + l * ex2(m - nm);
+      M = nm;
+    }
+    w.row_m[h * kBlock + i] = M;
+    w.row_invl[h * kBlock + i] = 1.0f / L;
   }
-  const size_t o = (static_cast<size_t>(h) * w.n_chunks + chunk) * kBlock + i;
-  w.cm[o] = M;
-  w.cl[o] = L;
-}
-
-// Per head: merge the chunk statistics into the global row max and 1 / row sum.
-__global__ void __launch_bounds__(128) row_final_kernel(const Dims d, const RoutePtrs w) {
-  const int h = blockIdx.x, i = threadIdx.x;
-  float M = -INFINITY, L = 0.f;
-  for (int c = 0; c < w.n_chunks; ++c) {
-    const size_t o = (static_cast<size_t>(h) * w.n_chunks + c) * kBlock + i;
-    const float m = w.cm[o], l = w.cl[o];
-    const float nm = fmaxf(M, m);
-    L = L * ex2(M - nm) + l * ex2(m - nm);
-    M = nm;
-  }
-  w.row_m[h * kBlock + i] = M;
-  w.row_invl[h * kBlock + i] = 1.0f / L;
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -361,10 +370,14 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// Per (head, chunk): one warp per key tile sums the normalised masses over the 128 proxy rows.
-__global__ void __launch_bounds__(128) tile_sums_kernel(const Dims d, const RoutePtrs w, float* __restrict__ p_v) {
+// Per (head, chunk): one warp per key tile sums the normalised masses over the 128 proxy rows.  The last CTA of
+// a head to finish then forms the slash scores from the two (three) triangle sums, C_struct from the anchor
+// partials, and the routing label.
+__global__ void __launch_bounds__(128) tile_sums_kernel(const Dims d, const RoutePtrs w, float* __restrict__ p_v,
+                                                        float* __restrict__ p_s, float* __restrict__ c_struct,
+                                                        int32_t* __restrict__ pattern) {
   const int h = blockIdx.y, chunk = blockIdx.x;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   float M[4], invl[4];
 #pragma unroll
   for (int r = 0; r < 4; ++r) {
@@ -392,12 +405,15 @@ __global__ void __launch_bounds__(128) tile_sums_kernel(const Dims d, const Rout
       p_v[static_cast<size_t>(h) * d.nb + J] = (lo + up) + hi;
     }
   }
-}
-
-// Per head: slash scores from the two triangle sums, C_struct from the anchor partials, routing label.
-__global__ void __launch_bounds__(256) finalize_kernel(const Dims d, const RoutePtrs w, float* __restrict__ p_s,
-                                                       float* __restrict__ c_struct, int32_t* __restrict__ pattern) {
-  const int h = blockIdx.x, tid = threadIdx.x;
+  __shared__ int is_last;
+  __shared__ float red[4];
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = atomicAdd(&w.head_done[h], 1) == static_cast<int>(gridDim.x) - 1;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // ---- the head's last CTA.  The tile sums came from other CTAs: read them from L2.
   const float* slo = w.slo + static_cast<size_t>(h) * d.nb;
   const float* sup = w.sup + static_cast<size_t>(h) * d.nb;
   const float* shi = w.shi + static_cast<size_t>(h) * d.nb;
@@ -405,23 +421,22 @@ __global__ void __launch_bounds__(256) finalize_kernel(const Dims d, const Route
   for (int sidx = tid; sidx < d.nb; sidx += blockDim.x) {
     const int jlo = d.nfull - 1 - sidx, jup = d.nfull - 2 - sidx, jhi = d.nfull - sidx;
     float v = 0.f;
-    if (jlo >= 0 && jlo < d.nb) v += slo[jlo];
-    if (jup >= 0 && jup < d.nb) v += sup[jup];
-    if (d.rho > 0 && jhi >= 0 && jhi < d.nb) v += shi[jhi];
+    if (jlo >= 0 && jlo < d.nb) v += __ldcg(slo + jlo);
+    if (jup >= 0 && jup < d.nb) v += __ldcg(sup + jup);
+    if (d.rho > 0 && jhi >= 0 && jhi < d.nb) v += __ldcg(shi + jhi);
     p_s[static_cast<size_t>(h) * d.nb + sidx] = v;
   }
-  __shared__ float red[4];
   float acc = 0.f;
-  if (tid < kBlock) {
-    const float M = w.row_m[h * kBlock + tid];
-    const float invl = w.row_invl[h * kBlock + tid] * (1.0f / kBlock);
+  {
+    const float Mr = w.row_m[h * kBlock + tid];
+    const float inv = w.row_invl[h * kBlock + tid] * (1.0f / kBlock);
     for (int slot = 0; slot < d.n_anchor_slots; ++slot) {
       const int J = slot < d.n_sink_tiles ? slot : d.first_local_tile + (slot - d.n_sink_tiles);
       const float m = w.pm[(static_cast<size_t>(h) * d.nb + J) * kBlock + tid];
-      acc += ex2(m - M) * invl * w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + tid];
+      acc += ex2(m - Mr) * inv * w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + tid];
     }
     acc = warp_sum(acc);
-    if ((tid & 31) == 0) red[tid >> 5] = acc;
+    if (lane == 0) red[warp] = acc;
   }
   __syncthreads();
   if (tid == 0) {
@@ -434,6 +449,24 @@ __global__ void __launch_bounds__(256) finalize_kernel(const Dims d, const Route
   }
 }
 
+// How the proxy kernel's grid is laid out: one CTA per SM; the (KV head, chunk of four query heads) groups share
+// the SMs evenly, each group's CTAs split its key tiles.
+struct ProxyGrid {
+  int n_head_chunks, groups, slices;
+};
+ProxyGrid proxy_grid(const Dims& d, int n_sm) {
+  ProxyGrid g;
+  g.n_head_chunks = (d.group + kProxyHeads - 1) / kProxyHeads;
+  g.groups = d.hkv * g.n_head_chunks;
+  g.slices = n_sm / g.groups;
+  if (g.slices < 1) g.slices = 1;
+  if (g.slices > d.nb) g.slices = d.nb;
+  return g;
+}
+// The workspace is sized without knowing the device: room for the CTAs of a 160-SM part; a larger device simply
+// runs with that many CTAs per group.
+constexpr int kSizedForSms = 160;
+
 RoutePtrs carve(const Dims& d, void* ws) {
   RoutePtrs w;
   uint8_t* p = static_cast<uint8_t*>(ws) + kWsHeader;
@@ -442,15 +475,21 @@ RoutePtrs carve(const Dims& d, void* ws) {
     p += align_up(n_floats * sizeof(float), 256);
     return r;
   };
+  // counters first: one memset clears them together with the header
+  const int n_head_chunks = (d.group + kProxyHeads - 1) / kProxyHeads;
+  w.group_done = reinterpret_cast<int*>(take(static_cast<size_t>(d.hkv) * n_head_chunks));
+  w.head_done = reinterpret_cast<int*>(take(d.hq));
+  w.zero_bytes = static_cast<size_t>(p - static_cast<uint8_t*>(ws));
   w.n_chunks = (d.nb + kChunk - 1) / kChunk;
+  w.n_slices = max(1, min(kSizedForSms / (d.hkv * n_head_chunks), d.nb));
   const size_t part = static_cast<size_t>(d.hq) * d.nb * kBlock;
   w.pm = take(part);
   w.plo = take(part);
   w.pup = take(part);
   w.phi = d.rho > 0 ? take(part) : nullptr;  // third band: only for lengths that are not multiples of 128
   w.panc = take(static_cast<size_t>(d.hq) * d.n_anchor_slots * kBlock);
-  w.cm = take(static_cast<size_t>(d.hq) * w.n_chunks * kBlock);
-  w.cl = take(static_cast<size_t>(d.hq) * w.n_chunks * kBlock);
+  w.cm = take(static_cast<size_t>(d.hq) * w.n_slices * kBlock);
+  w.cl = take(static_cast<size_t>(d.hq) * w.n_slices * kBlock);
   w.row_m = take(static_cast<size_t>(d.hq) * kBlock);
   w.row_invl = take(static_cast<size_t>(d.hq) * kBlock);
   w.slo = take(static_cast<size_t>(d.hq) * d.nb);
@@ -470,7 +509,7 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
                  float* p_v, float* p_s, cudaStream_t stream) {
   RoutePtrs w = carve(d, ws);
   int* status = static_cast<int*>(ws);
-  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "route: clear status");
+  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, stream), "route: clear status and counters");
   CUtensorMap tq, tk;
   int rc = make_tmap_bf16_nhd(&tq, q, d.n, d.hq);
   if (rc != CRISP_OK) return rc;
@@ -480,21 +519,13 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   auto* proxy = d.rho > 0 ? proxy_partials_kernel<true> : proxy_partials_kernel<false>;
   CRISP_CUDA_TRY(cudaFuncSetAttribute(proxy, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)),
                  "route: smem attribute");
-  // one CTA per SM: the (KV head, chunk of four query heads) groups share the SMs evenly, each group's CTAs
-  // split its key tiles
   int dev = 0, n_sm = 0;
   CRISP_CUDA_TRY(cudaGetDevice(&dev), "route: current device");
   CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "route: SM count");
-  const int n_head_chunks = (d.group + kProxyHeads - 1) / kProxyHeads;
-  const int groups = d.hkv * n_head_chunks;
-  int slices = n_sm / groups;
-  if (slices < 1) slices = 1;
-  if (slices > d.nb) slices = d.nb;
-  CRISP_KERNEL("proxy", stream, proxy<<<dim3(slices, groups), 288, smem, stream>>>(tq, tk, d, w, status, n_head_chunks));
-  CRISP_KERNEL("row_stats", stream, row_stats_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w));
-  CRISP_KERNEL("row_final", stream, row_final_kernel<<<d.hq, 128, 0, stream>>>(d, w));
-  CRISP_KERNEL("tile_sums", stream, tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v));
-  CRISP_KERNEL("finalize", stream, finalize_kernel<<<d.hq, 256, 0, stream>>>(d, w, p_s, c_struct, pattern));
+  ProxyGrid g = proxy_grid(d, n_sm);
+  if (g.slices > w.n_slices) g.slices = w.n_slices;
+  CRISP_KERNEL("proxy", stream, proxy<<<dim3(g.slices, g.groups), 288, smem, stream>>>(tq, tk, d, w, status, g.n_head_chunks));
+  CRISP_KERNEL("tile_sums", stream, tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v, p_s, c_struct, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route: launch");
   return CRISP_OK;
 }

@@ -1,18 +1,25 @@
 // Stage 3b-3c: block selection and expansion into per-query-block key-block lists.
 //
 //   VS heads  (Algorithm 3 lines 6-12 / Eq. 3-4; Algorithm 6 when selector == 1; the median floor of
-//     Appendix H when selector == 2):
-//     `select_vs_kernel`, one CTA per (head, direction), keeps p_d in shared memory, computes the
-//     noise floor, the budget k_d and the top-k_d set (ties to the lower index) as a bitmap.
-//   PE heads  (Algorithm 4): block means of Q and K (`pool_kernel`), pooled logits (`pe_logits_kernel`),
-//     causal row softmax normalised by the total (`pe_normalise_kernel`), then the gamma cut WITHOUT a
-//     sort: a three-level radix histogram over the fp32 bit patterns (`pe_hist_kernel`,
-//     `pe_cut_kernel`), with masses in exact fixed point, finds the value at the cut and how many
-//     entries tied with it are taken (ties in row-major order).
-//   Expansion + compaction: per (head, query block) a bitmap over key blocks is formed from the
-//     vertical bitmap, the shifted slash bitmap and the forced blocks {0, m}; popcounts give the row
-//     lengths (`count_vs_kernel`), one scan gives row_ptr (`scan_rows_kernel`), a second pass writes the
-//     ascending column lists (`fill_kernel`).  No atomics touch the lists, so they are reproducible.
+//     Appendix H when selector == 2): `prepare_kernel`, one CTA per head, keeps p_d in shared memory,
+//     computes the noise floor, the budget k_d and the top-k_d set (ties to the lower index) of both
+//     directions as bitmaps, then the length of every query block's list (popcounts of the vertical
+//     bitmap, the shifted slash bitmap and the forced blocks {0, m}) and their prefix sum inside the head.
+//     The other CTAs of the same launch compute the block means of Q and K that the PE heads need.
+//   PE heads  (Algorithm 4): pooled logits on the tensor cores (`pe_logits_kernel`), which also leaves the
+//     row maximum and 1 / (row sum * N_b) of every row, so the causal row softmax divided by the total is
+//     never written: every later pass recomputes an entry as 2^(z - max) * inv from the stored logit.  The
+//     gamma cut is found WITHOUT a sort by a three-level radix histogram (8 + 12 + 11 bits) over the fp32 bit patterns of
+//     those values (`pe_hist_kernel<level>`, masses in exact fixed point; the last CTA of a head to finish
+//     a level locates the cut in it), which yields the value at the cut and how many entries tied with it
+//     are taken (ties in row-major order).  The last level also counts, per row, the entries above the
+//     cut's bin; `pe_rows_kernel` re-reads only the rows that have entries inside that bin, distributes the
+//     ties and scans the row lengths of the head.
+//   `fill_kernel` adds the heads' totals up to global offsets, writes row_ptr and the ascending column
+//     lists.  No atomics touch the lists, and the histograms add integers, so everything is reproducible.
+//
+// Passes over the pooled map (4 N_b^2 / 2 bytes per PE head): one write (logits), three reads (histogram
+// levels), one read (fill); rows holding entries in the cut's last bin are read once more (a few).
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -21,8 +28,18 @@ using namespace sm100;
 
 namespace {
 
-constexpr int kL0Bins = 2048, kL1Bins = 2048, kL2Bins = 512;  // key bits 30..20, 19..9, 8..0
+// Radix levels over the fp32 bit pattern of a (positive) value: the exponent (key bits 30..23), then twelve and
+// eleven mantissa bits (22..11, 10..0).  Level 0 sees every entry, and a row's entries share two or three
+// exponents, so its few bins are fed through warp-wide sums; the lower levels see only the entries inside the
+// cut's bin, spread over thousands of bins.
+constexpr int kL0Bins = 256, kL1Bins = 4096, kL2Bins = 2048;
+constexpr int kL0Shift = 23, kL1Shift = 11;
 constexpr int kHistStride = kL0Bins + kL1Bins + kL2Bins;
+constexpr int kHistThreads = 512;
+constexpr int kMaxBins = 4096;
+__host__ __device__ constexpr int level_bins(int level) { return level == 0 ? kL0Bins : (level == 1 ? kL1Bins : kL2Bins); }
+__host__ __device__ constexpr int level_offset(int level) { return level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins); }
+__host__ __device__ constexpr int level_shift(int level) { return level == 0 ? kL0Shift : (level == 1 ? kL1Shift : 0); }
 
 // Masses are accumulated in 2^-60 fixed point: integer adds are exact and order independent, so the
 // histograms (built with atomics) and everything derived from them are reproducible.
@@ -36,21 +53,29 @@ struct CutState {                 // per head, device memory
 };
 
 struct SelectPtrs {
+  // ---- zeroed at the start of every call (one contiguous region)
+  unsigned int* hcount;        // [hq][kHistStride]
+  unsigned long long* hmass;   // [hq][kHistStride] fixed-point mass per bin
+  int* hist_done;              // [3][hq] CTAs of a head that finished a histogram level
+  int* rows_done;              // [hq]   CTAs of a head that finished pe_rows
+  size_t zero_bytes;
+  // ---- written before read
   uint32_t* selv;   // [hq][words] vertical bitmap
   uint32_t* selsr;  // [hq][words + 2] reversed slash bitmap: bit x = S_s contains N_b-1-x
   float* kbar;      // [hkv][nb][128]
   float* qbar;      // [hq][nb][128]
   __nv_bfloat16* ksplit;  // [3][nb][hkv][128] block means of K as three bf16 terms (hi + mid + lo = the fp32 mean)
   __nv_bfloat16* qsplit;  // [3][nb][hq][128]  the same for Q
-  float* amat;      // [hq][nb][nb] pooled map (row m uses columns 0..m)
-  unsigned int* hcount;  // [hq][kHistStride]
-  unsigned long long* hmass;  // [hq][kHistStride] fixed-point mass per bin
-  CutState* cut;         // [hq]
-  int* n_gt;        // [hq][nb]
-  int* n_eq;        // [hq][nb]
-  int* flags;       // [hq][nb] bit0: a[m][0] > cut, bit1: == cut, bit2: a[m][m] > cut, bit3: == cut
-  int* take;        // [hq][nb] ties of row m that are selected
+  float* amat;      // [hq][nb][nb] pooled logits in base-2 units (row m uses columns 0..m)
+  float* row_m;     // [hq][nb] row maximum of the pooled logits
+  float* row_inv;   // [hq][nb] 1 / (sum_J 2^(z - max) * N_b)
+  CutState* cut;    // [hq]
+  int* n_gt;        // [hq][nb] entries above the cut (first: above the cut's last bin)
+  int* n_eq;        // [hq][nb] entries inside the cut's last bin, then: entries tied with the cut
   int* counts;      // [hq][nb] row lengths
+  int* take;        // [hq][nb] ties of row m that are selected
+  int* local_off;   // [hq][nb] exclusive prefix sum of the row lengths inside the head
+  long long* head_total;  // [hq] entries of the head's lists
   int words;
 };
 
@@ -74,34 +99,83 @@ __device__ T block_sum(T v, T* scratch /* >= 32 */) {
   return total;
 }
 
-// ------------------------------------------------------------------------------------------------
-// VS heads: budget and top-k per direction
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024)
-select_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const float* __restrict__ p_v,
-                 const float* __restrict__ p_s, const SelectPtrs w) {
-  extern __shared__ uint8_t sm_raw[];
-  const int nb = d.nb;
-  double* sorted = reinterpret_cast<double*>(sm_raw);  // [nb] values in descending order (gamma rule)
-  float* p = reinterpret_cast<float*>(sorted + nb);    // [nb]
-  int* ranks = reinterpret_cast<int*>(p + nb);         // [nb]
-  uint8_t* sel = reinterpret_cast<uint8_t*>(ranks + nb);  // [nb]
-  __shared__ float fscratch[32];
-  __shared__ int iscratch[32];
-  __shared__ int s_k;
-  __shared__ float s_med[2];
-  const int h = blockIdx.x, dir = blockIdx.y, tid = threadIdx.x;
-  uint32_t* out = dir == 0 ? w.selv + static_cast<size_t>(h) * w.words
-                           : w.selsr + static_cast<size_t>(h) * (w.words + 2);
-  const int out_words = dir == 0 ? w.words : w.words + 2;
-  if (pattern[h] != CRISP_PATTERN_VS) {
-    for (int i = tid; i < out_words; i += blockDim.x) out[i] = 0u;
-    return;
+// Word `wd` (key blocks 32*wd .. 32*wd+31) of the keep bitmap of query block m of a VS head.
+__device__ __forceinline__ uint32_t vs_keep_word(const uint32_t* __restrict__ selv, const uint32_t* __restrict__ selsr,
+                                                 int nb, int m, int wd) {
+  const int sh = nb - 1 - m;              // slash offset s = m - J  <->  reversed bit J + sh
+  const int pos0 = wd * 32 + sh, pos1 = pos0 + 1;
+  const uint32_t a = __funnelshift_r(selsr[pos0 >> 5], selsr[(pos0 >> 5) + 1], pos0 & 31);
+  const uint32_t b = __funnelshift_r(selsr[pos1 >> 5], selsr[(pos1 >> 5) + 1], pos1 & 31);
+  uint32_t bits = selv[wd] | a | b;
+  if (wd == 0) bits |= 1u;
+  if (wd == (m >> 5)) {
+    bits |= 1u << (m & 31);
+    const int top = m & 31;
+    bits &= (top == 31) ? 0xffffffffu : ((2u << top) - 1u);
   }
-  const float* src = (dir == 0 ? p_v : p_s) + static_cast<size_t>(h) * nb;
+  return bits;
+}
+
+// ------------------------------------------------------------------------------------------------
+// First launch: CTAs [0, hq) select the blocks of the VS heads and size their lists; the remaining CTAs
+// pool Q and K for the PE heads.
+// ------------------------------------------------------------------------------------------------
+// Block means of eight [128 tokens, 128 dims] tiles per CTA (128 threads per tile).  x is [n, heads, 128] bf16.
+__device__ __forceinline__ void pool_tile(const Dims& d, const __nv_bfloat16* __restrict__ x, int heads, int J, int h,
+                                          int tid, float* __restrict__ out, __nv_bfloat16* __restrict__ split,
+                                          float2* other /* [64] shared */, int bar_id) {
+  const int pair = tid & 63, half = tid >> 6;
+  const __nv_bfloat162* base = reinterpret_cast<const __nv_bfloat162*>(
+      x + (static_cast<size_t>(J) * kBlock + half * 64) * heads * kHeadDim + static_cast<size_t>(h) * kHeadDim);
+  float a0 = 0.f, a1 = 0.f;
+  // the last block may hold fewer than 128 tokens: rows at or beyond n are not read
+  const int valid = min(kBlock, d.n - J * kBlock);
+  const int rows = min(max(valid - half * 64, 0), 64);
+  if (rows == 64) {
+    // full half block: a fixed trip count keeps all 64 loads of a thread in flight
+#pragma unroll
+    for (int t = 0; t < 64; ++t) {
+      const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
+      a0 += v.x;
+      a1 += v.y;
+    }
+  } else {
+    for (int t = 0; t < rows; ++t) {
+      const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
+      a0 += v.x;
+      a1 += v.y;
+    }
+  }
+  if (half == 1) other[pair] = make_float2(a0, a1);
+  named_bar_sync(bar_id, 128);
+  if (half == 0) {
+    float* o = out + (static_cast<size_t>(h) * d.nb + J) * kHeadDim;
+    const float inv = 1.0f / static_cast<float>(valid);
+    const float m0 = (a0 + other[pair].x) * inv, m1 = (a1 + other[pair].y) * inv;
+    o[2 * pair] = m0;
+    o[2 * pair + 1] = m1;
+    if (split != nullptr) {
+      // mean = hi + mid + lo with three bf16 terms (the remainders are exact in fp32): the pooled logits are
+      // then a sum of bf16 tensor-core products that reproduces the fp32 product to ~2^-24
+      float r0 = m0, r1 = m1;
+#pragma unroll
+      for (int pl = 0; pl < 3; ++pl) {
+        const __nv_bfloat162 t = __floats2bfloat162_rn(r0, r1);
+        reinterpret_cast<__nv_bfloat162*>(split + ((static_cast<size_t>(pl) * d.nb + J) * heads + h) * kHeadDim)[pair] = t;
+        r0 -= __low2float(t);
+        r1 -= __high2float(t);
+      }
+    }
+  }
+}
+
+// Budget and top-k of one direction of a VS head (Algorithm 3 / Algorithm 6 / Appendix H) as a bitmap.
+__device__ void select_direction(const Dims& d, const float* __restrict__ src, int dir, uint32_t* __restrict__ out,
+                                 int out_words, double* sorted, float* p, int* ranks, uint8_t* sel, float* fscratch,
+                                 int* iscratch, int* s_k, float* s_med) {
+  const int nb = d.nb, tid = threadIdx.x;
   for (int i = tid; i < nb; i += blockDim.x) p[i] = src[i];
   __syncthreads();
-
   bool need_rank = false;
   int k = nb;
   float thr = -1.f;  // N_b <= 2: every block is kept
@@ -171,10 +245,10 @@ select_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const float*
             break;
           }
         }
-        s_k = min(max(found, d.k_min), nb);
+        *s_k = min(max(found, d.k_min), nb);
       }
       __syncthreads();
-      k = s_k;
+      k = *s_k;
     }
     for (int e = tid; e < nb; e += blockDim.x) sel[e] = ranks[e] < k;
   }
@@ -191,292 +265,330 @@ select_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const float*
     }
     out[wd] = bits;
   }
-}
-
-// ------------------------------------------------------------------------------------------------
-// PE heads: pooling, pooled logits, row softmax
-// ------------------------------------------------------------------------------------------------
-// Block means of one [128 tokens, 128 dims] tile per CTA.  x is [n, heads, 128] bf16.
-__global__ void __launch_bounds__(128)
-pool_kernel(const Dims d, const __nv_bfloat16* __restrict__ x, int heads, int is_query,
-            const int32_t* __restrict__ pattern, float* __restrict__ out, __nv_bfloat16* __restrict__ split) {
-  const int J = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
-  if (pattern == nullptr) {
-    // comparison router: every head's block means are wanted
-  } else if (is_query) {
-    if (pattern[h] != CRISP_PATTERN_PE) return;
-  } else {
-    bool any = false;
-    for (int g = 0; g < d.group; ++g) any = any || (pattern[h * d.group + g] == CRISP_PATTERN_PE);
-    if (!any) return;
-  }
-  const int pair = tid & 63, half = tid >> 6;
-  const __nv_bfloat162* base = reinterpret_cast<const __nv_bfloat162*>(
-      x + (static_cast<size_t>(J) * kBlock + half * 64) * heads * kHeadDim + static_cast<size_t>(h) * kHeadDim);
-  float a0 = 0.f, a1 = 0.f;
-  // the last block may hold fewer than 128 tokens: rows at or beyond n are not read
-  const int valid = min(kBlock, d.n - J * kBlock);
-  const int rows = min(max(valid - half * 64, 0), 64);
-  if (rows == 64) {
-    // full half block: a fixed trip count keeps all 64 loads of a thread in flight
-#pragma unroll
-    for (int t = 0; t < 64; ++t) {
-      const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
-      a0 += v.x;
-      a1 += v.y;
-    }
-  } else {
-    for (int t = 0; t < rows; ++t) {
-      const float2 v = __bfloat1622float2(base[static_cast<size_t>(t) * heads * (kHeadDim / 2) + pair]);
-      a0 += v.x;
-      a1 += v.y;
-    }
-  }
-  __shared__ float2 other[64];
-  if (half == 1) other[pair] = make_float2(a0, a1);
   __syncthreads();
-  if (half == 0) {
-    float* o = out + (static_cast<size_t>(h) * d.nb + J) * kHeadDim;
-    const float inv = 1.0f / static_cast<float>(valid);
-    const float m0 = (a0 + other[pair].x) * inv, m1 = (a1 + other[pair].y) * inv;
-    o[2 * pair] = m0;
-    o[2 * pair + 1] = m1;
-    if (split != nullptr) {
-      // mean = hi + mid + lo with three bf16 terms (the remainders are exact in fp32): the pooled logits are
-      // then a sum of bf16 tensor-core products that reproduces the fp32 product to ~2^-24
-      float r0 = m0, r1 = m1;
-#pragma unroll
-      for (int pl = 0; pl < 3; ++pl) {
-        const __nv_bfloat162 t = __floats2bfloat162_rn(r0, r1);
-        reinterpret_cast<__nv_bfloat162*>(split + ((static_cast<size_t>(pl) * d.nb + J) * heads + h) * kHeadDim)[pair] = t;
-        r0 -= __low2float(t);
-        r1 -= __high2float(t);
-      }
-    }
-  }
 }
 
-// Pooled logits Z[m, J] = qbar[m] . kbar[J] * scale_log2, one 128 x 128 tile of (query block, key block) pairs per
-// CTA, on the tensor cores.  The selection compares these values, so bf16 operands alone would not do: each fp32
-// block mean is split into three bf16 terms (pool_kernel), and the six products hi*hi, hi*mid, mid*hi, mid*mid,
-// hi*lo, lo*hi - accumulated in fp32 in TMEM, smallest first - reproduce the fp32 dot product to ~2^-24.
+__global__ void __launch_bounds__(1024)
+prepare_kernel(const Dims d, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
+               const int32_t* __restrict__ pattern, const float* __restrict__ p_v, const float* __restrict__ p_s,
+               const SelectPtrs w, int vs_ctas, int pool_all_k) {
+  extern __shared__ uint8_t sm_raw[];
+  const int tid = threadIdx.x;
+  if (static_cast<int>(blockIdx.x) >= vs_ctas) {
+    // ---------------- pooling: eight (block, head) tiles per CTA; heads [0, hkv) are K, the rest Q
+    __shared__ float2 other[8][64];
+    const int sub = tid >> 7, t = tid & 127;
+    const long long tile = (static_cast<long long>(blockIdx.x) - vs_ctas) * 8 + sub;
+    const long long n_tiles = static_cast<long long>(d.nb) * (d.hkv + d.hq);
+    if (tile >= n_tiles) return;  // whole 128-thread groups leave together
+    const int hh = static_cast<int>(tile / d.nb), J = static_cast<int>(tile % d.nb);
+    if (hh < d.hkv) {
+      bool any = pool_all_k != 0;
+      for (int g = 0; g < d.group && !any; ++g) any = pattern[hh * d.group + g] == CRISP_PATTERN_PE;
+      if (!any) return;
+      pool_tile(d, k, d.hkv, J, hh, t, w.kbar, w.ksplit, other[sub], 1 + sub);
+    } else {
+      const int h = hh - d.hkv;
+      if (pattern == nullptr || pattern[h] != CRISP_PATTERN_PE) return;
+      pool_tile(d, q, d.hq, J, h, t, w.qbar, w.qsplit, other[sub], 1 + sub);
+    }
+    return;
+  }
+  // ---------------- VS head: both directions, then the lengths of its lists
+  const int h = blockIdx.x, nb = d.nb;
+  if (pattern[h] != CRISP_PATTERN_VS) return;
+  double* sorted = reinterpret_cast<double*>(sm_raw);  // [nb] values in descending order (gamma rule)
+  float* p = reinterpret_cast<float*>(sorted + nb);    // [nb]
+  int* ranks = reinterpret_cast<int*>(p + nb);         // [nb]
+  uint8_t* sel = reinterpret_cast<uint8_t*>(ranks + nb);  // [nb]
+  __shared__ float fscratch[32];
+  __shared__ int iscratch[32];
+  __shared__ long long lscratch[33];
+  __shared__ int s_k;
+  __shared__ float s_med[2];
+  uint32_t* selv = w.selv + static_cast<size_t>(h) * w.words;
+  uint32_t* selsr = w.selsr + static_cast<size_t>(h) * (w.words + 2);
+  select_direction(d, p_v + static_cast<size_t>(h) * nb, 0, selv, w.words, sorted, p, ranks, sel, fscratch, iscratch,
+                   &s_k, s_med);
+  select_direction(d, p_s + static_cast<size_t>(h) * nb, 1, selsr, w.words + 2, sorted, p, ranks, sel, fscratch,
+                   iscratch, &s_k, s_med);
+  // the bitmaps were written by this CTA; the barrier at the end of select_direction makes them visible to it
+  const int seg = (nb + 1023) / 1024;
+  const int b0 = min(tid * seg, nb), b1 = min(b0 + seg, nb);
+  const size_t base = static_cast<size_t>(h) * nb;
+  long long local = 0;
+  for (int m = b0; m < b1; ++m) {
+    int c = 0;
+    for (int wd = 0; wd <= (m >> 5); ++wd) c += __popc(vs_keep_word(selv, selsr, nb, m, wd));
+    w.counts[base + m] = c;
+    local += c;
+  }
+  long long total;
+  long long run = block_exclusive_scan_1024(local, lscratch, &total);
+  for (int m = b0; m < b1; ++m) {
+    w.local_off[base + m] = static_cast<int>(run);
+    run += w.counts[base + m];
+  }
+  if (tid == 0) w.head_total[h] = total;
+}
+
+// ------------------------------------------------------------------------------------------------
+// PE heads: pooled logits on the tensor cores
+// ------------------------------------------------------------------------------------------------
+// Z[m, J] = qbar[m] . kbar[J] * scale * log2(e).  The selection compares these values, so bf16 operands alone
+// would not do: each fp32 block mean is split into three bf16 terms (pool_tile), and the six products hi*hi,
+// hi*mid, mid*hi, mid*mid, hi*lo, lo*hi - accumulated in fp32 in TMEM - reproduce the fp32 dot product to ~2^-24.
+//
+// Persistent CTAs.  A work item is one PE head and one strip of 128 query blocks (rows m); the strip's three
+// operand terms stay in shared memory while the CTA walks over the strip's key tiles jt = 0 .. mt.  The K-side
+// operands arrive in two halves of 64 dims (two 48 KB slots): while the MMAs of one half run, the other slot is
+// refilled for the next tile.  Two TMEM accumulators and two groups of four epilogue warps (one thread per row;
+// group 0 drains the even tiles of an item, group 1 the odd ones) keep the MMAs of tile t + 1 running while tile
+// t is drained.  A strip holds complete rows, so the epilogue threads carry the running maximum and sum of their
+// row across their tiles and leave the row's softmax normalisers at the end of the item; the normalised map
+// itself is never written.
 struct LogitsMaps {
   CUtensorMap q[3], k[3];
 };
 struct LogitsSmem {
   alignas(1024) uint8_t a[3][2][16384];  // [term][64-dim half] 128 block means of Q, 128-byte swizzle
-  alignas(1024) uint8_t b[3][2][16384];  // the same for K
-  uint64_t bar_in, bar_mma;
+  alignas(1024) uint8_t b[2][3][16384];  // [64-dim half = slot][term] 128 block means of K
+  uint64_t bar_a_full, bar_a_free;
+  uint64_t bar_b_full[2], bar_b_free[2];
+  uint64_t bar_acc_full[2], bar_acc_free[2];
   uint32_t tmem_base;
   int abort_flag;
+  int n_pe;
+  float2 row_state[kBlock];  // (running maximum, running sum) of the rows' odd tiles, handed to the even tiles' threads
+  int pe_heads[1024];
 };
 
-__global__ void __launch_bounds__(160)
+// Item `idx` of CTA `cta`: positions of the size-sorted order (long strips first) are dealt out in rounds of
+// gridDim.x, alternating direction, so every CTA gets a similar number of tiles.
+__device__ __forceinline__ bool logits_item(int round, int cta, int n_cta, int n_items, int n_pe, int nt, int* h_slot,
+                                            int* mt) {
+  const int i = (round & 1) ? (n_cta - 1 - cta) : cta;
+  const int pos = round * n_cta + i;
+  if (pos >= n_items) return false;
+  *mt = nt - 1 - pos / n_pe;
+  *h_slot = pos % n_pe;
+  return true;
+}
+
+__global__ void __launch_bounds__(288, 1)
 pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const int32_t* __restrict__ pattern,
                  const SelectPtrs w, int* status) {
-  const int jt = blockIdx.x, mt = blockIdx.y, h = blockIdx.z;
-  if (jt > mt || pattern[h] != CRISP_PATTERN_PE) return;
   extern __shared__ uint8_t smem_raw[];
   LogitsSmem& s = *reinterpret_cast<LogitsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     s.abort_flag = 0;
-    mbar_init(&s.bar_in, 1);
-    mbar_init(&s.bar_mma, 1);
+    int n = 0;
+    for (int h = 0; h < d.hq && n < 1024; ++h)
+      if (pattern[h] == CRISP_PATTERN_PE) s.pe_heads[n++] = h;
+    s.n_pe = n;
+    mbar_init(&s.bar_a_full, 1);
+    mbar_init(&s.bar_a_free, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s.bar_b_full[i], 1);
+      mbar_init(&s.bar_b_free[i], 1);
+      mbar_init(&s.bar_acc_full[i], 1);
+      mbar_init(&s.bar_acc_free[i], 4);  // one arrival per warp of the group that drains the buffer
+    }
     fence_mbar_init();
   }
-  if (warp == 4) {
-    tmem_alloc(&s.tmem_base, 128);
+  __syncthreads();
+  const int n_pe = s.n_pe;
+  if (n_pe == 0) return;  // nothing routed to pooled estimation (uniform over the CTA)
+  if (warp == 8) {
+    tmem_alloc(&s.tmem_base, 256);
     tmem_relinquish();
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tm = s.tmem_base;
-  bool ok = true;
-  if (warp == 4) {
+  const int nt = (d.nb + kBlock - 1) / kBlock;
+  const int n_items = nt * n_pe, n_cta = gridDim.x, cta = blockIdx.x;
+
+  if (warp == 8) {
     if (lane == 0) {
-      mbar_arrive_expect_tx(&s.bar_in, 6u * 32768u);
+      // ---- TMA producer and MMA issuer
       for (int pl = 0; pl < 3; ++pl) {
-        tma_load_3d(s.a[pl][0], &maps.q[pl], &s.bar_in, 0, h, mt * kBlock);
-        tma_load_3d(s.a[pl][1], &maps.q[pl], &s.bar_in, 64, h, mt * kBlock);
-        tma_load_3d(s.b[pl][0], &maps.k[pl], &s.bar_in, 0, h / d.group, jt * kBlock);
-        tma_load_3d(s.b[pl][1], &maps.k[pl], &s.bar_in, 64, h / d.group, jt * kBlock);
+        prefetch_tmap(&maps.q[pl]);
+        prefetch_tmap(&maps.k[pl]);
       }
-      ok = mbar_wait(&s.bar_in, 0, &s.abort_flag);
-      if (ok) {
-        tc_fence_after_sync();
-        constexpr uint32_t idesc = umma_idesc_bf16(128, 128, false, false);
-        // (term of Q, term of K), smallest products first
-        const int pa[6] = {2, 0, 1, 1, 0, 0}, pb[6] = {0, 2, 1, 0, 1, 0};
+      constexpr uint32_t idesc = umma_idesc_bf16(128, 128, false, false);
+      // (term of Q, term of K), smallest products first
+      const int pa[6] = {2, 0, 1, 1, 0, 0}, pb[6] = {0, 2, 1, 0, 1, 0};
+      const uint64_t a_desc0 = umma_desc_sw128(smem_u32(s.a[0][0]), 0, 1024);
+      const uint64_t b_desc0 = umma_desc_sw128(smem_u32(s.b[0][0]), 0, 1024);
+      bool ok = true;
+      uint32_t T = 0;               // tiles issued so far by this CTA
+      uint32_t acc_uses[2] = {0, 0};  // tiles that went into each accumulator
+      auto load_b = [&](int hf, int kvh, int jt) {
+        mbar_arrive_expect_tx(&s.bar_b_full[hf], 3u * 16384u);
+        for (int pl = 0; pl < 3; ++pl) tma_load_3d(s.b[hf][pl], &maps.k[pl], &s.bar_b_full[hf], hf * 64, kvh, jt * kBlock);
+      };
+      for (int round = 0; ok; ++round) {
+        int hs, mt;
+        if (!logits_item(round, cta, n_cta, n_items, n_pe, nt, &hs, &mt)) break;
+        const int h = s.pe_heads[hs], kvh = h / d.group;
+        // the strip's operands may be replaced once every MMA of the previous item has read them
+        if (round > 0) ok = mbar_wait(&s.bar_a_free, (round - 1) & 1, &s.abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&s.bar_a_full, 6u * 16384u);
+        for (int pl = 0; pl < 3; ++pl)
+          for (int hf = 0; hf < 2; ++hf) tma_load_3d(s.a[pl][hf], &maps.q[pl], &s.bar_a_full, hf * 64, h, mt * kBlock);
+        // first tile of the item: both halves of the K-side operands (the slots are free: see the loop's end)
+        if (T > 0) {
+          ok = mbar_wait(&s.bar_b_free[0], (T - 1) & 1, &s.abort_flag) && mbar_wait(&s.bar_b_free[1], (T - 1) & 1, &s.abort_flag);
+          if (!ok) break;
+        }
+        load_b(0, kvh, 0);
+        load_b(1, kvh, 0);
+        ok = mbar_wait(&s.bar_a_full, round & 1, &s.abort_flag);
+        for (int jt = 0; jt <= mt && ok; ++jt, ++T) {
+          // even tiles of an item accumulate in buffer 0 (drained by epilogue group 0), odd ones in buffer 1
+          const int acc = jt & 1;
+          if (acc_uses[acc] > 0) ok = mbar_wait(&s.bar_acc_free[acc], (acc_uses[acc] - 1) & 1, &s.abort_flag);
+          ++acc_uses[acc];
+          for (int hf = 0; hf < 2 && ok; ++hf) {
+            ok = mbar_wait(&s.bar_b_full[hf], T & 1, &s.abort_flag);
+            if (!ok) break;
+            tc_fence_after_sync();
 #pragma unroll
-        for (int t = 0; t < 6; ++t)
+            for (int t = 0; t < 6; ++t)
 #pragma unroll
-          for (int kk = 0; kk < 8; ++kk) {
-            const uint64_t ad = umma_desc_sw128(smem_u32(s.a[pa[t]][kk >> 2]) + (kk & 3) * 32, 0, 1024);
-            const uint64_t bd = umma_desc_sw128(smem_u32(s.b[pb[t]][kk >> 2]) + (kk & 3) * 32, 0, 1024);
-            umma_ss(tm, ad, bd, idesc, (t > 0 || kk > 0) ? 1u : 0u);
+              for (int k4 = 0; k4 < 4; ++k4) {
+                // term: 32 KB apart (A) / 16 KB apart (B); 64-dim half: 16 KB (A) / 48 KB (B); 32 B per K step
+                const uint64_t ad = a_desc0 + static_cast<uint64_t>((pa[t] * 32768 + hf * 16384 + k4 * 32) >> 4);
+                const uint64_t bd = b_desc0 + static_cast<uint64_t>((hf * 49152 + pb[t] * 16384 + k4 * 32) >> 4);
+                umma_ss(tm + acc * 128, ad, bd, idesc, (hf > 0 || t > 0 || k4 > 0) ? 1u : 0u);
+              }
+            umma_commit(&s.bar_b_free[hf]);
+            if (hf == 0) {
+              // Slot 1 of this tile: free once the previous tile's second half has been multiplied, which the
+              // pipe does before it starts on the MMAs just issued; the load then has their time to arrive.
+              // (The first tile of an item had both slots filled in the item's prologue.)
+              if (jt > 0) {
+                ok = mbar_wait(&s.bar_b_free[1], (T - 1) & 1, &s.abort_flag);
+                if (ok) load_b(1, kvh, jt);
+              }
+            } else {
+              umma_commit(&s.bar_acc_full[acc]);
+              if (jt == mt) umma_commit(&s.bar_a_free);
+              // slot 0 for the next tile: free once this tile's first half is done, i.e. while its second runs
+              if (jt < mt) {
+                ok = mbar_wait(&s.bar_b_free[0], T & 1, &s.abort_flag);
+                if (ok) load_b(0, kvh, jt + 1);
+              }
+            }
           }
-        umma_commit(&s.bar_mma);
+        }
       }
     }
     __syncwarp();
   } else {
-    // ---- one thread per row of the tile: scale, then through shared memory so that the rows go out coalesced
-    ok = mbar_wait(&s.bar_mma, 0, &s.abort_flag);
-    float* stage = reinterpret_cast<float*>(s.a);  // 128 x 129 floats over the operand tiles, which are dead now
-    if (ok) {
-      tc_fence_after_sync();
-      const uint32_t lane_addr = static_cast<uint32_t>(warp * 32) << 16;
+    // ---- epilogue: one thread per row of the strip and group; group gr drains accumulator gr
+    const int gr = warp >> 2, r_ = tid & 127;
+    const uint32_t lane_addr = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const bool vec_ok = (d.nb & 3) == 0;
+    bool ok = true;
+    uint32_t uses = 0;  // tiles this group has drained
+    for (int round = 0; ok; ++round) {
+      int hs, mt;
+      if (!logits_item(round, cta, n_cta, n_items, n_pe, nt, &hs, &mt)) break;
+      const int h = s.pe_heads[hs];
+      const int m = mt * kBlock + r_;
+      const bool row_ok = m < d.nb;
+      float* zrow = w.amat + (static_cast<size_t>(h) * d.nb + (row_ok ? m : 0)) * d.nb;
+      float M = -INFINITY, S = 0.f;
+      for (int jt = gr; jt <= mt && ok; jt += 2, ++uses) {
+        ok = mbar_wait_warp(&s.bar_acc_full[gr], uses & 1, &s.abort_flag);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t r[4][32];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t r[32];
-        tmem_ld_x32(tm + lane_addr + c * 32, r);
+        for (int c = 0; c < 4; ++c) tmem_ld_x32(tm + lane_addr + gr * 128 + c * 32, r[c]);
         tmem_ld_wait();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s.bar_acc_free[gr]);
+        if (!row_ok) continue;
+        const int J0 = jt * kBlock;
+        const int n_valid = min(kBlock, m - J0 + 1);  // columns J <= m of this tile (128 except on the diagonal tile)
+        float tmax = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) stage[tid * 129 + c * 32 + i] = __uint_as_float(r[i]) * d.scale_log2;
-      }
-    }
-    named_bar_sync(1, 128);
-    if (ok) {
-      float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
-      for (int rr = warp; rr < kBlock; rr += 4) {
-        const int m = mt * kBlock + rr;
-        if (m >= d.nb) break;
+        for (int c = 0; c < 4; ++c)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          const int J = jt * kBlock + c * 32 + lane;
-          if (J <= m) am[static_cast<size_t>(m) * d.nb + J] = stage[rr * 129 + c * 32 + lane];
+          for (int i = 0; i < 32; ++i) {
+            const float z = __uint_as_float(r[c][i]) * d.scale_log2;
+            r[c][i] = __float_as_uint(z);
+            if (c * 32 + i < n_valid) tmax = fmaxf(tmax, z);
+          }
+        float tsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (c * 32 + i < n_valid) tsum += ex2(__uint_as_float(r[c][i]) - tmax);
+        const float nm = fmaxf(M, tmax);
+        S = S * ex2(M - nm) + tsum * ex2(tmax - nm);
+        M = nm;
+        if (vec_ok && n_valid == kBlock) {
+          float4* dst = reinterpret_cast<float4*>(zrow + J0);
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              dst[c * 8 + (i >> 2)] = make_float4(__uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1]),
+                                                  __uint_as_float(r[c][i + 2]), __uint_as_float(r[c][i + 3]));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c * 32 + i < n_valid) zrow[J0 + c * 32 + i] = __uint_as_float(r[c][i]);
         }
       }
+      // the odd tiles' statistics join the even tiles' (every row has an even tile: tile 0)
+      if (gr == 1) s.row_state[r_] = make_float2(M, S);
+      named_bar_sync(1, 256);
+      if (gr == 0 && ok && row_ok) {
+        const float2 o = s.row_state[r_];
+        const float nm = fmaxf(M, o.x);
+        S = S * ex2(M - nm) + (o.y > 0.f ? o.y * ex2(o.x - nm) : 0.f);
+        w.row_m[static_cast<size_t>(h) * d.nb + m] = nm;
+        w.row_inv[static_cast<size_t>(h) * d.nb + m] = 1.0f / (S * static_cast<float>(d.nb));
+      }
+      named_bar_sync(1, 256);  // row_state may be overwritten by the next item
+      // a wait that gave up in either group ends both (the flag was set before that group reached the barriers)
+      ok = ok && *reinterpret_cast<volatile int*>(&s.abort_flag) == 0;
     }
   }
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0 && s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
-  if (warp == 4) tmem_dealloc(tm, 128);
+  if (warp == 8) tmem_dealloc(tm, 256);
 }
 
-// Row softmax over J <= m, divided by N_b (= the total of the pooled map).
-__global__ void __launch_bounds__(256)
-pe_normalise_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
-  const int m = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
-  if (pattern[h] != CRISP_PATTERN_PE) return;
-  float* row = w.amat + (static_cast<size_t>(h) * d.nb + m) * d.nb;
-  __shared__ float red[32];
-  __shared__ float fscratch[32];
-  float mx = -INFINITY;
-  for (int J = tid; J <= m; J += 256) mx = fmaxf(mx, row[J]);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-  if ((tid & 31) == 0) red[tid >> 5] = mx;
-  __syncthreads();
-  mx = red[0];
-  for (int i = 1; i < 8; ++i) mx = fmaxf(mx, red[i]);
-  float sum = 0.f;
-  for (int J = tid; J <= m; J += 256) sum += exp2f(row[J] - mx);
-  const float total = block_sum<float>(sum, fscratch);
-  const float inv = 1.0f / (total * static_cast<float>(d.nb));
-  for (int J = tid; J <= m; J += 256) row[J] = exp2f(row[J] - mx) * inv;
-}
+// Entry (m, J) of the pooled map: causal row softmax divided by the total N_b.  Every pass computes it with
+// these two instructions, so all of them see the same bits.
+__device__ __forceinline__ float pe_value(float z, float row_max, float row_inv) { return ex2(z - row_max) * row_inv; }
 
 // ------------------------------------------------------------------------------------------------
 // PE heads: gamma cut by radix histogram over the value bits
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ bool key_in_level(unsigned int key, unsigned int prefix, int level, int* bin) {
-  if (level == 0) {
-    *bin = static_cast<int>(key >> 20);
-    return true;
-  }
-  if (level == 1) {
-    *bin = static_cast<int>((key >> 9) & 2047u);
-    return (key >> 20) == (prefix >> 20);
-  }
-  *bin = static_cast<int>(key & 511u);
-  return (key >> 9) == (prefix >> 9);
-}
-
-__global__ void __launch_bounds__(256)
-pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int level) {
-  const int h = blockIdx.y, tid = threadIdx.x;
-  if (pattern[h] != CRISP_PATTERN_PE) return;
-  __shared__ unsigned int cnt[2048];
-  __shared__ unsigned long long mass[2048];
-  const int nbins = level == 2 ? kL2Bins : 2048;
-  for (int i = tid; i < nbins; i += 256) {
-    cnt[i] = 0u;
-    mass[i] = 0ull;
-  }
-  __syncthreads();
-  const unsigned int prefix = w.cut[h].prefix;
-  if (level > 0 && w.cut[h].take == -1) return;  // gamma is out of reach: everything is kept
-  const float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
-  for (int m = blockIdx.x; m < d.nb; m += gridDim.x) {
-    const float* row = am + static_cast<size_t>(m) * d.nb;
-    // 1024 entries per pass: the four loads of a thread are issued before any of them is binned
-    for (int J0 = 0; J0 <= m; J0 += 1024) {
-      float vals[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int J = J0 + 256 * u + tid;
-        vals[u] = J <= m ? row[J] : 0.f;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int J = J0 + 256 * u + tid;
-        if (J0 + 256 * u > m) break;  // uniform: the whole chunk lies beyond the row
-        int bin = -1;
-        unsigned long long fixed = 0ull;
-        if (J <= m) {
-          const float v = vals[u];
-          int b;
-          if (key_in_level(__float_as_uint(v), prefix, level, &b)) {
-            bin = b;
-            fixed = __float2ull_rn(v * kMassScale);
-          }
-        }
-        // Level 0: neighbouring entries of a flat map fall into a handful of bins: lanes with the same bin elect a
-        // leader and add their counts and masses (three 20-bit limbs, summed exactly) in one atomic each.
-        if (level > 0) {
-          // lower levels: the 11 / 9 bits below the fixed prefix spread the entries over many bins
-          if (bin >= 0) {
-            atomicAdd(&cnt[bin], 1u);
-            atomicAdd(&mass[bin], fixed);
-          }
-          continue;
-        }
-        const unsigned int peers = __match_any_sync(0xffffffffu, bin);
-        const unsigned int l0 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed & 0xFFFFFull));
-        const unsigned int l1 = __reduce_add_sync(peers, static_cast<unsigned int>((fixed >> 20) & 0xFFFFFull));
-        const unsigned int l2 = __reduce_add_sync(peers, static_cast<unsigned int>(fixed >> 40));
-        if (bin >= 0 && (tid & 31) == __ffs(peers) - 1) {
-          atomicAdd(&cnt[bin], static_cast<unsigned int>(__popc(peers)));
-          atomicAdd(&mass[bin], static_cast<unsigned long long>(l0) + (static_cast<unsigned long long>(l1) << 20) +
-                                    (static_cast<unsigned long long>(l2) << 40));
-        }
-      }
-    }
-  }
-  __syncthreads();
-  const int off = level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins);
-  unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + off;
-  unsigned long long* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
-  for (int i = tid; i < nbins; i += 256)
-    if (cnt[i]) {
-      atomicAdd(&gc[i], cnt[i]);
-      atomicAdd(&gm[i], mass[i]);
-    }
-}
-
-// One CTA per head: the bins are read once, in parallel (two per thread, largest values first), an exclusive
-// block scan gives the mass above every bin, and the first non-empty bin at which the mass reaches gamma
-// is the one the cut falls into.
-__global__ void __launch_bounds__(1024)
-pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int level) {
-  const int h = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (pattern[h] != CRISP_PATTERN_PE) return;
-  const int nbins = level == 2 ? kL2Bins : 2048;
-  const int off = level == 0 ? 0 : (level == 1 ? kL0Bins : kL0Bins + kL1Bins);
+// The bin of the current level that holds the cut: the bins are read once, in parallel (largest values first),
+// an exclusive block scan gives the mass above every bin, and the first non-empty bin at which the mass reaches
+// gamma is the one.  Called by all kHistThreads threads of the last CTA of a head to finish the level.
+__device__ void locate_cut(const Dims& d, const SelectPtrs& w, int h, int level, unsigned long long* warp_tot /*[17]*/,
+                           int* first_hit) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int kPer = kMaxBins / kHistThreads;  // bins per thread
+  const int nbins = level_bins(level);
+  const int off = level_offset(level);
   const unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + off;
   const unsigned long long* gm = w.hmass + static_cast<size_t>(h) * kHistStride + off;
   CutState c = w.cut[h];
@@ -490,17 +602,19 @@ pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtr
   }
   const double gd = static_cast<double>(d.gamma) * static_cast<double>(kMassScale);
   const unsigned long long gamma = gd >= 1.8e19 ? 0xffffffffffffffffull : static_cast<unsigned long long>(gd);
-
-  // position p (0 = largest values) is bin nbins - 1 - p; thread t owns positions 2t and 2t + 1
-  const int p0 = 2 * tid, p1 = 2 * tid + 1;
-  const unsigned long long m0 = p0 < nbins ? gm[nbins - 1 - p0] : 0ull, m1 = p1 < nbins ? gm[nbins - 1 - p1] : 0ull;
-  const unsigned int c0 = p0 < nbins ? gc[nbins - 1 - p0] : 0u, c1 = p1 < nbins ? gc[nbins - 1 - p1] : 0u;
-  // exclusive scan of the per-thread sums: warp shuffles, then the 32 warp totals
-  __shared__ unsigned long long warp_tot[32];
-  __shared__ int first_hit;
-  __shared__ unsigned long long total_mass;
-  if (tid == 0) first_hit = 0x7fffffff;
-  const unsigned long long mine = m0 + m1;
+  // position p (0 = largest values) is bin nbins - 1 - p; thread t owns positions kPer t .. kPer t + kPer - 1.
+  // The histograms were built with atomics by other CTAs: read them from L2.
+  unsigned long long mm[kPer];
+  unsigned int cc[kPer];
+  unsigned long long mine = 0ull;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    const int p = kPer * tid + i;
+    mm[i] = p < nbins ? __ldcg(gm + (nbins - 1 - p)) : 0ull;
+    cc[i] = p < nbins ? __ldcg(gc + (nbins - 1 - p)) : 0u;
+    mine += mm[i];
+  }
+  if (tid == 0) *first_hit = 0x7fffffff;
   unsigned long long incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -510,200 +624,450 @@ pe_cut_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtr
   if (lane == 31) warp_tot[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    const unsigned long long wt = warp_tot[lane];
+    const unsigned long long wt = lane < kHistThreads / 32 ? warp_tot[lane] : 0ull;
     unsigned long long wi = wt;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const unsigned long long t = __shfl_up_sync(0xffffffffu, wi, o);
       if (lane >= o) wi += t;
     }
-    warp_tot[lane] = wi - wt;  // mass of the warps before this one
-    if (lane == 31) total_mass = wi;
+    if (lane < kHistThreads / 32) warp_tot[lane] = wi - wt;  // mass of the warps before this one
+    if (lane == 31) warp_tot[16] = wi;                       // total
   }
   __syncthreads();
-  const unsigned long long before0 = c.mass_above + warp_tot[warp] + (incl - mine);  // mass above position p0
-  const unsigned long long before1 = before0 + m0;
-  const bool hit0 = c0 != 0u && before0 + m0 >= gamma, hit1 = c1 != 0u && before1 + m1 >= gamma;
-  if (hit0 || hit1) atomicMin(&first_hit, hit0 ? p0 : p1);
+  unsigned long long before = c.mass_above + warp_tot[warp] + (incl - mine);  // mass above this thread's first position
+  int my_hit = 0x7fffffff;
+  unsigned long long hit_above = 0ull;
+  unsigned int hit_count = 0u;
+#pragma unroll
+  for (int i = 0; i < kPer; ++i) {
+    if (my_hit == 0x7fffffff && cc[i] != 0u && before + mm[i] >= gamma) {
+      my_hit = kPer * tid + i;
+      hit_above = before;
+      hit_count = cc[i];
+    }
+    before += mm[i];
+  }
+  if (my_hit != 0x7fffffff) atomicMin(first_hit, my_hit);
   __syncthreads();
-  const int fp = first_hit;
+  const int fp = *first_hit;
   if (fp == 0x7fffffff) {
     if (tid == 0) {
       // the target exceeds the total mass (gamma >= 1 or rounding): keep every causal entry
       c.cutkey = 0u;
       c.take = -1;
-      c.mass_above += total_mass;
+      c.mass_above += warp_tot[16];
       w.cut[h] = c;
     }
     return;
   }
-  if (fp != p0 && fp != p1) return;
+  if (fp != my_hit) return;
   // the thread that owns the bin of the cut finishes the level
   const int found = nbins - 1 - fp;
-  const unsigned long long above = fp == p0 ? before0 : before1;
-  const unsigned int found_count = fp == p0 ? c0 : c1;
-  c.mass_above = above;
-  const int shift = level == 0 ? 20 : (level == 1 ? 9 : 0);
-  c.prefix |= static_cast<unsigned int>(found) << shift;
+  c.mass_above = hit_above;
+  c.prefix |= static_cast<unsigned int>(found) << level_shift(level);
   if (level == 2) {
     c.cutkey = c.prefix;
     // all entries of this bin are equal; t = the smallest count whose mass reaches gamma
     const unsigned long long v = __float2ull_rn(__uint_as_float(c.cutkey) * kMassScale);
     long long t = 1;
     if (v > 0ull) {
-      const unsigned long long need = gamma - above;  // > 0 here
+      const unsigned long long need = gamma - hit_above;  // > 0 here
       t = static_cast<long long>((need + v - 1ull) / v);
     }
     if (t < 1) t = 1;
-    if (t > static_cast<long long>(found_count)) t = static_cast<long long>(found_count);
+    if (t > static_cast<long long>(hit_count)) t = static_cast<long long>(hit_count);
     c.take = t;
   }
   w.cut[h] = c;
 }
 
-// Per row of a PE head: how many entries lie above the cut, how many tie with it, and how the two
-// forced entries (column 0 and the diagonal) compare.
-__global__ void __launch_bounds__(256)
-pe_row_stats_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
-  const int m = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
-  if (pattern[h] != CRISP_PATTERN_PE) return;
-  __shared__ int iscratch[32];
-  const CutState c = w.cut[h];
-  const float* row = w.amat + (static_cast<size_t>(h) * d.nb + m) * d.nb;
-  int gt = 0, eq = 0;
-  for (int J = tid; J <= m; J += 256) {
-    const unsigned int key = __float_as_uint(row[J]);
-    gt += key > c.cutkey;
-    eq += key == c.cutkey;
-  }
-  gt = block_sum<int>(gt, iscratch);
-  eq = block_sum<int>(eq, iscratch);
-  if (tid == 0) {
-    const unsigned int k0 = __float_as_uint(row[0]), km = __float_as_uint(row[m]);
-    const int f = (k0 > c.cutkey ? 1 : 0) | (k0 == c.cutkey ? 2 : 0) | (km > c.cutkey ? 4 : 0) |
-                  (km == c.cutkey ? 8 : 0);
-    const size_t o = static_cast<size_t>(h) * d.nb + m;
-    w.n_gt[o] = gt;
-    w.n_eq[o] = eq;
-    w.flags[o] = f;
-  }
+// Mass bookkeeping of the histograms.  The mass of an entry is its value in 2^-60 fixed point,
+// round(v * 2^60); for a value with biased exponent e >= 90 that is exactly its 24-bit significand shifted left
+// by e - 90.  All entries of one bin share their exponent at every level (level 0 bins ARE exponents, the
+// lower levels only see entries inside the cut's exponent), so a bin's mass is the sum of its entries'
+// significands, shifted once when the bin is flushed.  The sum is kept in shared memory as two 32-bit words
+// (low and high twelve bits of the significands) next to the count: plain 32-bit adds, no 64-bit atomics.
+// A CTA sees fewer than 2^19 entries of a head (host-side grid choice), so none of the words can overflow.
+// The rare values below 2^-37 (exponent < 90, zero included) go straight to the global histogram.
+constexpr int kMinFastExp = 90;
+
+__device__ __forceinline__ void hist_slow_add(const SelectPtrs& w, int h, int level, int bin, float v) {
+  atomicAdd(w.hcount + static_cast<size_t>(h) * kHistStride + level_offset(level) + bin, 1u);
+  atomicAdd(w.hmass + static_cast<size_t>(h) * kHistStride + level_offset(level) + bin, __float2ull_rn(v * kMassScale));
 }
 
-// Per PE head: ties are taken in row-major order, so row m takes clamp(T - (ties in rows < m), 0, ties_m).
-__global__ void __launch_bounds__(1024)
-pe_take_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
-  const int h = blockIdx.x, tid = threadIdx.x;
-  if (pattern[h] != CRISP_PATTERN_PE) return;
-  __shared__ long long scratch[33];
-  const int seg = (d.nb + 1023) / 1024;
-  const int b0 = min(tid * seg, d.nb), b1 = min(b0 + seg, d.nb);
-  const size_t base = static_cast<size_t>(h) * d.nb;
-  long long local = 0;
-  for (int m = b0; m < b1; ++m) local += w.n_eq[base + m];
-  long long before = block_exclusive_scan_1024(local, scratch, nullptr);
-  const CutState c = w.cut[h];
-  for (int m = b0; m < b1; ++m) {
-    const int eq = w.n_eq[base + m];
-    int take;
-    if (c.take < 0) {
-      take = eq;
+// One group of 128 consecutive entries of a row (four per lane) at one level.
+template <int kLevel, bool kMasked>
+__device__ __forceinline__ void hist_group(const float (&z)[4], int J, int m, float M, float inv, unsigned int prefix,
+                                           unsigned int* cnt, unsigned int* slo, unsigned int* shi, const SelectPtrs& w,
+                                           int h, int lane, int& gt, int& in) {
+  unsigned int key[4];
+  bool ins[4];
+  bool any = false;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    key[e] = __float_as_uint(pe_value(z[e], M, inv));
+    const bool valid = !kMasked || J + e <= m;
+    if (kLevel == 0) {
+      ins[e] = valid;
+    } else if (kLevel == 1) {
+      ins[e] = valid && (key[e] >> kL0Shift) == (prefix >> kL0Shift);
     } else {
-      const long long left = c.take - before;
-      take = static_cast<int>(left <= 0 ? 0 : (left >= eq ? eq : left));
+      ins[e] = valid && (key[e] >> kL1Shift) == (prefix >> kL1Shift);
+      gt += (valid && (key[e] >> kL1Shift) > (prefix >> kL1Shift)) ? 1 : 0;
+      in += ins[e] ? 1 : 0;
     }
-    before += eq;
-    const int f = w.flags[base + m];
-    const bool sel0 = (f & 1) || ((f & 2) && take >= 1);
-    const bool selm = (f & 4) || ((f & 8) && take >= eq);
-    int count = w.n_gt[base + m] + take + (sel0 ? 0 : 1);
-    if (m > 0) count += selm ? 0 : 1;
-    w.take[base + m] = take;
-    w.counts[base + m] = count;
+    any = any || ins[e];
+  }
+  if (kLevel > 0 && !__any_sync(0xffffffffu, any)) return;  // nothing of this group lies in the cut's bin
+  int bin[4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const int b = kLevel == 0 ? static_cast<int>(key[e] >> kL0Shift)
+                              : (kLevel == 1 ? static_cast<int>((key[e] >> kL1Shift) & (kL1Bins - 1))
+                                             : static_cast<int>(key[e] & (kL2Bins - 1)));
+    bin[e] = ins[e] ? b : -1;
+    if (ins[e] && (key[e] >> 23) < kMinFastExp) {
+      hist_slow_add(w, h, kLevel, b, __uint_as_float(key[e]));
+      bin[e] = -1;
+    }
+  }
+  // warp-wide rounds: the bin of the first lane that still holds an entry collects all of its entries in the warp
+  constexpr int kRounds = kLevel == 0 ? 3 : 1;
+#pragma unroll 1
+  for (int round = 0; round < kRounds; ++round) {
+    const bool left = (bin[0] & bin[1] & bin[2] & bin[3]) >= 0;  // some bin is not -1
+    const uint32_t have = __ballot_sync(0xffffffffu, left);
+    if (have == 0u) return;
+    const int first = bin[0] >= 0 ? bin[0] : (bin[1] >= 0 ? bin[1] : (bin[2] >= 0 ? bin[2] : bin[3]));
+    const int ref = __shfl_sync(0xffffffffu, first, __ffs(have) - 1);
+    unsigned int n = 0u, lo = 0u, hi = 0u;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (bin[e] == ref) {
+        ++n;
+        lo += key[e] & 0xFFFu;
+        hi += ((key[e] >> 12) & 0x7FFu) | 0x800u;
+        bin[e] = -1;
+      }
+    n = __reduce_add_sync(0xffffffffu, n);
+    lo = __reduce_add_sync(0xffffffffu, lo);
+    hi = __reduce_add_sync(0xffffffffu, hi);
+    if (lane == 0) {
+      atomicAdd(&cnt[ref], n);
+      atomicAdd(&slo[ref], lo);
+      atomicAdd(&shi[ref], hi);
+    }
+  }
+  // whatever is left goes in lane by lane
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    if (bin[e] >= 0) {
+      atomicAdd(&cnt[bin[e]], 1u);
+      atomicAdd(&slo[bin[e]], key[e] & 0xFFFu);
+      atomicAdd(&shi[bin[e]], ((key[e] >> 12) & 0x7FFu) | 0x800u);
+    }
+}
+
+// Four consecutive logits of a row.  With kVec the row's storage is read as one float4 (columns beyond m but
+// inside the row's N_b slots hold unspecified values, which the callers mask); otherwise element by element.
+template <bool kVec>
+__device__ __forceinline__ void load_z4(const float* __restrict__ row, int J, int m, float (&z)[4]) {
+  if (kVec) {
+    const float4 v = *reinterpret_cast<const float4*>(row + J);
+    z[0] = v.x; z[1] = v.y; z[2] = v.z; z[3] = v.w;
+  } else {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) z[e] = (J + e <= m) ? row[J + e] : 0.f;
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-// Expansion of VS heads, row lengths, scan, fill
-// ------------------------------------------------------------------------------------------------
-// Word `wd` (key blocks 32*wd .. 32*wd+31) of the keep bitmap of query block m of a VS head.
-__device__ __forceinline__ uint32_t vs_keep_word(const uint32_t* __restrict__ selv, const uint32_t* __restrict__ selsr,
-                                                 int nb, int m, int wd) {
-  const int sh = nb - 1 - m;              // slash offset s = m - J  <->  reversed bit J + sh
-  const int pos0 = wd * 32 + sh, pos1 = pos0 + 1;
-  const uint32_t a = __funnelshift_r(selsr[pos0 >> 5], selsr[(pos0 >> 5) + 1], pos0 & 31);
-  const uint32_t b = __funnelshift_r(selsr[pos1 >> 5], selsr[(pos1 >> 5) + 1], pos1 & 31);
-  uint32_t bits = selv[wd] | a | b;
-  if (wd == 0) bits |= 1u;
-  if (wd == (m >> 5)) {
-    bits |= 1u << (m & 31);
-    const int top = m & 31;
-    bits &= (top == 31) ? 0xffffffffu : ((2u << top) - 1u);
-  }
-  return bits;
-}
-
-__global__ void __launch_bounds__(256)
-count_vs_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m = blockIdx.x * 8 + warp, h = blockIdx.y;
-  if (m >= d.nb || pattern[h] != CRISP_PATTERN_VS) return;
-  const uint32_t* selv = w.selv + static_cast<size_t>(h) * w.words;
-  const uint32_t* selsr = w.selsr + static_cast<size_t>(h) * (w.words + 2);
-  int c = 0;
-  for (int wd = lane; wd <= (m >> 5); wd += 32) c += __popc(vs_keep_word(selv, selsr, d.nb, m, wd));
-  c = warp_sum_i(c);
-  if (lane == 0) w.counts[static_cast<size_t>(h) * d.nb + m] = c;
-}
-
-// Exclusive scan of all row lengths (head-major) into row_ptr; total into *nnz_needed; capacity check.
-__global__ void __launch_bounds__(1024)
-scan_rows_kernel(const Dims d, const SelectPtrs w, int64_t* __restrict__ row_ptr, int64_t capacity,
-                 int64_t* __restrict__ nnz_needed, int* status) {
-  const int tid = threadIdx.x;
-  const long long total_rows = static_cast<long long>(d.hq) * d.nb;
-  __shared__ long long scratch[33];
-  long long carry = 0;
-  // 4096 consecutive rows per pass, four per thread (coalesced), scanned across the block
-  for (long long base = 0; base < total_rows; base += 4096) {
-    const long long r0 = base + 4 * tid;
-    int c[4];
-    long long local = 0;
+// One histogram level of one head per CTA column (blockIdx.y = head).  A warp takes one row at a time (rows dealt
+// round robin from the longest down), reads its logits as float4 - 512 entries in flight per warp - recomputes
+// the normalised values and bins the ones whose upper bits match the prefix found so far.  Entries that share a
+// bin with the first pending entry of the warp are added across the warp and cost one set of adds (three such
+// rounds at level 0, where a row's values share two or three exponents; one at the lower levels, whose entries
+// are spread over thousands of bins unless the map is flat); what is left goes in lane by lane.  Level 2 also
+// counts, per row, the entries above and inside the cut's last bin.  The last CTA of a head to finish locates
+// the cut in the head's finished histogram.
+template <int kLevel, bool kVec>
+__global__ void __launch_bounds__(kHistThreads)
+pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  const int h = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
+  extern __shared__ uint8_t hist_raw[];
+  constexpr int nbins = level_bins(kLevel);
+  unsigned int* cnt = reinterpret_cast<unsigned int*>(hist_raw);  // [nbins] each
+  unsigned int* slo = cnt + nbins;
+  unsigned int* shi = slo + nbins;
+  __shared__ unsigned long long warp_tot[17];
+  __shared__ int first_hit;
+  __shared__ int is_last;
+  const CutState cs = w.cut[h];  // written by the previous level's last CTA (an earlier launch)
+  const bool skip = kLevel > 0 && cs.take == -1;  // gamma is out of reach: everything is kept
+  if (!skip) {
+    for (int i = tid; i < 3 * nbins; i += kHistThreads) cnt[i] = 0u;
+    __syncthreads();
+    const unsigned int prefix = cs.prefix;
+    const float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
+    const float* rm = w.row_m + static_cast<size_t>(h) * d.nb;
+    const float* ri = w.row_inv + static_cast<size_t>(h) * d.nb;
+    const int n_warps = gridDim.x * (kHistThreads / 32), gw = blockIdx.x * (kHistThreads / 32) + warp;
+    for (int m = d.nb - 1 - gw; m >= 0; m -= n_warps) {
+      const float* row = am + static_cast<size_t>(m) * d.nb;
+      const float M = rm[m], inv = ri[m];
+      int gt = 0, in = 0;
+      int J0 = 0;
+      // whole steps of 512 entries: the four loads of a lane are issued before any of them is binned
+      for (; J0 + 511 <= m; J0 += 512) {
+        float z[4][4];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      c[u] = r0 + u < total_rows ? w.counts[r0 + u] : 0;
-      local += c[u];
-    }
-    long long pass_total;
-    long long run = carry + block_exclusive_scan_1024(local, scratch, &pass_total);
+        for (int u = 0; u < 4; ++u) load_z4<kVec>(row, J0 + 128 * u + 4 * lane, m, z[u]);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const long long r = r0 + u;
-      if (r < total_rows) {
-        const int h = static_cast<int>(r / d.nb), m = static_cast<int>(r % d.nb);
-        row_ptr[static_cast<size_t>(h) * (d.nb + 1) + m] = run;
-        run += c[u];
-        if (m == d.nb - 1) row_ptr[static_cast<size_t>(h) * (d.nb + 1) + d.nb] = run;
+        for (int u = 0; u < 4; ++u)
+          hist_group<kLevel, false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
+      }
+      // the rest of the row, 128 entries at a time
+      for (; J0 <= m; J0 += 128) {
+        float z[4];
+        load_z4<kVec>(row, J0 + 4 * lane, m, z);
+        hist_group<kLevel, true>(z, J0 + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
+      }
+      if (kLevel == 2) {
+        gt = warp_sum_i(gt);
+        in = warp_sum_i(in);
+        if (lane == 0) {
+          w.n_gt[static_cast<size_t>(h) * d.nb + m] = gt;
+          w.n_eq[static_cast<size_t>(h) * d.nb + m] = in;
+        }
       }
     }
-    carry += pass_total;
+    __syncthreads();
+    unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + level_offset(kLevel);
+    unsigned long long* gm = w.hmass + static_cast<size_t>(h) * kHistStride + level_offset(kLevel);
+    for (int i = tid; i < nbins; i += kHistThreads)
+      if (cnt[i]) {
+        // the bin's exponent: its own index at level 0, the cut's exponent below
+        const int e = kLevel == 0 ? i : static_cast<int>(prefix >> kL0Shift);
+        const unsigned long long sig = (static_cast<unsigned long long>(shi[i]) << 12) + slo[i];
+        atomicAdd(&gc[i], cnt[i]);
+        atomicAdd(&gm[i], sig << (e - kMinFastExp));
+      }
   }
-  if (tid == 0) {
-    *nnz_needed = carry;
-    if (carry > capacity) atomicExch(status, CRISP_ERR_CAPACITY);
+  // the last CTA of this head to get here locates the cut in the finished histogram
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = atomicAdd(&w.hist_done[kLevel * d.hq + h], 1) == static_cast<int>(gridDim.x) - 1;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  locate_cut(d, w, h, kLevel, warp_tot, &first_hit);
+}
+
+// Per PE head: exact per-row counts of the entries above and tied with the cut, the ties taken per row (in
+// row-major order: row m takes clamp(T - ties in rows < m, 0, ties_m)), the row lengths and their prefix sum.
+// Only rows with an entry inside the cut's last bin (2048 adjacent fp32 values) are read again; the last CTA of a head to finish
+// does the head-wide part.
+__global__ void __launch_bounds__(1024)
+pe_rows_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  const int h = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
+  __shared__ long long scratch[33];
+  __shared__ int is_last;
+  const CutState c = w.cut[h];
+  const size_t base = static_cast<size_t>(h) * d.nb;
+  const float* am = w.amat + base * d.nb;
+  if (c.take != -1) {
+    const int n_warps = gridDim.x * 32, gw = blockIdx.x * 32 + warp;
+    for (int m = gw; m < d.nb; m += n_warps) {
+      if (w.n_eq[base + m] == 0) continue;  // no entry inside the cut's bin: the counts of level 2 are exact
+      const float* row = am + static_cast<size_t>(m) * d.nb;
+      const float M = w.row_m[base + m], inv = w.row_inv[base + m];
+      int gt = 0, eq = 0;
+      for (int J = lane; J <= m; J += 32) {
+        const unsigned int key = __float_as_uint(pe_value(row[J], M, inv));
+        gt += key > c.cutkey;
+        eq += key == c.cutkey;
+      }
+      gt = warp_sum_i(gt);
+      eq = warp_sum_i(eq);
+      if (lane == 0) {
+        w.n_gt[base + m] = gt;
+        w.n_eq[base + m] = eq;
+      }
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) is_last = atomicAdd(&w.rows_done[h], 1) == static_cast<int>(gridDim.x) - 1;
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  const int seg = (d.nb + 1023) / 1024;
+  const int b0 = min(tid * seg, d.nb), b1 = min(b0 + seg, d.nb);
+  long long local = 0;
+  if (c.take != -1)
+    for (int m = b0; m < b1; ++m) local += __ldcg(&w.n_eq[base + m]);
+  long long before = block_exclusive_scan_1024(local, scratch, nullptr);
+  long long len_local = 0;
+  for (int m = b0; m < b1; ++m) {
+    int count, take;
+    if (c.take == -1) {
+      take = 0;
+      count = m + 1;  // every causal entry
+    } else {
+      const int eq = __ldcg(&w.n_eq[base + m]);
+      const long long left = c.take - before;
+      take = static_cast<int>(left <= 0 ? 0 : (left >= eq ? eq : left));
+      before += eq;
+      // the forced entries (column 0 and the diagonal): selected already, or to be added
+      const float M = w.row_m[base + m], inv = w.row_inv[base + m];
+      const float* row = am + static_cast<size_t>(m) * d.nb;
+      const unsigned int k0 = __float_as_uint(pe_value(row[0], M, inv)), km = __float_as_uint(pe_value(row[m], M, inv));
+      const bool sel0 = k0 > c.cutkey || (k0 == c.cutkey && take >= 1);   // column 0 is the row's first tie
+      const bool selm = km > c.cutkey || (km == c.cutkey && take >= eq);  // the diagonal is its last
+      count = __ldcg(&w.n_gt[base + m]) + take + (sel0 ? 0 : 1);
+      if (m > 0) count += selm ? 0 : 1;
+    }
+    w.take[base + m] = take;
+    w.counts[base + m] = count;
+    len_local += count;
+  }
+  long long total;
+  long long run = block_exclusive_scan_1024(len_local, scratch, &total);
+  for (int m = b0; m < b1; ++m) {
+    w.local_off[base + m] = static_cast<int>(run);
+    run += w.counts[base + m];
+  }
+  if (tid == 0) w.head_total[h] = total;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Global offsets and the lists
+// ------------------------------------------------------------------------------------------------
+// The kept columns of one group of 128 consecutive entries of a PE row (four per lane) go, in ascending order,
+// to stage[base ...]; returns how many there were.  kEdge: the group may reach beyond the row's end.
+template <bool kEdge>
+__device__ __forceinline__ int fill_group(const float (&z)[4], int J, int m, float M, float inv, unsigned int cutkey,
+                                          bool all, int take, int& ties_seen, int* stage, int base, int lane) {
+  bool keep[4], eq[4];
+  int n_eq_lane = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const unsigned int key = __float_as_uint(pe_value(z[e], M, inv));
+    const bool valid = !kEdge || J + e <= m;
+    keep[e] = valid && (all || key > cutkey || J + e == 0 || J + e == m);
+    eq[e] = valid && !all && key == cutkey;
+    n_eq_lane += eq[e] ? 1 : 0;
+  }
+  // ties are rare: their ranks in the row are worked out only in groups that hold one
+  if (__any_sync(0xffffffffu, n_eq_lane > 0)) {
+    int incl = n_eq_lane;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    int rank = ties_seen + incl - n_eq_lane;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (eq[e]) {
+        keep[e] = keep[e] || rank < take;
+        ++rank;
+      }
+    ties_seen += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  const int n_keep = (keep[0] ? 1 : 0) + (keep[1] ? 1 : 0) + (keep[2] ? 1 : 0) + (keep[3] ? 1 : 0);
+  int incl = n_keep;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  int pos = base + incl - n_keep;
+#pragma unroll
+  for (int e = 0; e < 4; ++e)
+    if (keep[e]) stage[pos++] = J + e;
+  return __shfl_sync(0xffffffffu, incl, 31);
+}
+
+template <bool kVec>
+__device__ __forceinline__ void fill_pe_row(const float* __restrict__ row, int m, float M, float inv, unsigned int cutkey,
+                                            bool all, int take, int32_t* __restrict__ out, int* stage, int lane) {
+  int written = 0, ties_seen = 0;
+  // Steps of 512 columns (four loads per lane in flight); the kept columns of a step are gathered in shared
+  // memory and leave as contiguous 128-byte stores.
+  for (int J0 = 0; J0 <= m; J0 += 512) {
+    const bool whole = J0 + 511 < m;  // the step lies inside the row and does not hold the diagonal
+    float z[4][4];
+    int n = 0;
+    if (whole) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) load_z4<kVec>(row, J0 + 128 * u + 4 * lane, m, z[u]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        n += fill_group<false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, cutkey, all, take, ties_seen, stage, n, lane);
+    } else {
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (J0 + 128 * u <= m) load_z4<kVec>(row, J0 + 128 * u + 4 * lane, m, z[u]);
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (J0 + 128 * u <= m)
+          n += fill_group<true>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, cutkey, all, take, ties_seen, stage, n, lane);
+    }
+    __syncwarp();
+    for (int i = lane; i < n; i += 32) out[written + i] = stage[i];
+    written += n;
+    __syncwarp();
   }
 }
 
 __global__ void __launch_bounds__(256)
-fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w,
-            const int64_t* __restrict__ row_ptr, int32_t* __restrict__ col_idx, int64_t capacity,
-            const int64_t* __restrict__ nnz_needed) {
-  if (*nnz_needed > capacity) return;
+fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int64_t* __restrict__ row_ptr,
+            int32_t* __restrict__ col_idx, int64_t capacity, int64_t* __restrict__ nnz_needed, int* status) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m = blockIdx.x * 8 + warp, h = blockIdx.y;
-  if (m >= d.nb) return;
-  int32_t* out = col_idx + row_ptr[static_cast<size_t>(h) * (d.nb + 1) + m];
-  int written = 0;
+  const int h = blockIdx.y;
+  // offsets of the heads: every CTA adds the (few) head totals itself
+  __shared__ long long s_base, s_total;
+  __shared__ int stage_all[8][512];
+  if (threadIdx.x < 32) {
+    long long before = 0, all = 0;
+    for (int hh = lane; hh < d.hq; hh += 32) {
+      const long long t = w.head_total[hh];
+      all += t;
+      if (hh < h) before += t;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      before += __shfl_xor_sync(0xffffffffu, before, o);
+      all += __shfl_xor_sync(0xffffffffu, all, o);
+    }
+    if (lane == 0) {
+      s_base = before;
+      s_total = all;
+    }
+  }
+  __syncthreads();
+  const long long head_base = s_base, total = s_total;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+    *nnz_needed = total;
+    if (total > capacity) atomicExch(status, CRISP_ERR_CAPACITY);
+  }
+  // long rows first, so that the tail of the launch is made of short ones
+  const int m = d.nb - 1 - (blockIdx.x * 8 + warp);
+  if (m < 0) return;
+  const size_t rbase = static_cast<size_t>(h) * d.nb;
+  const long long start = head_base + w.local_off[rbase + m];
+  if (lane == 0) {
+    row_ptr[static_cast<size_t>(h) * (d.nb + 1) + m] = start;
+    if (m == d.nb - 1) row_ptr[static_cast<size_t>(h) * (d.nb + 1) + d.nb] = head_base + w.head_total[h];
+  }
+  if (total > capacity) return;  // the lists do not fit: col_idx stays untouched
+  int32_t* out = col_idx + start;
   if (pattern[h] == CRISP_PATTERN_VS) {
+    int written = 0;
     const uint32_t* selv = w.selv + static_cast<size_t>(h) * w.words;
     const uint32_t* selsr = w.selsr + static_cast<size_t>(h) * (w.words + 2);
     const int nwords = (m >> 5) + 1;
@@ -729,30 +1093,13 @@ fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs 
     }
   } else {
     const CutState c = w.cut[h];
-    const float* row = w.amat + (static_cast<size_t>(h) * d.nb + m) * d.nb;
-    const int take = w.take[static_cast<size_t>(h) * d.nb + m];
-    int ties_seen = 0;
-    // 128 columns per pass: the four loads of a lane are issued before the (serial) bookkeeping of the pass
-    for (int J0 = 0; J0 <= m; J0 += 128) {
-      unsigned int key[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int J = J0 + 32 * u + lane;
-        key[u] = J <= m ? __float_as_uint(row[J]) : 0u;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int J = J0 + 32 * u + lane;
-        const bool in = J <= m;
-        const bool gt = in && key[u] > c.cutkey, eq = in && key[u] == c.cutkey;
-        const uint32_t eqmask = __ballot_sync(0xffffffffu, eq);
-        const int my_tie = ties_seen + __popc(eqmask & ((1u << lane) - 1u));
-        const bool keep = in && (gt || (eq && my_tie < take) || J == 0 || J == m);
-        const uint32_t keepmask = __ballot_sync(0xffffffffu, keep);
-        if (keep) out[written + __popc(keepmask & ((1u << lane) - 1u))] = J;
-        written += __popc(keepmask);
-        ties_seen += __popc(eqmask);
-      }
+    const float* row = w.amat + (rbase + m) * d.nb;
+    const float M = w.row_m[rbase + m], inv = w.row_inv[rbase + m];
+    const int take = w.take[rbase + m];
+    if ((d.nb & 3) == 0) {
+      fill_pe_row<true>(row, m, M, inv, c.cutkey, c.take == -1, take, out, stage_all[warp], lane);
+    } else {
+      fill_pe_row<false>(row, m, M, inv, c.cutkey, c.take == -1, take, out, stage_all[warp], lane);
     }
   }
 }
@@ -767,6 +1114,12 @@ SelectPtrs carve(const Dims& d, void* ws, size_t* total) {
     return r;
   };
   w.words = (d.nb + 31) / 32;
+  // zeroed region first (directly behind the header, so one memset covers both)
+  w.hcount = static_cast<unsigned int*>(take(sizeof(unsigned int) * d.hq * kHistStride));
+  w.hmass = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * d.hq * kHistStride));
+  w.hist_done = static_cast<int*>(take(sizeof(int) * 3 * d.hq));
+  w.rows_done = static_cast<int*>(take(sizeof(int) * d.hq));
+  w.zero_bytes = off;
   w.selv = static_cast<uint32_t*>(take(sizeof(uint32_t) * d.hq * w.words));
   w.selsr = static_cast<uint32_t*>(take(sizeof(uint32_t) * d.hq * (w.words + 2)));
   w.kbar = static_cast<float*>(take(sizeof(float) * d.hkv * d.nb * kHeadDim));
@@ -774,16 +1127,31 @@ SelectPtrs carve(const Dims& d, void* ws, size_t* total) {
   w.ksplit = static_cast<__nv_bfloat16*>(take(sizeof(__nv_bfloat16) * 3 * static_cast<size_t>(d.hkv) * d.nb * kHeadDim));
   w.qsplit = static_cast<__nv_bfloat16*>(take(sizeof(__nv_bfloat16) * 3 * static_cast<size_t>(d.hq) * d.nb * kHeadDim));
   w.amat = static_cast<float*>(take(sizeof(float) * static_cast<size_t>(d.hq) * d.nb * d.nb));
-  w.hcount = static_cast<unsigned int*>(take(sizeof(unsigned int) * d.hq * kHistStride));
-  w.hmass = static_cast<unsigned long long*>(take(sizeof(unsigned long long) * d.hq * kHistStride));
+  w.row_m = static_cast<float*>(take(sizeof(float) * d.hq * d.nb));
+  w.row_inv = static_cast<float*>(take(sizeof(float) * d.hq * d.nb));
   w.cut = static_cast<CutState*>(take(sizeof(CutState) * d.hq));
   w.n_gt = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
   w.n_eq = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
-  w.flags = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
-  w.take = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
   w.counts = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  w.take = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  w.local_off = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
+  w.head_total = static_cast<long long*>(take(sizeof(long long) * d.hq));
   *total = off;
   return w;
+}
+
+int launch_prepare(const Dims& d, const __nv_bfloat16* qb, const __nv_bfloat16* kb, const int32_t* pattern,
+                   const float* p_v, const float* p_s, const SelectPtrs& w, int vs_ctas, int pool_all_k,
+                   cudaStream_t stream) {
+  const size_t vs_smem = (sizeof(double) + sizeof(float) + sizeof(int) + 1) * static_cast<size_t>(d.nb) + 16;
+  CRISP_CUDA_TRY(cudaFuncSetAttribute(prepare_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      static_cast<int>(vs_smem)),
+                 "select: smem attribute");
+  const long long n_tiles = static_cast<long long>(d.nb) * (d.hkv + d.hq);
+  const int pool_ctas = static_cast<int>((n_tiles + 7) / 8);
+  CRISP_KERNEL("prepare", stream, prepare_kernel<<<vs_ctas + pool_ctas, 1024, vs_smem, stream>>>(
+                                      d, qb, kb, pattern, p_v, p_s, w, vs_ctas, pool_all_k));
+  return CRISP_OK;
 }
 
 }  // namespace
@@ -797,30 +1165,24 @@ size_t select_ws_bytes(const Dims& d) {
 int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pattern, const float* p_v,
                   const float* p_s, void* ws, int64_t* row_ptr, int32_t* col_idx, int64_t capacity,
                   int64_t* nnz_needed, cudaStream_t stream) {
-  if (d.nb > 8192) return CRISP_ERR_UNSUPPORTED;
+  if (d.nb > 8192 || d.hq > 1024) return CRISP_ERR_UNSUPPORTED;
   size_t total;
   SelectPtrs w = carve(d, ws, &total);
   int* status = static_cast<int*>(ws);
-  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "select: clear status");
-  CRISP_CUDA_TRY(cudaMemsetAsync(w.hcount, 0, sizeof(unsigned int) * d.hq * kHistStride, stream), "select: clear");
-  CRISP_CUDA_TRY(cudaMemsetAsync(w.hmass, 0, sizeof(unsigned long long) * d.hq * kHistStride, stream), "select: clear");
+  // status word, histograms and completion counters
+  CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, w.zero_bytes, stream), "select: clear");
 
-  // VS heads
-  const size_t vs_smem = (sizeof(double) + sizeof(float) + sizeof(int) + 1) * static_cast<size_t>(d.nb) + 16;
-  CRISP_CUDA_TRY(cudaFuncSetAttribute(select_vs_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      static_cast<int>(vs_smem)),
-                 "select: smem attribute");
-  CRISP_KERNEL("select_vs", stream, select_vs_kernel<<<dim3(d.hq, 2), 1024, vs_smem, stream>>>(d, pattern, p_v, p_s, w));
-
-  // PE heads (every kernel returns at once for heads routed to VS)
-  const __nv_bfloat16* qb = static_cast<const __nv_bfloat16*>(q);
-  const __nv_bfloat16* kb = static_cast<const __nv_bfloat16*>(k);
-  CRISP_KERNEL("pool_k", stream, pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, kb, d.hkv, 0, pattern, w.kbar, w.ksplit));
-  CRISP_KERNEL("pool_q", stream, pool_kernel<<<dim3(d.nb, d.hq), 128, 0, stream>>>(d, qb, d.hq, 1, pattern, w.qbar, w.qsplit));
+  // VS heads: selection and list lengths; PE heads: block means (the PE kernels return at once for VS heads)
+  int rc = launch_prepare(d, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k), pattern, p_v,
+                          p_s, w, d.hq, 0, stream);
+  if (rc != CRISP_OK) return rc;
+  int dev = 0, n_sm = 0;
+  CRISP_CUDA_TRY(cudaGetDevice(&dev), "select: device");
+  CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "select: SM count");
   {
     LogitsMaps maps;
     for (int pl = 0; pl < 3; ++pl) {
-      int rc = make_tmap_bf16_nhd(&maps.q[pl], w.qsplit + static_cast<size_t>(pl) * d.nb * d.hq * kHeadDim, d.nb, d.hq);
+      rc = make_tmap_bf16_nhd(&maps.q[pl], w.qsplit + static_cast<size_t>(pl) * d.nb * d.hq * kHeadDim, d.nb, d.hq);
       if (rc != CRISP_OK) return rc;
       rc = make_tmap_bf16_nhd(&maps.k[pl], w.ksplit + static_cast<size_t>(pl) * d.nb * d.hkv * kHeadDim, d.nb, d.hkv);
       if (rc != CRISP_OK) return rc;
@@ -830,22 +1192,28 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
                                         static_cast<int>(smem)),
                    "select: smem attribute");
     const int nt = (d.nb + kBlock - 1) / kBlock;
-    CRISP_KERNEL("pe_logits", stream, pe_logits_kernel<<<dim3(nt, nt, d.hq), 160, smem, stream>>>(maps, d, pattern, w, status));
+    const int grid = min(n_sm, nt * d.hq);
+    CRISP_KERNEL("pe_logits", stream, pe_logits_kernel<<<grid, 288, smem, stream>>>(maps, d, pattern, w, status));
   }
-  CRISP_KERNEL("pe_normalise", stream, pe_normalise_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w));
-  const int hist_ctas = d.nb < 128 ? d.nb : 128;
-  for (int level = 0; level < 3; ++level) {
-    CRISP_KERNEL("pe_hist", stream, pe_hist_kernel<<<dim3(hist_ctas, d.hq), 256, 0, stream>>>(d, pattern, w, level));
-    CRISP_KERNEL("pe_cut", stream, pe_cut_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w, level));
-  }
-  CRISP_KERNEL("pe_row_stats", stream, pe_row_stats_kernel<<<dim3(d.nb, d.hq), 256, 0, stream>>>(d, pattern, w));
-  CRISP_KERNEL("pe_take", stream, pe_take_kernel<<<d.hq, 1024, 0, stream>>>(d, pattern, w));
-
-  // expansion + compaction
-  CRISP_KERNEL("count_vs", stream, count_vs_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w));
-  CRISP_KERNEL("scan_rows", stream, scan_rows_kernel<<<1, 1024, 0, stream>>>(d, w, row_ptr, capacity, nnz_needed, status));
-  CRISP_KERNEL("fill", stream, fill_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(d, pattern, w, row_ptr, col_idx, capacity,
-                                                              nnz_needed));
+  // up to four CTAs per SM if every head is PE (two when half of them are); a warp takes a row at a time
+  // ... and never more than 2^18 entries of a head per CTA (the 32-bit mass words of pe_hist_kernel)
+  const long long causal = static_cast<long long>(d.nb) * (d.nb + 1) / 2;
+  int hist_ctas = max(1, min((d.nb + 15) / 16, (4 * n_sm + d.hq - 1) / d.hq));
+  hist_ctas = max(hist_ctas, static_cast<int>((causal + (1 << 18) - 1) >> 18));
+  auto hist_smem = [](int level) { return static_cast<size_t>(level_bins(level)) * 12; };
+  const bool vec = (d.nb & 3) == 0;  // rows start on 16-byte boundaries
+  auto* hist0 = vec ? pe_hist_kernel<0, true> : pe_hist_kernel<0, false>;
+  auto* hist1 = vec ? pe_hist_kernel<1, true> : pe_hist_kernel<1, false>;
+  auto* hist2 = vec ? pe_hist_kernel<2, true> : pe_hist_kernel<2, false>;
+  CRISP_CUDA_TRY(cudaFuncSetAttribute(hist1, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(hist_smem(1))),
+                 "select: smem attribute");
+  CRISP_KERNEL("pe_hist0", stream, hist0<<<dim3(hist_ctas, d.hq), kHistThreads, hist_smem(0), stream>>>(d, pattern, w));
+  CRISP_KERNEL("pe_hist1", stream, hist1<<<dim3(hist_ctas, d.hq), kHistThreads, hist_smem(1), stream>>>(d, pattern, w));
+  CRISP_KERNEL("pe_hist2", stream, hist2<<<dim3(hist_ctas, d.hq), kHistThreads, hist_smem(2), stream>>>(d, pattern, w));
+  const int rows_ctas = max(1, min((d.nb + 31) / 32, 8));
+  CRISP_KERNEL("pe_rows", stream, pe_rows_kernel<<<dim3(rows_ctas, d.hq), 1024, 0, stream>>>(d, pattern, w));
+  CRISP_KERNEL("fill", stream, fill_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(
+                                   d, pattern, w, row_ptr, col_idx, capacity, nnz_needed, status));
   CRISP_CUDA_TRY(cudaGetLastError(), "select: launch");
   return CRISP_OK;
 }
@@ -937,8 +1305,9 @@ int launch_route_jsd(const Dims& d, const void* q, const void* k, const float* p
   size_t total;
   SelectPtrs w = carve(d, ws, &total);
   CRISP_CUDA_TRY(cudaMemsetAsync(ws, 0, kWsHeader, stream), "route_jsd: clear status");
-  CRISP_KERNEL("pool_k", stream, pool_kernel<<<dim3(d.nb, d.hkv), 128, 0, stream>>>(d, static_cast<const __nv_bfloat16*>(k), d.hkv, 0, nullptr,
-                                                     w.kbar, nullptr));
+  // block means of K for every KV head (no VS work, no Q pooling)
+  int rc = launch_prepare(d, nullptr, static_cast<const __nv_bfloat16*>(k), nullptr, nullptr, nullptr, w, 0, 1, stream);
+  if (rc != CRISP_OK) return rc;
   CRISP_KERNEL("jsd", stream, jsd_kernel<<<d.hq, 256, sizeof(float) * d.nb, stream>>>(d, static_cast<const __nv_bfloat16*>(q), w.kbar, p_v,
                                                          tau_jsd, jsd, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route_jsd: launch");
