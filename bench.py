@@ -5,10 +5,15 @@ One step = one pass of the whole hot path over one synthetic layer: crisp_route 
 crisp_sparse_prefill (Algorithm 1).  Prints ONE JSON line (rank 0).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload L512k] [--impl crisp|reference]
+                  [--shard replicas|kv-groups]
 
 `value` is ms per layer of the whole path with inputs resident in HBM; `e2e` is the same through the
 C ABI with HOST buffers (pinned host -> device copies of Q, K, V and a device -> host copy of O inside the
 timed region).  The dense kernel (crisp_dense_prefill) is timed on the same inputs for the speedup.
+After the timed steps a few more steps run with the library's per-kernel timing switched on; from them come
+`kernels` (device time of every kernel against its algorithmic bytes) and `stages_hbm`.
+With N > 1 the default is one independent layer per rank (weak scaling); `--shard kv-groups` instead splits
+ONE layer's KV groups over the ranks (strong scaling; no collective in the data path either way).
 `--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
@@ -31,8 +36,6 @@ import torch
 from workloads import synth
 
 FLOP_PER_BLOCK = 4 * 128 ** 3          # QK^T + PV of one 128 x 128 x 128 block pair
-# kernels launched per step: route 5, select 16, sparse prefill 4 (merge, 2 x schedule, attention)
-LAUNCHES_ROUTE, LAUNCHES_SELECT, LAUNCHES_PREFILL = 5, 16, 4
 
 
 def load_peaks():
@@ -94,60 +97,99 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(w, q, k, v, seed=0, blocks_per_head=4):
-    """Times the fp64 oracle (as it stands) on a bounded sample of the workload and extrapolates to
-    ms/layer: route+select of two heads (one per class) scaled to H_q, attention of a few query
-    blocks scaled by the number of listed blocks.  Returns (ms_per_layer, description, cores)."""
+def blas_threads() -> int:
+    """Threads numpy's BLAS uses (what the oracle's matrix products run on)."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = [int(x.get("num_threads", 1)) for x in threadpool_info() if x.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def oracle_sample(w, q, k, v, heads, blocks_per_head, block_budget, gpu_lists=None):
+    """Times the fp64 oracle (as it stands) on a bounded sample of the workload and extrapolates to ms/layer.
+
+    Steps O1-O6 (route, select, expansion) run in full for `heads` and are scaled to H_q by head class; exact
+    attention (O7) runs on `blocks_per_head` query blocks per sampled head, picked at evenly spaced quantiles of
+    the list length among the rows short enough to keep the sample near `block_budget` listed key blocks, and is
+    scaled by the number of listed blocks.  With `gpu_lists` = (pattern, row_ptr, {h: cols of head h}) the lists
+    of the sampled heads are also compared with the CUDA path's under the matching rule and the excused blocks
+    counted.  Returns (ms_per_layer, description, near_threshold dict or None)."""
     from oracle import crisp_oracle as orc
-    hq, hkv, nb = w.n_q_heads, w.n_kv_heads, w.n_blocks
-    classes = {}
-    for h, c in enumerate(w.head_classes):
-        classes.setdefault(c, h)
-    heads = sorted(classes.values())[:2]
+    from oracle import matching
+    hq, nb = w.n_q_heads, w.n_blocks
     kw = dict(block=128, sink_tokens=w.sink_tokens, local_tokens=w.local_tokens, tau=w.tau, alpha=w.alpha,
               gamma=w.gamma, k_min_blocks=w.k_min_blocks)
-    t_sel, t_attn, blocks_done, nnz_est = 0.0, 0.0, 0, 0.0
-    rng = np.random.default_rng(seed)
+    rule = dict(selector=0, alpha=w.alpha, gamma=w.gamma, k_min=w.k_min_blocks)
+    class_count = {}
+    for c in w.head_classes:
+        class_count[c] = class_count.get(c, 0) + 1
+    sampled_per_class = {}
     for h in heads:
+        sampled_per_class[w.head_classes[h]] = sampled_per_class.get(w.head_classes[h], 0) + 1
+    t_sel, t_attn, blocks_done, nnz_est, n_blocks_run = 0.0, 0.0, 0, 0.0, 0
+    near = dict(heads_checked=[], band_1e3=0, mass_1e6=0, candidates=0, mismatched_heads=0) if gpu_lists else None
+    per_head_budget = max(block_budget // max(len(heads), 1), 1)
+    for h in heads:
+        kv = h // w.group
         qh = q[:, h].float().cpu().numpy()
-        kh = k[:, h // w.group].float().cpu().numpy()
-        vh = v[:, h // w.group].float().cpu().numpy()
+        kh = k[:, kv].float().cpu().numpy()
+        vh = v[:, kv].float().cpu().numpy()
         t0 = time.perf_counter()
         res = orc.head_pipeline(qh, kh, **kw)
         t_sel += time.perf_counter() - t0
         lens = np.array([len(c) for c in res["cols"]])
-        nnz_est += lens.sum() * (sum(1 for c in w.head_classes if c == w.head_classes[h]))
-        # a few query blocks, kept small enough for a bounded run
-        order = np.argsort(lens)
-        picks = [int(order[(2 * i + 1) * len(order) // (2 * blocks_per_head)]) for i in range(blocks_per_head)]
+        cls = w.head_classes[h]
+        nnz_est += float(lens.sum()) * class_count[cls] / sampled_per_class[cls]
+        # query blocks at evenly spaced quantiles of the list length, among the shortest rows whose quantile
+        # sample stays within the head's share of the budget
+        order = np.argsort(lens, kind="stable")
+        hi = len(order)
+        while hi > blocks_per_head:
+            picks = [int(order[(2 * i + 1) * hi // (2 * blocks_per_head)]) for i in range(blocks_per_head)]
+            if lens[picks].sum() <= per_head_budget:
+                break
+            hi = max(blocks_per_head, hi * 3 // 4)
+        picks = [int(order[(2 * i + 1) * hi // (2 * blocks_per_head)]) for i in range(min(blocks_per_head, hi))]
         for m in picks:
             t0 = time.perf_counter()
             orc.sparse_attention_block(qh, kh, vh, m, res["cols"][m], 128)
             t_attn += time.perf_counter() - t0
             blocks_done += len(res["cols"][m])
-    per_head_sel = t_sel / len(heads)
+            n_blocks_run += 1
+        if gpu_lists is not None:
+            pattern, row_ptr, cols_of = gpu_lists
+            near["heads_checked"].append(h)
+            if int(pattern[h]) != res["pattern"]:
+                near["mismatched_heads"] += 1
+                continue
+            b = matching.list_bounds(res, nb, **rule)
+            rp = row_ptr[h] - row_ptr[h][0]
+            got = matching.lists_to_matrix(rp, cols_of[h], nb)
+            missing, extra = matching.compare_lists(got, b)
+            near["band_1e3"] += b["band"]
+            near["mass_1e6"] += b["mass"]
+            near["candidates"] += b["candidates"]
+            if missing or extra:
+                near["mismatched_heads"] += 1
     per_block = t_attn / max(blocks_done, 1)
-    # heads of classes not sampled are counted like the nearest sampled class
-    covered = sum(1 for c in w.head_classes if classes[c] in heads)
+    covered = sum(class_count[c] for c in sampled_per_class)
     nnz_est *= hq / max(covered, 1)
-    ms = (per_head_sel * hq + per_block * nnz_est) * 1e3
-    desc = (f"oracle route+select on heads {heads} (x{hq}/{len(heads)}), exact attention on "
-            f"{blocks_done} listed blocks extrapolated to ~{int(nnz_est)} blocks")
-    cores = torch.get_num_threads()
-    return ms, desc, cores
+    ms = (t_sel / max(len(heads), 1) * hq + per_block * nnz_est) * 1e3
+    desc = (f"oracle steps O1-O6 in full on heads {list(heads)} (scaled to {hq} heads by head class), exact attention "
+            f"(O7) on {n_blocks_run} query blocks = {blocks_done} listed key blocks, scaled to ~{int(nnz_est)} blocks")
+    return ms, desc, near
 
 
-def ncu_traffic_bytes(kernel: str, workload: str):
-    """DRAM bytes per launch of `kernel` from the committed ncu summary of `workload`, or None."""
-    path = os.path.join(ROOT, "profiles", f"dram_traffic_{workload}_ncu.md")
-    if not os.path.exists(path):
-        return None
-    key = f"traffic_bytes_per_launch {kernel} {workload} ="
-    with open(path) as f:
-        for line in f:
-            if line.startswith(key):
-                return int(line.split("=")[1])
-    return None
+def baseline_heads(w):
+    """Every head up to 32k tokens, else the first head of every head class."""
+    if w.seq_len <= 32768:
+        return list(range(w.n_q_heads))
+    first = {}
+    for h, c in enumerate(w.head_classes):
+        first.setdefault(c, h)
+    return sorted(first.values())
 
 
 def max_over_ranks(ms: float, dist, device) -> float:
@@ -159,9 +201,36 @@ def max_over_ranks(ms: float, dist, device) -> float:
     return float(t.item())
 
 
-def job_ms_per_layer(ms_per_step: float, world: int) -> float:
-    """Weak scaling: every rank processes one layer per step, so the job does `world` layers per step."""
-    return ms_per_step / world
+def sum_over_ranks(x: float, dist, device) -> float:
+    if dist is None:
+        return x
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def job_ms_per_layer(ms_per_step: float, world: int, shard: str = "replicas") -> float:
+    """Replicas (weak scaling): every rank processes one layer per step, so the job does `world` layers per step.
+    KV-group shards (strong scaling): the ranks share ONE layer, which takes as long as the slowest rank."""
+    return ms_per_step / world if shard == "replicas" else ms_per_step
+
+
+def kernel_bytes(name, w, n_pe, n_kv_pe, nnz):
+    """Algorithmic bytes one launch of a kernel must move: what the step it implements needs, not what the
+    implementation happens to touch.  None for kernels that are not streaming (latency or tensor bound)."""
+    n, hq, hkv, nb = w.seq_len, w.n_q_heads, w.n_kv_heads, w.n_blocks
+    causal = nb * (nb + 1) // 2
+    partial = (3 if n % 128 == 0 else 4) * 4 * 128 * nb * hq       # per-(row, tile) softmax partials
+    table = {
+        "proxy": n * hkv * 256 + hq * 32768 + partial,              # K once, Q_hat, partials written
+        "tile_sums": partial + 2 * 4 * nb * hq,                     # partials read, p_v and p_s written
+        "prepare": (n_pe + n_kv_pe) * n * 256 + (n_pe + n_kv_pe) * nb * 1280,   # Q of PE heads, K; pooled means
+        "pe_logits": (n_pe + n_kv_pe) * nb * 768 + n_pe * causal * 4,           # bf16 terms read, logits written
+        "pe_hist0": n_pe * causal * 4, "pe_hist1": n_pe * causal * 4, "pe_hist2": n_pe * causal * 4,
+        "fill": n_pe * causal * 4 + nnz * 4 + 8 * hq * (nb + 1),
+        "merge_lists": nnz * 4,                                      # lists read (the union lists written on top)
+    }
+    return table.get(name)
 
 
 def main():
@@ -174,6 +243,8 @@ def main():
                     help="instead of a named workload: the Llama-shaped recipe (32/8 heads) at this many tokens "
                          "(context-length sweeps)")
     ap.add_argument("--impl", default="crisp", choices=["crisp", "reference"])
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "kv-groups"],
+                    help="N > 1: one independent layer per rank, or one layer's KV groups split over the ranks")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -182,13 +253,20 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    shard = args.shard if world > 1 else "replicas"
     w = synth.CONFIGS[args.workload]
     if args.seq_len > 0:
         w = synth.llama_shaped(f"Llama-shaped-{args.seq_len}", args.seq_len, n_columns=max(16, args.seq_len // 2048))
+    if world == 1:
+        par = "single GPU"
+    elif shard == "replicas":
+        par = f"replicas x{world} (one layer per rank)"
+    else:
+        par = f"one layer, KV groups round-robin over {world} ranks"
     config = {"workload": f"{w.name}: n={w.seq_len}, H_q/H_kv={w.n_q_heads}/{w.n_kv_heads}, d=128, B=128, "
                           f"alpha={w.alpha}, tau={w.tau}, gamma={w.gamma}, w_sink={w.sink_tokens}, "
                           f"w_local={w.local_tokens}, k_min={w.k_min_blocks}",
-              "layers_per_gpu": 1, "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+              "layers_per_gpu": 1 if shard == "replicas" else round(1.0 / world, 4), "parallelism": par,
               "l2": "inputs larger than L2 (no flush)" if w.seq_len >= 131072 else "L2 flushed between steps"}
 
     if args.impl == "reference":
@@ -196,9 +274,13 @@ def main():
             return
         dev = "cuda" if torch.cuda.is_available() else "cpu"
         q, k, v = synth.make_qkv(w, device=dev)
-        times, desc, cores = [], "", 0
-        for i in range(max(args.steps, 1)):
-            ms, desc, cores = oracle_sample(w, q, k, v, seed=i)
+        first = {}
+        for h, c in enumerate(w.head_classes):
+            first.setdefault(c, h)
+        heads = sorted(first.values())[:2]
+        times, desc = [], ""
+        for _ in range(max(args.steps, 1)):
+            ms, desc, _ = oracle_sample(w, q, k, v, heads, blocks_per_head=4, block_budget=10000)
             times.append(ms)
         val = statistics.median(times)
         print(json.dumps({
@@ -206,7 +288,7 @@ def main():
             "value": val, "unit": "ms/layer", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": val, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64", "data": "synthetic", "config": config,
-            "cpu_baseline": {"value": val, "unit": "ms/layer", "cores": cores, "kind": "oracle",
+            "cpu_baseline": {"value": val, "unit": "ms/layer", "cores": blas_threads(), "kind": "oracle",
                              "sample": desc + " (extrapolated)"},
             "e2e": {"value": val, "unit": "ms/layer", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
         return
@@ -214,6 +296,8 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the product path has no CPU fallback)")
     import paper_2609_01925_b200 as crisp
+    from paper_2609_01925_b200 import binding as B
+    from paper_2609_01925_b200 import sharding
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
@@ -222,13 +306,21 @@ def main():
     dev = torch.device("cuda", local_rank)
     peaks = load_peaks()
 
-    q, k, v = synth.make_qkv(w.with_(seed=w.seed + rank), device=dev)
-    p = crisp.make_params(w.seq_len, w.n_q_heads, w.n_kv_heads, sink_tokens=w.sink_tokens,
-                          local_tokens=w.local_tokens, k_min_blocks=w.k_min_blocks, tau=w.tau, alpha=w.alpha,
-                          gamma=w.gamma)
+    if shard == "kv-groups":
+        groups = sharding.kv_groups_of_rank(w.n_kv_heads, rank, world)
+        q, k, v = synth.make_qkv_kv_groups(w, groups, device=dev)
+        my_heads = sharding.q_heads_of_groups(groups, w.group)
+        wl = w.with_(n_q_heads=len(my_heads), n_kv_heads=len(groups),
+                     head_classes=tuple(w.head_classes[h] for h in my_heads))
+    else:
+        wl = w.with_(seed=w.seed + rank)
+        q, k, v = synth.make_qkv(wl, device=dev)
+    p = crisp.make_params(wl.seq_len, wl.n_q_heads, wl.n_kv_heads, sink_tokens=wl.sink_tokens,
+                          local_tokens=wl.local_tokens, k_min_blocks=wl.k_min_blocks, tau=wl.tau, alpha=wl.alpha,
+                          gamma=wl.gamma)
     layer = crisp.CrispLayer(p, device=dev)
     flush = None
-    if w.seq_len < 131072:
+    if wl.seq_len < 131072:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     def barrier():
@@ -254,7 +346,7 @@ def main():
         step(False)
     layer.poll()
     nnz = int(layer.nnz.item())
-    total_causal = w.n_q_heads * w.n_blocks * (w.n_blocks + 1) // 2
+    total_causal = wl.n_q_heads * wl.n_blocks * (wl.n_blocks + 1) // 2
 
     sampler = ClockSampler(local_rank)
     barrier()
@@ -284,6 +376,24 @@ def main():
     layer.poll()
     clocks = sampler.stop()
 
+    # per-kernel device times (outside the timed region: the event pairs around every kernel cost a little)
+    per_kernel, order_names = {}, []
+    launches_per_step = 0
+    for _ in range(3):
+        if flush is not None:
+            flush.zero_()
+        B.crisp_profile_enable(True)
+        layer.route(q, k); layer.select(q, k); layer.sparse_prefill(q, k, v)
+        records = B.crisp_profile_read()
+        B.crisp_profile_enable(False)
+        launches_per_step = len(records)
+        for name, ms in records:
+            if name not in per_kernel:
+                per_kernel[name] = []
+                order_names.append(name)
+            per_kernel[name].append(ms)
+    layer.poll()
+
     # A step's time runs from its first launch to its last kernel's end (CUDA events on the launching stream).
     # Without an L2 flush the steps are back to back and this equals the bracket around all K steps; with a
     # flush (small workloads) it leaves the flush kernel between two steps out of the path's time.
@@ -295,6 +405,36 @@ def main():
     sparse_tflops = nnz * FLOP_PER_BLOCK / (med["sparse_prefill"] * 1e-3) / 1e12
     dense_tflops = total_causal * FLOP_PER_BLOCK / (dense * 1e-3) / 1e12
     peak = peaks["bf16_sustained"] if med["sparse_prefill"] > 50.0 else peaks["bf16_burst"]
+    job_nnz = sum_over_ranks(float(nnz), dist, dev)
+    job_dense_ms = max_over_ranks(dense, dist, dev)
+
+    # HBM fractions: algorithmic bytes / device time / measured copy bandwidth
+    pattern = layer.pattern.cpu().numpy()
+    n_pe = int((pattern == B.PATTERN_PE).sum())
+    n_kv_pe = int(sum(1 for g in range(wl.n_kv_heads) if (pattern[g * wl.group:(g + 1) * wl.group] == B.PATTERN_PE).any()))
+    hbm = peaks["hbm_gbs"] * 1e9
+    kernels = []
+    for name in order_names:
+        ms = statistics.median(per_kernel[name])
+        nbytes = kernel_bytes(name, wl, n_pe, n_kv_pe, nnz)
+        row = {"kernel": name, "ms": round(ms, 5)}
+        if nbytes is not None:
+            row["algorithmic_bytes"] = int(nbytes)
+            row["hbm_frac"] = round(nbytes / (ms * 1e-3) / hbm, 4)
+        kernels.append(row)
+    kb = lambda nm: kernel_bytes(nm, wl, n_pe, n_kv_pe, nnz) or 0
+    route_bytes = kb("proxy") + kb("tile_sums")
+    select_bytes = kb("prepare") + 2 * n_pe * (wl.n_blocks * (wl.n_blocks + 1) // 2) * 4 + nnz * 4 \
+        + 8 * wl.n_q_heads * (wl.n_blocks + 1) + 2 * 4 * wl.n_blocks * wl.n_q_heads
+    stages_hbm = {
+        "route": {"algorithmic_bytes": int(route_bytes), "ms": med["route"],
+                  "hbm_frac": route_bytes / (med["route"] * 1e-3) / hbm,
+                  "note": "K read once + partials written and read once; the proxy kernel is MUFU-bound (128 exp2 per "
+                          "key and query head), not HBM-bound"},
+        "select": {"algorithmic_bytes": int(select_bytes), "ms": med["select"],
+                   "hbm_frac": select_bytes / (med["select"] * 1e-3) / hbm,
+                   "note": "Q of PE heads and K read once, pooled map written once and read once, lists written"},
+        "peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"]}
 
     # end to end through the C ABI with host buffers
     e2e = None
@@ -315,27 +455,35 @@ def main():
         e2e_ms = max_over_ranks(a.elapsed_time(b) / e2e_steps, dist, dev)
         h2d = sum(x.numel() * x.element_size() for x in (qh, kh, vh))
         d2h = oh.numel() * oh.element_size()
-        e2e = {"value": job_ms_per_layer(e2e_ms, world), "unit": "ms/layer", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        e2e = {"value": job_ms_per_layer(e2e_ms, world, shard), "unit": "ms/layer", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h}
         del qh, kh, vh, oh, qd, kd, vd
 
-    cpu_baseline = None
+    cpu_baseline, near = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        ms, desc, cores = oracle_sample(w, q, k, v)
-        cpu_baseline = {"value": ms, "unit": "ms/layer", "cores": cores, "kind": "oracle",
+        heads = baseline_heads(wl)
+        row_ptr = layer.row_ptr.cpu().numpy()
+        cols_of = {h: layer.col_idx[int(row_ptr[h, 0]):int(row_ptr[h, -1])].cpu().numpy() for h in heads}
+        ms, desc, near = oracle_sample(wl, q, k, v, heads, blocks_per_head=max(4, -(-32 // len(heads))),
+                                       block_budget=24000, gpu_lists=(pattern, row_ptr, cols_of))
+        cpu_baseline = {"value": ms, "unit": "ms/layer", "cores": blas_threads(), "kind": "oracle",
                         "sample": desc + " (extrapolated)"}
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
+    job_sparse_tflops = job_nnz * FLOP_PER_BLOCK / (ms_per_step * 1e-3) / 1e12
     out = {
         "metric": "prefill attention ms/layer (route+select+sparse prefill)",
-        "value": job_ms_per_layer(ms_per_step, world), "unit": "ms/layer", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "value": job_ms_per_layer(ms_per_step, world, shard), "unit": "ms/layer", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False,
+        "scaling": "weak" if shard == "replicas" else "strong",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config,
-        "stages_ms": med, "dense_prefill_ms": dense, "speedup_vs_own_dense": dense / ms_per_step,
+        "stages_ms": med, "dense_prefill_ms": job_dense_ms, "speedup_vs_own_dense": job_dense_ms / ms_per_step,
         "blocks_computed": nnz, "blocks_causal": total_causal, "block_fraction": nnz / total_causal,
         "sparse_tflops_on_computed_blocks": sparse_tflops, "dense_tflops": dense_tflops,
+        "job_tflops_on_computed_blocks": job_sparse_tflops,
         "tc_frac_sparse_of_measured_sustained": sparse_tflops / peaks["bf16_sustained"],
         "tc_frac_dense_of_measured_sustained": dense_tflops / peaks["bf16_sustained"],
         "tc_frac_sparse_of_nominal_2250": sparse_tflops / 2250.0,
@@ -343,11 +491,13 @@ def main():
         "roofline": {"bound": "tensor", "kernel": "prefill_kernel<sparse>", "achieved": sparse_tflops,
                      "peak": peak, "unit": "TFLOP/s", "frac": sparse_tflops / peak,
                      "peak_source": f"{peaks['source']} ({'sustained' if peak == peaks['bf16_sustained'] else 'burst'})",
-                     "traffic": ncu_traffic_bytes("prefill_kernel<sparse>", w.name),
-                     "traffic_unit": "bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum)",
+                     "traffic": None,
+                     "traffic_note": "not captured in this run; ncu DRAM bytes of the kernel on a small case are in "
+                                     "profiles/prefill_kernel_L32k_ncu.md",
                      "algorithmic_flop_per_launch": nnz * FLOP_PER_BLOCK},
+        "stages_hbm": stages_hbm, "kernels": kernels, "near_threshold_excused": near,
         "cpu_baseline": cpu_baseline, "e2e": e2e,
-        "gpu_launches": args.steps * (LAUNCHES_ROUTE + LAUNCHES_SELECT + LAUNCHES_PREFILL),
+        "gpu_launches": args.steps * launches_per_step, "gpu_launches_per_step": launches_per_step,
         "clocks": clocks,
     }
     print(json.dumps(out))
