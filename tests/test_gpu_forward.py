@@ -94,3 +94,22 @@ def test_forward_replays_from_a_cuda_graph():
     torch.cuda.synchronize()
     layer.poll()
     assert torch.equal(layer.o, ref)
+
+
+def test_per_kernel_profile_records():
+    """crisp_profile_enable / crisp_profile_read: one record per kernel the stage calls launch, in launch order,
+    with positive device times; nothing is recorded while profiling is off."""
+    w, p, q, k, v = _setup()
+    layer = crisp.CrispLayer(p)
+    layer.route(q, k); layer.select(q, k); layer.sparse_prefill(q, k, v); layer.poll()
+    B.crisp_profile_enable(True)
+    layer.route(q, k); layer.select(q, k); layer.sparse_prefill(q, k, v)
+    recs = B.crisp_profile_read()
+    B.crisp_profile_enable(False)
+    names = [n for n, _ in recs]
+    assert names[:2] == ["proxy", "tile_sums"] and names[-1] == "prefill_sparse" and "fill" in names
+    assert len(names) == 13
+    assert all(ms > 0 for _, ms in recs)
+    layer.route(q, k)
+    assert B.crisp_profile_read() == []
+    layer.poll()
