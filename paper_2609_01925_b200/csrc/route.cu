@@ -81,12 +81,17 @@ struct ProxySmem {
 // Persistent CTAs, one per SM.  A CTA owns up to four query heads of one KV group - their 128 proxy queries
 // are loaded once and stay in shared memory - and walks over every gridDim.x-th key tile: TMA brings the K
 // tile in (two buffers, the load of the tile after next is issued while the current one is worked on), one
-// thread issues a 128 x 128 x 128 tcgen05 MMA per head into one of four TMEM buffers, and two groups of four
-// warps (one thread per proxy row; group 0 takes the even heads, group 1 the odd ones) reduce the logits to the
-// tile partials.  Two warps per scheduler keep the MUFU busy while the other loads its logits from TMEM.
+// thread issues a 128 x 128 x 128 tcgen05 MMA per head into that head's TMEM buffer, and four groups of four
+// warps (one group per head, one thread per proxy row) reduce the logits to the tile partials.  The row threads
+// wait on the latencies of their own chain (TMEM load, row maximum, dependent exp2 / add pairs), not on MUFU
+// throughput, so what counts is the number of warps per scheduler: a thread reads its row in two halves of 64
+// keys - half a row of registers - which lets four warps per scheduler fit (the maximum needs a first pass over
+// both halves; the second half stays in registers for the sums, the first is read again).
 // kRagged: n is not a multiple of 128 (third band possible); the aligned instantiation drops its predicates.
+constexpr int kProxyThreads = 32 * (4 * kProxyHeads + 1);
+
 template <bool kRagged>
-__global__ void __launch_bounds__(288, 1)
+__global__ void __launch_bounds__(kProxyThreads, 1)
 proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const Dims d, const RoutePtrs w, int* status, int n_head_chunks) {
   extern __shared__ uint8_t smem_raw[];
@@ -97,6 +102,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   const int gc = min(kProxyHeads, G - g0);            // heads of this CTA
   const int stride = gridDim.x;
   const int n_my_tiles = static_cast<int>(blockIdx.x) < d.nb ? (d.nb - 1 - static_cast<int>(blockIdx.x)) / stride + 1 : 0;
+  constexpr int kIssuerWarp = 4 * kProxyHeads;
 
   if (tid == 0) {
     s.abort_flag = 0;
@@ -111,7 +117,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     }
     fence_mbar_init();
   }
-  if (warp == 8) {
+  if (warp == kIssuerWarp) {
     tmem_alloc(&s.tmem_base, 512);
     tmem_relinquish();
   }
@@ -119,10 +125,8 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tm = s.tmem_base;
-  // jobs (tile, head) of group gr per tile: the even heads for group 0, the odd ones for group 1
-  const int jobs0 = (gc + 1) >> 1, jobs1 = gc >> 1;
 
-  if (warp == 8) {
+  if (warp == kIssuerWarp) {
     if (lane == 0 && n_my_tiles > 0) {
       // ---- producer + MMA issuer
       prefetch_tmap(&tmap_q);
@@ -148,10 +152,8 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
         const int kb = n & 1;
         ok = mbar_wait(&s.bar_k_full[kb], (n >> 1) & 1, &s.abort_flag);
         for (int g = 0; g < gc && ok; ++g) {
-          const int gr = g & 1;
-          const int job = n * (gr ? jobs1 : jobs0) + (g >> 1);  // running job number of the group
-          const int buf = gr * 2 + (job & 1), use = job >> 1;
-          if (use > 0) ok = mbar_wait(&s.bar_s_free[buf], (use - 1) & 1, &s.abort_flag);
+          // head g's logits go to TMEM buffer g, which its group has finished reading for the previous tile
+          if (n > 0) ok = mbar_wait(&s.bar_s_free[g], (n - 1) & 1, &s.abort_flag);
           if (!ok) break;
           tc_fence_after_sync();
           // descriptors: only the 14-bit start-address field moves (head: +32 KB, buffer: +32 KB, K step kk:
@@ -161,9 +163,9 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
           for (int kk = 0; kk < 8; ++kk) {
             constexpr uint32_t kHalf = 16384 >> 4, kStep = 32 >> 4;
             const uint64_t off = static_cast<uint64_t>((kk >> 2) * kHalf + (kk & 3) * kStep);
-            umma_ss(tm + buf * 128, ad0 + off, bd0 + off, idesc, kk > 0);
+            umma_ss(tm + g * 128, ad0 + off, bd0 + off, idesc, kk > 0);
           }
-          umma_commit(&s.bar_s_full[buf]);
+          umma_commit(&s.bar_s_full[g]);
           // As early in this tile as the pipe allows, refill the other buffer (the previous tile's, whose MMAs
           // were issued a whole tile ago) with the next tile, so its latency hides behind this tile's work.
           if (g == 0 && n >= 1 && n + 1 < n_my_tiles) {
@@ -176,8 +178,8 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       }
     }
     __syncwarp();
-  } else {
-    // ---- one thread per proxy row; group 0 = warps 0-3, group 1 = warps 4-7
+  } else if ((warp >> 2) < gc) {
+    // ---- one thread per proxy row; group gr = warps 4 gr .. 4 gr + 3 takes head gr of the CTA
     const int gr = warp >> 2;
     const int i = tid & 127;
     const int wq = warp & 3;  // warp within the group = TMEM sub-partition = rows 32 wq .. 32 wq + 31
@@ -187,12 +189,11 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     // ("hi": jl <= i + rho - 128, possible only when rho > 0).  A band with a negative offset is invisible.
     const int a_thr = i + d.rho;           // jl <= a_thr  <=>  not in the "up" band
     const int b_thr = i + d.rho - kBlock;  // jl <= b_thr  <=>  in the "hi" band
-    const uint32_t lane_addr = static_cast<uint32_t>(wq * 32) << 16;
-    const int my_jobs = gr ? jobs1 : jobs0;
-    int job = 0;
+    const uint32_t s_addr = tm + (static_cast<uint32_t>(wq * 32) << 16) + gr * 128;
+    const int h = kvh * G + g0 + gr;
     bool ok = true;
-    // running maximum and sum of this row over the CTA's tiles, per head of the group (two at most)
-    float run_m[2] = {-INFINITY, -INFINITY}, run_l[2] = {0.f, 0.f};
+    // running maximum and sum of this row over the CTA's tiles
+    float run_m = -INFINITY, run_l = 0.f;
     for (int n = 0; n < n_my_tiles && ok; ++n) {
       const int J = blockIdx.x + n * stride;
       const int qoff = d.nfull - 1 - J;
@@ -201,49 +202,74 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       const int jl = min(max(d.n - d.w_local - J * kBlock, 0), kBlock);  // anchor: local key >= jl
       const bool has_slot = (J < d.n_sink_tiles) || (J >= d.first_local_tile);
       const int slot = (J < d.n_sink_tiles) ? J : d.n_sink_tiles + (J - d.first_local_tile);
-      for (int gj = 0; gj < my_jobs; ++gj, ++job) {
-        const int g = 2 * gj + gr;
-        const int buf = gr * 2 + (job & 1), use = job >> 1;
-        if (!mbar_wait(&s.bar_s_full[buf], use & 1, &s.abort_flag)) {
-          ok = false;
-          break;
-        }
-        tc_fence_after_sync();
-        uint32_t r[4][32];
+      if (!mbar_wait(&s.bar_s_full[gr], n & 1, &s.abort_flag)) {
+        ok = false;
+        break;
+      }
+      tc_fence_after_sync();
+      const bool interior = !kRagged && vis_up;  // every key visible, band of key jl decided by jl <= i alone
+      uint32_t r[2][32];
+      // ---- first pass: the row maximum over the visible keys, half A (keys 0-63) then half B (64-127)
+      float mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld_x32(tm + lane_addr + buf * 128 + c * 32, r[c]);
+      for (int half = 0; half < 2; ++half) {
+        tmem_ld_x32(s_addr + half * 64, r[0]);
+        tmem_ld_x32(s_addr + half * 64 + 32, r[1]);
         tmem_ld_wait();
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s.bar_s_free[buf]);
-
-        float mx, lo = 0.f, up = 0.f, hi = 0.f, anc = 0.f;
-        bool any = true;
-        if (!kRagged && vis_up) {
-          // ---- interior tile of an aligned sequence (all but the last tile): every key is visible, and the
-          // band of key jl is decided by jl <= i alone.  Rows of warp w lie in [32 w, 32 w + 31], so a
-          // 32-key chunk c lies wholly on/below the diagonal for c < w and wholly above it for c > w: only
-          // the chunk c == w needs a per-key test.
+        if (interior) {
           float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
+          for (int c = 0; c < 2; ++c)
 #pragma unroll
             for (int t = 0; t < 32; t += 2) {
               m0 = fmaxf(m0, __uint_as_float(r[c][t]));
               m1 = fmaxf(m1, __uint_as_float(r[c][t + 1]));
             }
-          mx = fmaxf(m0, m1) * d.scale_log2;
+          mx = fmaxf(mx, fmaxf(m0, m1));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int t = 0; t < 32; ++t) {
+              const int j = half * 64 + c * 32 + t;
+              const bool visible = (kRagged && j <= b_thr) || (j <= a_thr ? vis_lo : vis_up);
+              if (visible) mx = fmaxf(mx, __uint_as_float(r[c][t]));
+            }
+        }
+      }
+      mx *= d.scale_log2;  // (the scale is positive)
+      // a row may see no key of this tile (ragged n: the tiles around the proxy block): leave a neutral partial
+      const bool any = mx > -INFINITY;
+      if (!any) mx = -1e30f;
+      float lo = 0.f, up = 0.f, hi = 0.f, anc = 0.f;
+      // ---- second pass: the sums, half B from the registers it is still in, then half A read again
+#pragma unroll
+      for (int pass = 0; pass < 2; ++pass) {
+        const int half = 1 - pass;
+        if (pass == 1) {
+          tmem_ld_x32(s_addr, r[0]);
+          tmem_ld_x32(s_addr + 32, r[1]);
+          tmem_ld_wait();
+          // the buffer has been read for good: the next tile's logits of this head may come in
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s.bar_s_free[gr]);
+        }
+        if (interior) {
+          // Rows of warp wq lie in [32 wq, 32 wq + 31], so a 32-key chunk c lies wholly on/below the diagonal
+          // for c < wq and wholly above it for c > wq: only the chunk c == wq needs a per-key test.
           const uint64_t scale2 = pack2f(d.scale_log2, d.scale_log2), negm2 = pack2f(-mx, -mx);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            uint64_t sa = pack2f(0.f, 0.f), sb = pack2f(0.f, 0.f);
+          for (int cc = 0; cc < 2; ++cc) {
+            const int c = 2 * half + cc;
             if (c != wq) {
               // the whole chunk lies in one band: packed fp32x2 arithmetic, no per-key test
+              uint64_t sa = pack2f(0.f, 0.f), sb = pack2f(0.f, 0.f);
 #pragma unroll
               for (int t = 0; t < 32; t += 4) {
                 float a0, a1, b0, b1;
-                unpack2f(fma2f(pack2f(__uint_as_float(r[c][t]), __uint_as_float(r[c][t + 1])), scale2, negm2), a0, a1);
-                unpack2f(fma2f(pack2f(__uint_as_float(r[c][t + 2]), __uint_as_float(r[c][t + 3])), scale2, negm2), b0, b1);
+                unpack2f(fma2f(pack2f(__uint_as_float(r[cc][t]), __uint_as_float(r[cc][t + 1])), scale2, negm2), a0, a1);
+                unpack2f(fma2f(pack2f(__uint_as_float(r[cc][t + 2]), __uint_as_float(r[cc][t + 3])), scale2, negm2), b0, b1);
                 sa = add2f(sa, pack2f(ex2(a0), ex2(a1)));
                 sb = add2f(sb, pack2f(ex2(b0), ex2(b1)));
               }
@@ -262,8 +288,8 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
               float d0 = 0.f, d1 = 0.f, u0 = 0.f, u1 = 0.f;
 #pragma unroll
               for (int t = 0; t < 32; t += 2) {
-                const float e0 = ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
-                const float e1 = ex2(fmaf(__uint_as_float(r[c][t + 1]), d.scale_log2, -mx));
+                const float e0 = ex2(fmaf(__uint_as_float(r[cc][t]), d.scale_log2, -mx));
+                const float e1 = ex2(fmaf(__uint_as_float(r[cc][t + 1]), d.scale_log2, -mx));
                 d0 += t <= il ? e0 : 0.f;
                 u0 += t <= il ? 0.f : e0;
                 d1 += t + 1 <= il ? e1 : 0.f;
@@ -274,66 +300,50 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
             }
           }
           if (has_slot) {
-            // the few tiles that hold anchor keys (sinks, the local window) take a second pass for their sum
+            // the few tiles that hold anchor keys (sinks, the local window) take another pass for their sum
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int cc = 0; cc < 2; ++cc)
 #pragma unroll
               for (int t = 0; t < 32; ++t) {
-                const int j = c * 32 + t;
-                if (j < js || j >= jl) anc += ex2(fmaf(__uint_as_float(r[c][t]), d.scale_log2, -mx));
+                const int j = half * 64 + cc * 32 + t;
+                if (j < js || j >= jl) anc += ex2(fmaf(__uint_as_float(r[cc][t]), d.scale_log2, -mx));
               }
           }
         } else {
-        mx = -INFINITY;
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+          for (int cc = 0; cc < 2; ++cc)
 #pragma unroll
-          for (int t = 0; t < 32; ++t) {
-            const int j = c * 32 + t;
-            const float x = __uint_as_float(r[c][t]) * d.scale_log2;
-            r[c][t] = __float_as_uint(x);
-            const bool visible = (kRagged && j <= b_thr) || (j <= a_thr ? vis_lo : vis_up);
-            if (visible) mx = fmaxf(mx, x);
-          }
-        // a row may see no key of this tile (ragged n: the tiles around the proxy block): leave a neutral partial
-        any = mx > -INFINITY;
-        if (!any) mx = -1e30f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int t = 0; t < 32; ++t) {
-            const int j = c * 32 + t;
-            const float e = ex2(__uint_as_float(r[c][t]) - mx);
-            const bool in_hi = kRagged && j <= b_thr, in_lo = !in_hi && j <= a_thr, in_up = j > a_thr;
-            const bool visible = in_hi || (in_lo && vis_lo) || (in_up && vis_up);
-            hi += in_hi ? e : 0.f;
-            lo += (in_lo && vis_lo) ? e : 0.f;
-            up += (in_up && vis_up) ? e : 0.f;
-            anc += (visible && (j < js || j >= jl)) ? e : 0.f;
-          }
+            for (int t = 0; t < 32; ++t) {
+              const int j = half * 64 + cc * 32 + t;
+              const float e = ex2(fmaf(__uint_as_float(r[cc][t]), d.scale_log2, -mx));
+              const bool in_hi = kRagged && j <= b_thr, in_lo = !in_hi && j <= a_thr, in_up = j > a_thr;
+              const bool visible = in_hi || (in_lo && vis_lo) || (in_up && vis_up);
+              hi += in_hi ? e : 0.f;
+              lo += (in_lo && vis_lo) ? e : 0.f;
+              up += (in_up && vis_up) ? e : 0.f;
+              anc += (visible && (j < js || j >= jl)) ? e : 0.f;
+            }
         }
-        if (!any) lo = up = hi = anc = 0.f;
-        {
-          const float sum = lo + up + hi;
-          const float nm = fmaxf(run_m[gj & 1], mx);
-          run_l[gj & 1] = run_l[gj & 1] * ex2(run_m[gj & 1] - nm) + sum * ex2(mx - nm);
-          run_m[gj & 1] = nm;
-        }
-        const int h = kvh * G + g0 + g;
-        const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
-        w.pm[off] = mx;
-        w.plo[off] = lo;
-        w.pup[off] = up;
-        if (kRagged) w.phi[off] = hi;
-        if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
       }
+      if (!any) lo = up = hi = anc = 0.f;
+      {
+        const float sum = lo + up + hi;
+        const float nm = fmaxf(run_m, mx);
+        run_l = run_l * ex2(run_m - nm) + sum * ex2(mx - nm);
+        run_m = nm;
+      }
+      const size_t off = (static_cast<size_t>(h) * d.nb + J) * kBlock + i;
+      w.pm[off] = mx;
+      w.plo[off] = lo;
+      w.pup[off] = up;
+      if (kRagged) w.phi[off] = hi;
+      if (has_slot) w.panc[(static_cast<size_t>(h) * d.n_anchor_slots + slot) * kBlock + i] = anc;
     }
     // this CTA's share of the row statistics
-    for (int gj = 0; gj < my_jobs; ++gj) {
-      const int h = kvh * G + g0 + 2 * gj + gr;
+    {
       const size_t o = (static_cast<size_t>(h) * w.n_slices + blockIdx.x) * kBlock + i;
-      w.cm[o] = run_m[gj];
-      w.cl[o] = run_l[gj];
+      w.cm[o] = run_m;
+      w.cl[o] = run_l;
     }
   }
   tc_fence_before_sync();
@@ -343,7 +353,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     if (s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
     s.is_last = atomicAdd(&w.group_done[blockIdx.y], 1) == static_cast<int>(gridDim.x) - 1;
   }
-  if (warp == 8) tmem_dealloc(tm, 512);
+  if (warp == kIssuerWarp) tmem_dealloc(tm, 512);
   __syncthreads();
   if (!s.is_last) return;
   // The last CTA of the group to finish merges the per-CTA statistics (written by other CTAs: read from L2)
@@ -524,7 +534,7 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "route: SM count");
   ProxyGrid g = proxy_grid(d, n_sm);
   if (g.slices > w.n_slices) g.slices = w.n_slices;
-  CRISP_KERNEL("proxy", stream, proxy<<<dim3(g.slices, g.groups), 288, smem, stream>>>(tq, tk, d, w, status, g.n_head_chunks));
+  CRISP_KERNEL("proxy", stream, proxy<<<dim3(g.slices, g.groups), kProxyThreads, smem, stream>>>(tq, tk, d, w, status, g.n_head_chunks));
   CRISP_KERNEL("tile_sums", stream, tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v, p_s, c_struct, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route: launch");
   return CRISP_OK;
