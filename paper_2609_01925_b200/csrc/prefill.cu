@@ -809,32 +809,37 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
 // Counting sort of the items by (KV head, decreasing cost).  Grouping by KV head keeps the CTAs that
 // run at the same time on the same K/V blocks (L2 reuse); sorting by cost inside a group lets the
 // dynamic hand-out start the long lists (PE heads) before the short ones (VS heads).
-__global__ void __launch_bounds__(1024) sched_scan_kernel(int* __restrict__ cost_hist, int n_bins) {
-  __shared__ long long scratch[33];
-  const int tid = threadIdx.x;
-  const int seg = (n_bins + 1023) / 1024;
-  const int b0 = min(tid * seg, n_bins), b1 = min(b0 + seg, n_bins);
-  int local = 0;
-  for (int i = b0; i < b1; ++i) local += cost_hist[i];
-  int run = static_cast<int>(block_exclusive_scan_1024(local, scratch, nullptr));
-  for (int i = b0; i < b1; ++i) {
-    const int c = cost_hist[i];
-    cost_hist[i] = run;  // first position of this key in the sorted order
-    run += c;
-  }
-}
-
+// One thread per pair.  Every CTA first turns the histogram of its own segment (the keys of its KV head; all
+// keys when the order is global) into first positions in shared memory - a segment holds a known number of
+// items, so its base needs no other segment - and then places its items with one atomic each on a cursor array.
 __global__ void __launch_bounds__(256)
-sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, int* __restrict__ cost_hist,
-                     int* __restrict__ order, int n_pairs, int n_cost, int group_kv,
+sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int* __restrict__ cost_hist,
+                     int* __restrict__ cursor, int* __restrict__ order, int n_pairs, int n_cost, int group_kv,
                      const int* __restrict__ gate, const int* __restrict__ status) {
-  const int u = blockIdx.x * blockDim.x + threadIdx.x, h = blockIdx.y;
-  if (u >= n_pairs || (gate != nullptr && *gate != 0)) return;
+  extern __shared__ int first_pos[];  // [n_cost]
+  __shared__ long long scratch[33];
+  if (gate != nullptr && *gate != 0) return;
   if (*status != 0) return;  // a list failed validation: its row lengths cannot be trusted as histogram keys
+  const int tid = threadIdx.x, h = blockIdx.y;
+  const int seg = group_kv ? h / d.group : 0;
+  const int* hist = cost_hist + static_cast<size_t>(seg) * n_cost;
+  const int per = (n_cost + 255) / 256;
+  const int b0 = min(tid * per, n_cost), b1 = min(b0 + per, n_cost);
+  int local = 0;
+  for (int i = b0; i < b1; ++i) local += hist[i];
+  int run = static_cast<int>(block_exclusive_scan<256>(local, scratch, nullptr));
+  for (int i = b0; i < b1; ++i) {
+    first_pos[i] = run;
+    run += hist[i];
+  }
+  __syncthreads();
+  const int u = blockIdx.x * blockDim.x + tid;
+  if (u >= n_pairs) return;
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int m0 = 2 * u, mend = min(2 * u + 2, d.nb);
-  const int cost = static_cast<int>(rp[mend] - rp[m0]);
-  const int pos = atomicAdd(&cost_hist[(group_kv ? h / d.group : 0) * n_cost + (n_cost - 1 - cost)], 1);
+  const int bin = n_cost - 1 - static_cast<int>(rp[mend] - rp[m0]);
+  const int base = group_kv ? seg * n_pairs * d.group : 0;
+  const int pos = base + first_pos[bin] + atomicAdd(&cursor[static_cast<size_t>(seg) * n_cost + bin], 1);
   order[pos] = (n_pairs - 1 - u) * d.hq + h;
 }
 
@@ -842,6 +847,7 @@ struct PrefillWs {
   int* item_len;
   int* order;
   int* cost_hist;
+  int* cursor;  // per sort key: items placed so far
   int n_cost;  // distinct cost values (0 .. 2 N_b + 1)
   int n_bins;  // n_cost per KV head
   size_t zero_bytes;  // header + histogram
@@ -853,10 +859,12 @@ PrefillWs carve(const Dims& d, void* ws, size_t* total) {
   uint8_t* base = static_cast<uint8_t*>(ws);
   size_t off = kWsHeader;
   const int n_pairs = (d.nb + 1) / 2;
-  // the histogram sits directly behind the header: one memset clears both
+  // the histogram and the cursors sit directly behind the header: one memset clears all three
   w.n_cost = 2 * d.nb + 2;
   w.n_bins = w.n_cost * d.hkv;
   w.cost_hist = reinterpret_cast<int*>(base + off);
+  off += align_up(sizeof(int) * static_cast<size_t>(w.n_bins), 256);
+  w.cursor = reinterpret_cast<int*>(base + off);
   off += align_up(sizeof(int) * static_cast<size_t>(w.n_bins), 256);
   w.zero_bytes = off;
   w.item_len = reinterpret_cast<int*>(base + off);
@@ -924,10 +932,14 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
                                                        stream>>>(
         d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate, a.status,
         static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2));
-    CRISP_KERNEL("sched_scan", stream, sched_scan_kernel<<<1, 1024, 0, stream>>>(w.cost_hist, w.n_bins));
-    CRISP_KERNEL("sched_scatter", stream, sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, 0, stream>>>(d, row_ptr, w.cost_hist,
-                                                                               w.order, a.n_pairs, w.n_cost, a.group_kv, gate,
-                                                                               a.status));
+    const size_t scatter_smem = sizeof(int) * static_cast<size_t>(w.n_cost);
+    if (scatter_smem > 48 * 1024)
+      CRISP_CUDA_TRY(cudaFuncSetAttribute(sched_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(scatter_smem)),
+                     "prefill: scatter smem attribute");
+    CRISP_KERNEL("sched_scatter", stream,
+                 sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, scatter_smem, stream>>>(
+                     d, row_ptr, w.cost_hist, w.cursor, w.order, a.n_pairs, w.n_cost, a.group_kv, gate, a.status));
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
