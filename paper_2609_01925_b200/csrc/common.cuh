@@ -2,6 +2,7 @@
 #pragma once
 #include <cstddef>
 #include <cstdint>
+#include <utility>
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
@@ -65,12 +66,39 @@ struct ProfScope {
     if (on) prof_end(stream);
   }
 };
-// CRISP_KERNEL("name", stream, kernel<<<grid, block, smem, stream>>>(args));
+// CRISP_KERNEL("name", stream, launch_pdl(kernel, grid, block, smem, stream, args...));
 #define CRISP_KERNEL(name, stream, ...)          \
   do {                                           \
     ::crisp::ProfScope prof_scope__(name, stream); \
     __VA_ARGS__;                                 \
   } while (0)
+
+#ifdef __CUDACC__
+// Launch with programmatic dependent launch allowed: the kernel's CTAs may become resident while the kernel
+// before it on the stream is still running.  Every kernel launched this way calls pdl_enter() as its first
+// statement, which lets the kernel after it do the same and then waits until the kernel before it has
+// completed and its writes are visible, so the stream's order is kept; what is saved is the launch latency
+// between two short kernels.  (A kernel that follows a memset or an event record simply starts after it.)
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                       Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr = {};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(std::forward<Args>(args))...);  // errors: cudaGetLastError
+}
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+#endif
 
 #ifdef __CUDACC__
 // Exclusive prefix sum over the kThreads threads of a block (a multiple of 32, at most 1024), in thread order

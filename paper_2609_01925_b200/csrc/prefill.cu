@@ -3,7 +3,9 @@
 // One CTA processes work items; an item is one query head and a PAIR of adjacent query blocks
 // (two 128-row tiles).  Both tiles share every K/V block that TMA brings into shared memory, which
 // halves the L2 -> shared-memory traffic per flop.  The key blocks of the pair are the sorted union
-// of the two blocks' lists; each entry carries two flags saying which tile uses it.
+// of the two blocks' lists; each entry carries two flags saying which tile uses it.  (When the pairs of a problem
+// do not even fill the SMs, an item is a single query block instead: tile 1 stays idle, the CTAs are twice as many
+// and a block alone steps faster than a pair.)
 //
 // Warp roles (384 threads):
 //   warps 0-3   softmax of tile 0 (one thread per query row; TMEM lanes 0-127)
@@ -52,7 +54,8 @@ struct PrefillArgs {
   __nv_bfloat16* o;        // [n][hq][128]
   float* lse;              // [hq][n] or null
   int* status;
-  int n_pairs;
+  int n_pairs;             // items per head
+  int rows_per_item;       // 2: an item is a pair of query blocks; 1: a single block (small problems)
   int n_items;
   int group_kv;            // 1: schedule one KV head at a time, 0: one global order by cost (small problems)
   const int* gate;         // optional device word: when non-zero the lists are invalid and nothing is done
@@ -100,9 +103,9 @@ __device__ __forceinline__ Item decode_item(int pos, const Dims& d, const Prefil
   it.h = idx % d.hq;
   const int u = a.n_pairs - 1 - idx / d.hq;  // long rows first
   it.kvh = it.h / d.group;
-  it.m0 = 2 * u;
-  it.m1 = 2 * u + 1;
-  it.tile1 = it.m1 < d.nb;
+  it.m0 = a.rows_per_item * u;
+  it.m1 = it.m0 + 1;
+  it.tile1 = a.rows_per_item == 2 && it.m1 < d.nb;
   if (kDense) {
     it.n_entries = it.tile1 ? it.m1 + 1 : it.m0 + 1;
     it.base = 0;
@@ -307,6 +310,7 @@ template <bool kDense>
 __global__ void __launch_bounds__(384, 1)
 prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                const __grid_constant__ CUtensorMap tmap_v, const Dims d, const PrefillArgs a) {
+  pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   PrefillSmem& s = *reinterpret_cast<PrefillSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -713,13 +717,13 @@ __device__ __forceinline__ void merge_pair(const Dims& d, const int64_t* __restr
                                            int* __restrict__ item_len, int* __restrict__ cost_hist, int n_pairs,
                                            int n_cost, int group_kv, int* __restrict__ status,
                                            long long merged_capacity, uint32_t* b0, uint32_t* b1, int words, int u,
-                                           int h, int lane) {
-  const int m0 = 2 * u, m1 = 2 * u + 1;
+                                           int h, int lane, int rows_per_item) {
+  const int m0 = rows_per_item * u, m1 = m0 + 1;
   for (int i = lane; i < 2 * words; i += 32) b0[i] = 0u;
   __syncwarp();
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int64_t s0 = rp[m0], e0 = rp[m0 + 1];
-  const bool has1 = m1 < d.nb;
+  const bool has1 = rows_per_item == 2 && m1 < d.nb;
   const int64_t e1 = has1 ? rp[m1 + 1] : e0;
   // The lists may come from the caller, so nothing about them is trusted: a row of query block m must hold
   // between 1 and m + 1 entries inside the workspace's range, strictly ascending, none above m, the last
@@ -769,7 +773,7 @@ __device__ __forceinline__ void merge_pair(const Dims& d, const int64_t* __restr
   int32_t* out = merged + s0;
   int written = 0;
   // one 32-block word per step, lane b owning bit b: the entries of a word go out as one contiguous store
-  const int last_word = min(words - 1, (m1 < d.nb ? m1 : m0) >> 5);
+  const int last_word = min(words - 1, (has1 ? m1 : m0) >> 5);
   for (int wd = 0; wd <= last_word; ++wd) {
     const uint32_t x0 = b0[wd], x1 = b1[wd];  // broadcast reads
     const uint32_t un = x0 | x1;
@@ -794,7 +798,8 @@ __global__ void __launch_bounds__(128)
 merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                    int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
                    int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate, int* __restrict__ status,
-                   long long merged_capacity) {
+                   long long merged_capacity, int rows_per_item) {
+  pdl_enter();
   extern __shared__ uint32_t bm[];
   if (gate != nullptr && *gate != 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -803,7 +808,7 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   uint32_t* b0 = bm + static_cast<size_t>(warp) * 2 * words;
   if (u < n_pairs)
     merge_pair(d, row_ptr, col_idx, merged, item_len, cost_hist, n_pairs, n_cost, group_kv, status, merged_capacity,
-               b0, b0 + words, words, u, h, lane);
+               b0, b0 + words, words, u, h, lane, rows_per_item);
 }
 
 // Counting sort of the items by (KV head, decreasing cost).  Grouping by KV head keeps the CTAs that
@@ -815,7 +820,8 @@ merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
 __global__ void __launch_bounds__(256)
 sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int* __restrict__ cost_hist,
                      int* __restrict__ cursor, int* __restrict__ order, int n_pairs, int n_cost, int group_kv,
-                     const int* __restrict__ gate, const int* __restrict__ status) {
+                     const int* __restrict__ gate, const int* __restrict__ status, int rows_per_item) {
+  pdl_enter();
   extern __shared__ int first_pos[];  // [n_cost]
   __shared__ long long scratch[33];
   if (gate != nullptr && *gate != 0) return;
@@ -836,7 +842,7 @@ sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const in
   const int u = blockIdx.x * blockDim.x + tid;
   if (u >= n_pairs) return;
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
-  const int m0 = 2 * u, mend = min(2 * u + 2, d.nb);
+  const int m0 = rows_per_item * u, mend = min(m0 + rows_per_item, d.nb);
   const int bin = n_cost - 1 - static_cast<int>(rp[mend] - rp[m0]);
   const int base = group_kv ? seg * n_pairs * d.group : 0;
   const int pos = base + first_pos[bin] + atomicAdd(&cursor[static_cast<size_t>(seg) * n_cost + bin], 1);
@@ -858,7 +864,7 @@ PrefillWs carve(const Dims& d, void* ws, size_t* total) {
   PrefillWs w;
   uint8_t* base = static_cast<uint8_t*>(ws);
   size_t off = kWsHeader;
-  const int n_pairs = (d.nb + 1) / 2;
+  const int n_pairs = d.nb;  // items per head at most (single-block items)
   // the histogram and the cursors sit directly behind the header: one memset clears all three
   w.n_cost = 2 * d.nb + 2;
   w.n_bins = w.n_cost * d.hkv;
@@ -899,7 +905,13 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   if (rc != CRISP_OK) return rc;
 
   PrefillArgs a;
-  a.n_pairs = (d.nb + 1) / 2;
+  int dev = 0, n_sm = 0;
+  CRISP_CUDA_TRY(cudaGetDevice(&dev), "prefill: device");
+  CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "prefill: SM count");
+  // An item is a pair of adjacent query blocks, which share every K/V block in shared memory.  When the pairs do
+  // not even fill the SMs, single blocks do better: twice the CTAs, and a block alone steps faster than a pair.
+  a.rows_per_item = ((d.nb + 1) / 2) * d.hq < n_sm ? 1 : 2;
+  a.n_pairs = (d.nb + a.rows_per_item - 1) / a.rows_per_item;
   a.n_items = a.n_pairs * d.hq;
   a.merged = w.merged;
   a.row_ptr = row_ptr;
@@ -915,9 +927,6 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   // the longest items of every head should start first.
   a.group_kv = 0;  // set below, once the SM count is known
 
-  int dev = 0, n_sm = 0;
-  CRISP_CUDA_TRY(cudaGetDevice(&dev), "prefill: device");
-  CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "prefill: SM count");
   const int grid = a.n_items < n_sm ? a.n_items : n_sm;
   a.group_kv = a.n_items >= 16 * n_sm ? 1 : 0;
   const size_t smem = sizeof(PrefillSmem) + 1024;
@@ -925,25 +934,24 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
-    CRISP_KERNEL("prefill_dense", stream, prefill_kernel<true><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a));
+    CRISP_KERNEL("prefill_dense", stream, launch_pdl(prefill_kernel<true>, dim3(grid), dim3(384), smem, stream, tq, tk, tv, d, a));
   } else {
     const int words = (d.nb + 31) / 32;
-    CRISP_KERNEL("merge_lists", stream, merge_lists_kernel<<<dim3((a.n_pairs + 3) / 4, d.hq), 128, sizeof(uint32_t) * 8 * words,
-                                                       stream>>>(
+    CRISP_KERNEL("merge_lists", stream, launch_pdl(merge_lists_kernel, dim3((a.n_pairs + 3) / 4, d.hq), dim3(128), sizeof(uint32_t) * 8 * words, stream, 
         d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate, a.status,
-        static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2));
+        static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2, a.rows_per_item));
     const size_t scatter_smem = sizeof(int) * static_cast<size_t>(w.n_cost);
     if (scatter_smem > 48 * 1024)
       CRISP_CUDA_TRY(cudaFuncSetAttribute(sched_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(scatter_smem)),
                      "prefill: scatter smem attribute");
     CRISP_KERNEL("sched_scatter", stream,
-                 sched_scatter_kernel<<<dim3((a.n_pairs + 255) / 256, d.hq), 256, scatter_smem, stream>>>(
-                     d, row_ptr, w.cost_hist, w.cursor, w.order, a.n_pairs, w.n_cost, a.group_kv, gate, a.status));
+                 launch_pdl(sched_scatter_kernel, dim3((a.n_pairs + 255) / 256, d.hq), dim3(256), scatter_smem, stream, 
+                     d, row_ptr, w.cost_hist, w.cursor, w.order, a.n_pairs, w.n_cost, a.group_kv, gate, a.status, a.rows_per_item));
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
-    CRISP_KERNEL("prefill_sparse", stream, prefill_kernel<false><<<grid, 384, smem, stream>>>(tq, tk, tv, d, a));
+    CRISP_KERNEL("prefill_sparse", stream, launch_pdl(prefill_kernel<false>, dim3(grid), dim3(384), smem, stream, tq, tk, tv, d, a));
   }
   CRISP_CUDA_TRY(cudaGetLastError(), "prefill: launch");
   return CRISP_OK;

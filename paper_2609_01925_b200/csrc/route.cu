@@ -94,6 +94,7 @@ template <bool kRagged>
 __global__ void __launch_bounds__(kProxyThreads, 1)
 proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                       const Dims d, const RoutePtrs w, int* status, int n_head_chunks) {
+  pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   ProxySmem& s = *reinterpret_cast<ProxySmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -386,6 +387,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 __global__ void __launch_bounds__(128) tile_sums_kernel(const Dims d, const RoutePtrs w, float* __restrict__ p_v,
                                                         float* __restrict__ p_s, float* __restrict__ c_struct,
                                                         int32_t* __restrict__ pattern) {
+  pdl_enter();
   const int h = blockIdx.y, chunk = blockIdx.x;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   float M[4], invl[4];
@@ -534,8 +536,8 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "route: SM count");
   ProxyGrid g = proxy_grid(d, n_sm);
   if (g.slices > w.n_slices) g.slices = w.n_slices;
-  CRISP_KERNEL("proxy", stream, proxy<<<dim3(g.slices, g.groups), kProxyThreads, smem, stream>>>(tq, tk, d, w, status, g.n_head_chunks));
-  CRISP_KERNEL("tile_sums", stream, tile_sums_kernel<<<dim3(w.n_chunks, d.hq), 128, 0, stream>>>(d, w, p_v, p_s, c_struct, pattern));
+  CRISP_KERNEL("proxy", stream, launch_pdl(proxy, dim3(g.slices, g.groups), dim3(kProxyThreads), smem, stream, tq, tk, d, w, status, g.n_head_chunks));
+  CRISP_KERNEL("tile_sums", stream, launch_pdl(tile_sums_kernel, dim3(w.n_chunks, d.hq), dim3(128), 0, stream, d, w, p_v, p_s, c_struct, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route: launch");
   return CRISP_OK;
 }

@@ -272,6 +272,7 @@ __global__ void __launch_bounds__(1024)
 prepare_kernel(const Dims d, const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k,
                const int32_t* __restrict__ pattern, const float* __restrict__ p_v, const float* __restrict__ p_s,
                const SelectPtrs w, int vs_ctas, int pool_all_k) {
+  pdl_enter();
   extern __shared__ uint8_t sm_raw[];
   const int tid = threadIdx.x;
   if (static_cast<int>(blockIdx.x) >= vs_ctas) {
@@ -378,6 +379,7 @@ __device__ __forceinline__ bool logits_item(int round, int cta, int n_cta, int n
 __global__ void __launch_bounds__(288, 1)
 pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const int32_t* __restrict__ pattern,
                  const SelectPtrs w, int* status) {
+  pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   LogitsSmem& s = *reinterpret_cast<LogitsSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -794,6 +796,7 @@ __device__ __forceinline__ void load_z4(const float* __restrict__ row, int J, in
 template <int kLevel, bool kVec>
 __global__ void __launch_bounds__(kHistThreads)
 pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  pdl_enter();
   const int h = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (pattern[h] != CRISP_PATTERN_PE) return;
   extern __shared__ uint8_t hist_raw[];
@@ -871,6 +874,7 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
 // does the head-wide part.
 __global__ void __launch_bounds__(1024)
 pe_rows_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  pdl_enter();
   const int h = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (pattern[h] != CRISP_PATTERN_PE) return;
   __shared__ long long scratch[33];
@@ -1027,6 +1031,7 @@ __device__ __forceinline__ void fill_pe_row(const float* __restrict__ row, int m
 __global__ void __launch_bounds__(256)
 fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int64_t* __restrict__ row_ptr,
             int32_t* __restrict__ col_idx, int64_t capacity, int64_t* __restrict__ nnz_needed, int* status) {
+  pdl_enter();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int h = blockIdx.y;
   // offsets of the heads: every CTA adds the (few) head totals itself
@@ -1149,7 +1154,7 @@ int launch_prepare(const Dims& d, const __nv_bfloat16* qb, const __nv_bfloat16* 
                  "select: smem attribute");
   const long long n_tiles = static_cast<long long>(d.nb) * (d.hkv + d.hq);
   const int pool_ctas = static_cast<int>((n_tiles + 7) / 8);
-  CRISP_KERNEL("prepare", stream, prepare_kernel<<<vs_ctas + pool_ctas, 1024, vs_smem, stream>>>(
+  CRISP_KERNEL("prepare", stream, launch_pdl(prepare_kernel, dim3(vs_ctas + pool_ctas), dim3(1024), vs_smem, stream, 
                                       d, qb, kb, pattern, p_v, p_s, w, vs_ctas, pool_all_k));
   return CRISP_OK;
 }
@@ -1193,7 +1198,7 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
                    "select: smem attribute");
     const int nt = (d.nb + kBlock - 1) / kBlock;
     const int grid = min(n_sm, nt * d.hq);
-    CRISP_KERNEL("pe_logits", stream, pe_logits_kernel<<<grid, 288, smem, stream>>>(maps, d, pattern, w, status));
+    CRISP_KERNEL("pe_logits", stream, launch_pdl(pe_logits_kernel, dim3(grid), dim3(288), smem, stream, maps, d, pattern, w, status));
   }
   // up to four CTAs per SM if every head is PE (two when half of them are); a warp takes a row at a time
   // ... and never more than 2^18 entries of a head per CTA (the 32-bit mass words of pe_hist_kernel)
@@ -1207,12 +1212,12 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   auto* hist2 = vec ? pe_hist_kernel<2, true> : pe_hist_kernel<2, false>;
   CRISP_CUDA_TRY(cudaFuncSetAttribute(hist1, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(hist_smem(1))),
                  "select: smem attribute");
-  CRISP_KERNEL("pe_hist0", stream, hist0<<<dim3(hist_ctas, d.hq), kHistThreads, hist_smem(0), stream>>>(d, pattern, w));
-  CRISP_KERNEL("pe_hist1", stream, hist1<<<dim3(hist_ctas, d.hq), kHistThreads, hist_smem(1), stream>>>(d, pattern, w));
-  CRISP_KERNEL("pe_hist2", stream, hist2<<<dim3(hist_ctas, d.hq), kHistThreads, hist_smem(2), stream>>>(d, pattern, w));
+  CRISP_KERNEL("pe_hist0", stream, launch_pdl(hist0, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(0), stream, d, pattern, w));
+  CRISP_KERNEL("pe_hist1", stream, launch_pdl(hist1, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(1), stream, d, pattern, w));
+  CRISP_KERNEL("pe_hist2", stream, launch_pdl(hist2, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(2), stream, d, pattern, w));
   const int rows_ctas = max(1, min((d.nb + 31) / 32, 8));
-  CRISP_KERNEL("pe_rows", stream, pe_rows_kernel<<<dim3(rows_ctas, d.hq), 1024, 0, stream>>>(d, pattern, w));
-  CRISP_KERNEL("fill", stream, fill_kernel<<<dim3((d.nb + 7) / 8, d.hq), 256, 0, stream>>>(
+  CRISP_KERNEL("pe_rows", stream, launch_pdl(pe_rows_kernel, dim3(rows_ctas, d.hq), dim3(1024), 0, stream, d, pattern, w));
+  CRISP_KERNEL("fill", stream, launch_pdl(fill_kernel, dim3((d.nb + 7) / 8, d.hq), dim3(256), 0, stream, 
                                    d, pattern, w, row_ptr, col_idx, capacity, nnz_needed, status));
   CRISP_CUDA_TRY(cudaGetLastError(), "select: launch");
   return CRISP_OK;
@@ -1227,6 +1232,7 @@ namespace {
 __global__ void __launch_bounds__(256)
 jsd_kernel(const Dims d, const __nv_bfloat16* __restrict__ q, const float* __restrict__ kbar,
            const float* __restrict__ p_v, float tau_jsd, float* __restrict__ jsd, int32_t* __restrict__ pattern) {
+  pdl_enter();
   extern __shared__ float z[];  // [nb] pooled logits, then a_bar
   __shared__ float qbar[kHeadDim];
   __shared__ float fscratch[32];
@@ -1308,7 +1314,7 @@ int launch_route_jsd(const Dims& d, const void* q, const void* k, const float* p
   // block means of K for every KV head (no VS work, no Q pooling)
   int rc = launch_prepare(d, nullptr, static_cast<const __nv_bfloat16*>(k), nullptr, nullptr, nullptr, w, 0, 1, stream);
   if (rc != CRISP_OK) return rc;
-  CRISP_KERNEL("jsd", stream, jsd_kernel<<<d.hq, 256, sizeof(float) * d.nb, stream>>>(d, static_cast<const __nv_bfloat16*>(q), w.kbar, p_v,
+  CRISP_KERNEL("jsd", stream, launch_pdl(jsd_kernel, dim3(d.hq), dim3(256), sizeof(float) * d.nb, stream, d, static_cast<const __nv_bfloat16*>(q), w.kbar, p_v,
                                                          tau_jsd, jsd, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route_jsd: launch");
   return CRISP_OK;
