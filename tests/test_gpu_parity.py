@@ -178,6 +178,27 @@ def test_iid_inputs_custom_scale():
     pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples, key="o_dense", dense=True)
 
 
+def test_logits_growing_along_the_keys_rescale_every_half_step():
+    """Eq. 1 with logits that rise by 12 log2 units every 64 keys: the running maximum of every row outgrows the
+    attention kernel's lazy-rescale threshold (2^8) at every half step, so the accumulator is rescaled in
+    place all the way along the row (inputs with a sink-dominated maximum never take that path)."""
+    pu = _pu()
+    import paper_2609_01925_b200 as crisp
+    n, hq, hkv = 2048, 4, 2
+    q, k, v = synth.random_qkv(n, hq, hkv, seed=11, device="cuda")
+    q = (q.float() * 0.1)
+    k = (k.float() * 0.1)
+    q[:, :, 0] = 4.0
+    k[:, :, 0] = (24.0 * (torch.arange(n, device="cuda") // 64)).unsqueeze(1)   # exact in bf16
+    q, k = q.to(torch.bfloat16), k.to(torch.bfloat16)
+    p = crisp.make_params(n, hq, hkv, sink_tokens=4, k_min_blocks=2)
+    g = pu.run_gpu(p, q, k, v, dense=True)
+    samples = [(h, m) for h in range(hq) for m in range(n // 128)]
+    pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples)
+    pu.check_attention(g, q.cpu(), k.cpu(), v.cpu(), p, samples, key="o_dense", dense=True)
+    assert np.isfinite(g["o"]).all() and np.isfinite(g["o_dense"]).all()
+
+
 def test_zero_inputs_massive_ties():
     """Q = K = 0: every proxy row is uniform and every pooled row is flat (ties everywhere)."""
     pu = _pu()
