@@ -247,6 +247,8 @@ def main():
                     help="N > 1: one independent layer per rank, or one layer's KV groups split over the ranks")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-kv-groups-per-chunk", type=int, default=1,
+                    help="chunk size of the end-to-end leg (crisp_forward_host), in KV groups")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -439,25 +441,28 @@ def main():
     # end to end through the C ABI with host buffers
     e2e = None
     if not args.no_e2e:
+        # crisp_forward_host: the layer goes through the device one KV group at a time, the copies of one group
+        # overlapping the kernels of another; every step copies Q, K, V in and O out
         qh = q.cpu().pin_memory(); kh = k.cpu().pin_memory(); vh = v.cpu().pin_memory()
         oh = torch.empty(layer.o.shape, dtype=layer.o.dtype).pin_memory()
-        qd, kd, vd = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+        gpc = args.e2e_kv_groups_per_chunk
+        stage = torch.empty(B.crisp_forward_host_stage_bytes(p, gpc), dtype=torch.uint8, device=dev)
         e2e_steps = min(args.steps, 3)
         for i in range(1 + e2e_steps):
             if i == 1:
                 barrier()
                 a = ev(); a.record()
-            qd.copy_(qh, non_blocking=True); kd.copy_(kh, non_blocking=True); vd.copy_(vh, non_blocking=True)
-            layer.forward(qd, kd, vd)
-            oh.copy_(layer.o, non_blocking=True)
+            rc, _ = B.crisp_forward_host(p, qh, kh, vh, oh, gpc, stage)
+            B.check(rc, "crisp_forward_host")
         b = ev(); b.record()
         barrier()
         e2e_ms = max_over_ranks(a.elapsed_time(b) / e2e_steps, dist, dev)
         h2d = sum(x.numel() * x.element_size() for x in (qh, kh, vh))
         d2h = oh.numel() * oh.element_size()
         e2e = {"value": job_ms_per_layer(e2e_ms, world, shard), "unit": "ms/layer", "h2d_bytes_per_step": h2d,
-               "d2h_bytes_per_step": d2h}
-        del qh, kh, vh, oh, qd, kd, vd
+               "d2h_bytes_per_step": d2h,
+               "call": f"crisp_forward_host, {gpc} KV group(s) per chunk, pinned host buffers, copies overlapped with the kernels"}
+        del qh, kh, vh, oh, stage
 
     cpu_baseline, near = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

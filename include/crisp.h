@@ -242,6 +242,29 @@ int crisp_forward_varlen(const crisp_params* p, const int64_t* cu_seqlens, int32
                          int32_t* device_status, void* o, float* lse, int32_t dense_below_tokens, void* cuda_stream);
 
 /*
+ * Algorithm 1 for a layer whose Q, K, V and O live in HOST memory (the paper's Algorithm 1 is per head and has
+ * no counterpart for the transfers: the chunking below is this library's).  The layer is cut into chunks of
+ * kv_groups_per_chunk whole KV groups (a KV head with its H_q / H_kv query heads); chunk c is copied to the
+ * device, run through crisp_route, crisp_select and crisp_sparse_prefill exactly as crisp_forward runs it, and
+ * its output copied back, and the copies of one chunk overlap the kernels of another.  Every head's result is
+ * bit for bit what crisp_forward gives for the whole layer.
+ *   q_host, o_host [seq_len][H_q][128], k_host, v_host [seq_len][H_kv][128] bf16: HOST pointers.  Page-locked
+ *     memory lets the copies overlap with the kernels; pageable memory works, but serialises them.
+ *   kv_groups_per_chunk: 1 .. H_kv, a divisor of H_kv.
+ *   stage: DEVICE buffer, 256-byte aligned, of at least crisp_forward_host_stage_bytes(p, kv_groups_per_chunk)
+ *     bytes: two copies of a chunk's Q, K, V and O, the chunk's workspaces, routing outputs and lists (sized for
+ *     all causal blocks, so the lists always fit).  Its contents after the call are unspecified.
+ *   pattern_host (HOST, [H_q] i32) and nnz_host (HOST, one int64: blocks listed over all heads) are optional.
+ * The kernels run on cuda_stream, the copies on two streams the library creates on first use (per device, kept
+ * for the life of the process).  The call is synchronous: it returns when o_host is complete, with the first
+ * error of any chunk (host-side, or a device status word: CRISP_ERR_DEVICE_TIMEOUT ...), else CRISP_OK.
+ */
+size_t crisp_forward_host_stage_bytes(const crisp_params* p, int32_t kv_groups_per_chunk);
+int crisp_forward_host(const crisp_params* p, const void* q_host, const void* k_host, const void* v_host,
+                       void* o_host, int32_t kv_groups_per_chunk, void* stage, size_t stage_bytes,
+                       int32_t* pattern_host, int64_t* nnz_host, void* cuda_stream);
+
+/*
  * Diagnostic (the paper has no counterpart): per-kernel device times of the stage calls, for benchmarks.
  * crisp_profile_enable(1) discards earlier records and switches recording on: from then on every kernel the
  * library launches is bracketed by two CUDA events on the caller's stream (the events are created on first use

@@ -30,6 +30,7 @@ EXPORTS = (
     "crisp_route", "crisp_route_static", "crisp_select", "crisp_sparse_prefill", "crisp_dense_prefill",
     "crisp_poll_device_status", "crisp_forward", "crisp_route_jsd", "crisp_varlen_layout",
     "crisp_forward_varlen", "crisp_selftest_bounded_wait", "crisp_profile_enable", "crisp_profile_read",
+    "crisp_forward_host", "crisp_forward_host_stage_bytes",
 )
 
 
@@ -105,6 +106,10 @@ def load() -> ctypes.CDLL:
     lib.crisp_forward_varlen.restype = ctypes.c_int
     lib.crisp_forward_varlen.argtypes = [P, vp, ctypes.c_int32, vp, vp, vp, vp, sz, vp, sz, vp, sz, vp, vp, vp, vp,
                                          vp, vp, i64, vp, vp, vp, vp, ctypes.c_int32, vp]
+    lib.crisp_forward_host_stage_bytes.restype = sz
+    lib.crisp_forward_host_stage_bytes.argtypes = [P, ctypes.c_int32]
+    lib.crisp_forward_host.restype = ctypes.c_int
+    lib.crisp_forward_host.argtypes = [P, vp, vp, vp, vp, ctypes.c_int32, vp, sz, vp, vp, vp]
     lib.crisp_profile_enable.restype = ctypes.c_int
     lib.crisp_profile_enable.argtypes = [ctypes.c_int]
     lib.crisp_profile_read.restype = ctypes.c_int
@@ -200,6 +205,25 @@ def crisp_forward(p, q, k, v, route_ws, select_ws, prefill_ws, c_struct, pattern
                                 _ptr(c_struct), _ptr(pattern), _ptr(p_v), _ptr(p_s), _ptr(row_ptr),
                                 _ptr(col_idx), int(capacity), _ptr(nnz_needed), _ptr(o), _ptr(lse),
                                 int(dense_below_tokens), _stream(stream))
+
+
+def crisp_forward_host_stage_bytes(p, kv_groups_per_chunk: int) -> int:
+    return int(load().crisp_forward_host_stage_bytes(ctypes.byref(p), int(kv_groups_per_chunk)))
+
+
+def crisp_forward_host(p, q_host, k_host, v_host, o_host, kv_groups_per_chunk, stage, pattern_host=None,
+                       stream=None):
+    """Algorithm 1 on HOST tensors (CPU, ideally pinned), chunk by chunk of whole KV groups, copies overlapped with
+    the kernels (see include/crisp.h).  `stage` is a device byte tensor of crisp_forward_host_stage_bytes bytes.
+    Returns (status, blocks listed)."""
+    for t in (q_host, k_host, v_host, o_host):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("crisp_forward_host takes contiguous CPU tensors")
+    nnz = ctypes.c_int64(0)
+    rc = load().crisp_forward_host(ctypes.byref(p), _ptr(q_host), _ptr(k_host), _ptr(v_host), _ptr(o_host),
+                                   int(kv_groups_per_chunk), _ptr(stage), _nbytes(stage), _ptr(pattern_host),
+                                   ctypes.addressof(nnz), _stream(stream))
+    return rc, int(nnz.value)
 
 
 def _host_i64(values):

@@ -456,6 +456,221 @@ int crisp_selftest_bounded_wait(void* ws, size_t ws_bytes, int64_t limit_ns, voi
   return launch_selftest_bounded_wait(ws, limit_ns, static_cast<cudaStream_t>(cuda_stream));
 }
 
+namespace {
+// Carving of crisp_forward_host's staging buffer for one chunk shape.
+struct HostStage {
+  void* q[2];
+  void* k[2];
+  void* v[2];
+  void* o[2];
+  void* route_ws;
+  void* select_ws;
+  void* prefill_ws;
+  float* c_struct;
+  int32_t* pattern;
+  float* p_v;
+  float* p_s;
+  int64_t* row_ptr;
+  int64_t* nnz;
+  int32_t* col_idx;
+  int64_t capacity;
+  size_t route_bytes, select_bytes, prefill_bytes;
+};
+HostStage carve_host_stage(const Dims& dc, void* stage, size_t* total) {
+  HostStage hs;
+  uint8_t* base = static_cast<uint8_t*>(stage);
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    void* ptr = base + off;
+    off += (bytes + 255) & ~static_cast<size_t>(255);
+    return ptr;
+  };
+  const size_t qo = static_cast<size_t>(dc.n) * dc.hq * kHeadDim * 2, kv = static_cast<size_t>(dc.n) * dc.hkv * kHeadDim * 2;
+  for (int b = 0; b < 2; ++b) {
+    hs.q[b] = take(qo);
+    hs.k[b] = take(kv);
+    hs.v[b] = take(kv);
+    hs.o[b] = take(qo);
+  }
+  hs.route_bytes = route_ws_bytes(dc);
+  hs.select_bytes = select_ws_bytes(dc);
+  hs.prefill_bytes = prefill_ws_bytes(dc);
+  hs.route_ws = take(hs.route_bytes);
+  hs.select_ws = take(hs.select_bytes);
+  hs.prefill_ws = take(hs.prefill_bytes);
+  hs.c_struct = static_cast<float*>(take(sizeof(float) * dc.hq));
+  hs.pattern = static_cast<int32_t*>(take(sizeof(int32_t) * dc.hq));
+  hs.p_v = static_cast<float*>(take(sizeof(float) * dc.hq * dc.nb));
+  hs.p_s = static_cast<float*>(take(sizeof(float) * dc.hq * dc.nb));
+  hs.row_ptr = static_cast<int64_t*>(take(sizeof(int64_t) * dc.hq * (dc.nb + 1)));
+  hs.nnz = static_cast<int64_t*>(take(sizeof(int64_t)));
+  hs.capacity = static_cast<int64_t>(dc.hq) * dc.nb * (static_cast<int64_t>(dc.nb) + 1) / 2;
+  hs.col_idx = static_cast<int32_t*>(take(sizeof(int32_t) * static_cast<size_t>(hs.capacity)));
+  *total = off;
+  return hs;
+}
+// chunk shape: the layer's parameters with kv_groups_per_chunk KV groups
+int chunk_dims(const crisp_params* p, int32_t gpc, crisp_params* pc, Dims* dc) {
+  Dims d;
+  int rc = validate(p, &d);
+  if (rc != CRISP_OK) return rc;
+  if (gpc < 1 || gpc > p->n_kv_heads || p->n_kv_heads % gpc != 0) return CRISP_ERR_INVALID_ARG;
+  *pc = *p;
+  pc->n_kv_heads = gpc;
+  pc->n_q_heads = gpc * (p->n_q_heads / p->n_kv_heads);
+  return validate(pc, dc);
+}
+// copy streams of crisp_forward_host and a page-locked block for the per-chunk status words, per device
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  int* words = nullptr;  // [kMaxChunks][8]: three status words, nnz (two words)
+  std::mutex busy;       // one crisp_forward_host call per device at a time (they share the block above)
+};
+constexpr int kMaxChunks = 1024;
+std::mutex g_pipe_mutex;
+HostPipe g_pipes[64];
+int host_pipe(HostPipe** out) {
+  int dev = 0;
+  CRISP_CUDA_TRY(cudaGetDevice(&dev), "forward_host: device");
+  if (dev < 0 || dev >= 64) return CRISP_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_pipe_mutex);
+  HostPipe& hp = g_pipes[dev];
+  if (!hp.in) CRISP_CUDA_TRY(cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking), "forward_host: stream");
+  if (!hp.out) CRISP_CUDA_TRY(cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking), "forward_host: stream");
+  if (!hp.words) CRISP_CUDA_TRY(cudaHostAlloc(&hp.words, sizeof(int) * 8 * kMaxChunks, cudaHostAllocDefault), "forward_host: status block");
+  *out = &hp;
+  return CRISP_OK;
+}
+}  // namespace
+
+size_t crisp_forward_host_stage_bytes(const crisp_params* p, int32_t kv_groups_per_chunk) {
+  crisp_params pc;
+  Dims dc;
+  if (chunk_dims(p, kv_groups_per_chunk, &pc, &dc) != CRISP_OK) return 0;
+  size_t total = 0;
+  carve_host_stage(dc, nullptr, &total);
+  return total;
+}
+
+int crisp_forward_host(const crisp_params* p, const void* q_host, const void* k_host, const void* v_host,
+                       void* o_host, int32_t kv_groups_per_chunk, void* stage, size_t stage_bytes,
+                       int32_t* pattern_host, int64_t* nnz_host, void* cuda_stream) {
+  crisp_params pc;
+  Dims dc;
+  int rc = chunk_dims(p, kv_groups_per_chunk, &pc, &dc);
+  if (rc != CRISP_OK) return rc;
+  if (!q_host || !k_host || !v_host || !o_host || !stage) return CRISP_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(stage) & 255) != 0) return CRISP_ERR_WORKSPACE;
+  size_t need = 0;
+  const HostStage hs = carve_host_stage(dc, stage, &need);
+  if (stage_bytes < need) return CRISP_ERR_WORKSPACE;
+  const int n_chunks = p->n_kv_heads / kv_groups_per_chunk;
+  if (n_chunks > kMaxChunks) return CRISP_ERR_UNSUPPORTED;
+  HostPipe* hp = nullptr;
+  rc = host_pipe(&hp);
+  if (rc != CRISP_OK) return rc;
+  std::lock_guard<std::mutex> one_call(hp->busy);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+
+  // events: [buffer] inputs on the device / kernels finished / output on the host
+  cudaEvent_t in_done[2] = {nullptr, nullptr}, comp_done[2] = {nullptr, nullptr}, out_done[2] = {nullptr, nullptr};
+  cudaEvent_t start = nullptr;
+  auto destroy = [&]() {
+    for (int b = 0; b < 2; ++b) {
+      if (in_done[b]) cudaEventDestroy(in_done[b]);
+      if (comp_done[b]) cudaEventDestroy(comp_done[b]);
+      if (out_done[b]) cudaEventDestroy(out_done[b]);
+    }
+    if (start) cudaEventDestroy(start);
+  };
+  cudaError_t ce = cudaEventCreateWithFlags(&start, cudaEventDisableTiming);
+  for (int b = 0; b < 2 && ce == cudaSuccess; ++b) {
+    ce = cudaEventCreateWithFlags(&in_done[b], cudaEventDisableTiming);
+    if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&comp_done[b], cudaEventDisableTiming);
+    if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&out_done[b], cudaEventDisableTiming);
+  }
+  if (ce != cudaSuccess) {
+    destroy();
+    set_cuda_error(ce, "forward_host: events");
+    return CRISP_ERR_CUDA;
+  }
+#define CRISP_FH_TRY(expr, where)        \
+  do {                                   \
+    cudaError_t e__ = (expr);            \
+    if (e__ != cudaSuccess) {            \
+      cudaStreamSynchronize(hp->in);     \
+      cudaStreamSynchronize(st);         \
+      cudaStreamSynchronize(hp->out);    \
+      destroy();                         \
+      set_cuda_error(e__, where);        \
+      return CRISP_ERR_CUDA;             \
+    }                                    \
+  } while (0)
+
+  // the copy streams start behind whatever the caller has already enqueued on cuda_stream
+  CRISP_FH_TRY(cudaEventRecord(start, st), "forward_host: record");
+  CRISP_FH_TRY(cudaStreamWaitEvent(hp->in, start, 0), "forward_host: wait");
+  CRISP_FH_TRY(cudaStreamWaitEvent(hp->out, start, 0), "forward_host: wait");
+  const size_t row_q = static_cast<size_t>(p->n_q_heads) * kHeadDim * 2, row_kv = static_cast<size_t>(p->n_kv_heads) * kHeadDim * 2;
+  const size_t row_qc = static_cast<size_t>(dc.hq) * kHeadDim * 2, row_kvc = static_cast<size_t>(dc.hkv) * kHeadDim * 2;
+  int launch_rc = CRISP_OK;
+  for (int c = 0; c < n_chunks && launch_rc == CRISP_OK; ++c) {
+    const int b = c & 1;
+    // ---- inputs of chunk c: its heads are a column slice of every token's row
+    if (c >= 2) CRISP_FH_TRY(cudaStreamWaitEvent(hp->in, comp_done[b], 0), "forward_host: wait");  // chunk c - 2 has read buffer b
+    CRISP_FH_TRY(cudaMemcpy2DAsync(hs.k[b], row_kvc, static_cast<const uint8_t*>(k_host) + c * row_kvc, row_kv, row_kvc, dc.n,
+                                   cudaMemcpyHostToDevice, hp->in), "forward_host: copy K");
+    CRISP_FH_TRY(cudaMemcpy2DAsync(hs.q[b], row_qc, static_cast<const uint8_t*>(q_host) + c * row_qc, row_q, row_qc, dc.n,
+                                   cudaMemcpyHostToDevice, hp->in), "forward_host: copy Q");
+    CRISP_FH_TRY(cudaMemcpy2DAsync(hs.v[b], row_kvc, static_cast<const uint8_t*>(v_host) + c * row_kvc, row_kv, row_kvc, dc.n,
+                                   cudaMemcpyHostToDevice, hp->in), "forward_host: copy V");
+    CRISP_FH_TRY(cudaEventRecord(in_done[b], hp->in), "forward_host: record");
+    // ---- kernels of chunk c
+    CRISP_FH_TRY(cudaStreamWaitEvent(st, in_done[b], 0), "forward_host: wait");
+    if (c >= 2) CRISP_FH_TRY(cudaStreamWaitEvent(st, out_done[b], 0), "forward_host: wait");  // O of chunk c - 2 has left buffer b
+    launch_rc = crisp_forward(&pc, hs.q[b], hs.k[b], hs.v[b], hs.route_ws, hs.route_bytes, hs.select_ws, hs.select_bytes,
+                              hs.prefill_ws, hs.prefill_bytes, hs.c_struct, hs.pattern, hs.p_v, hs.p_s, hs.row_ptr,
+                              hs.col_idx, hs.capacity, hs.nnz, hs.o[b], nullptr, 0, st);
+    if (launch_rc != CRISP_OK) break;
+    // the chunk's status words, list size and labels leave on the kernels' stream, before the next chunk reuses them
+    int* wd = hp->words + 8 * c;
+    CRISP_FH_TRY(cudaMemcpyAsync(wd + 0, hs.route_ws, sizeof(int), cudaMemcpyDeviceToHost, st), "forward_host: status");
+    CRISP_FH_TRY(cudaMemcpyAsync(wd + 1, hs.select_ws, sizeof(int), cudaMemcpyDeviceToHost, st), "forward_host: status");
+    CRISP_FH_TRY(cudaMemcpyAsync(wd + 2, hs.prefill_ws, sizeof(int), cudaMemcpyDeviceToHost, st), "forward_host: status");
+    CRISP_FH_TRY(cudaMemcpyAsync(wd + 4, hs.nnz, sizeof(int64_t), cudaMemcpyDeviceToHost, st), "forward_host: nnz");
+    if (pattern_host)
+      CRISP_FH_TRY(cudaMemcpyAsync(pattern_host + c * dc.hq, hs.pattern, sizeof(int32_t) * dc.hq, cudaMemcpyDeviceToHost, st),
+                   "forward_host: labels");
+    CRISP_FH_TRY(cudaEventRecord(comp_done[b], st), "forward_host: record");
+    // ---- output of chunk c
+    CRISP_FH_TRY(cudaStreamWaitEvent(hp->out, comp_done[b], 0), "forward_host: wait");
+    CRISP_FH_TRY(cudaMemcpy2DAsync(static_cast<uint8_t*>(o_host) + c * row_qc, row_q, hs.o[b], row_qc, row_qc, dc.n,
+                                   cudaMemcpyDeviceToHost, hp->out), "forward_host: copy O");
+    CRISP_FH_TRY(cudaEventRecord(out_done[b], hp->out), "forward_host: record");
+  }
+  // everything this call enqueued has finished when the three streams are idle; cuda_stream also waits for the
+  // last output copy, so work the caller enqueues behind this call sees o_host complete
+  cudaError_t e_in = cudaStreamSynchronize(hp->in), e_st = cudaStreamSynchronize(st), e_out = cudaStreamSynchronize(hp->out);
+  destroy();
+#undef CRISP_FH_TRY
+  if (launch_rc != CRISP_OK) return launch_rc;
+  if (e_in != cudaSuccess || e_st != cudaSuccess || e_out != cudaSuccess) {
+    set_cuda_error(e_in != cudaSuccess ? e_in : (e_st != cudaSuccess ? e_st : e_out), "forward_host: synchronize");
+    return CRISP_ERR_CUDA;
+  }
+  int64_t nnz = 0;
+  for (int c = 0; c < n_chunks; ++c) {
+    const int* wd = hp->words + 8 * c;
+    for (int i = 0; i < 3; ++i)
+      if (wd[i] != 0) return wd[i];
+    int64_t chunk_nnz;
+    std::memcpy(&chunk_nnz, wd + 4, sizeof(chunk_nnz));
+    nnz += chunk_nnz;
+  }
+  if (nnz_host) *nnz_host = nnz;
+  return CRISP_OK;
+}
+
 int crisp_poll_device_status(void* ws, void* cuda_stream) {
   if (!ws) return CRISP_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
