@@ -15,6 +15,7 @@
 #include <cstdio>
 #include <mutex>
 
+#include <algorithm>
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -79,7 +80,8 @@ struct ProxySmem {
 };
 
 // Persistent CTAs, one per SM.  A CTA owns up to four query heads of one KV group - their 128 proxy queries
-// are loaded once and stay in shared memory - and walks over every gridDim.x-th key tile: TMA brings the K
+// are loaded once and stay in shared memory - and walks over every S-th key tile, S being the number of CTAs of
+// its group (the groups share the SMs evenly; SMs left over go to the first groups): TMA brings the K
 // tile in (two buffers, the load of the tile after next is issued while the current one is worked on), one
 // thread issues a 128 x 128 x 128 tcgen05 MMA per head into that head's TMEM buffer, and four groups of four
 // warps (one group per head, one thread per proxy row) reduce the logits to the tile partials.  The row threads
@@ -93,16 +95,30 @@ constexpr int kProxyThreads = 32 * (4 * kProxyHeads + 1);
 template <bool kRagged>
 __global__ void __launch_bounds__(kProxyThreads, 1)
 proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                      const Dims d, const RoutePtrs w, int* status, int n_head_chunks) {
+                      const Dims d, const RoutePtrs w, int* status, int n_head_chunks, int base_slices,
+                      int extra_groups) {
   pdl_enter();
   extern __shared__ uint8_t smem_raw[];
   ProxySmem& s = *reinterpret_cast<ProxySmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = d.group;
-  const int kvh = blockIdx.y / n_head_chunks, g0 = (blockIdx.y % n_head_chunks) * kProxyHeads;
+  // CTA -> (group, slice): the first extra_groups groups have base_slices + 1 CTAs, the others base_slices
+  int grp, sl, stride;
+  {
+    const int b = blockIdx.x, big = extra_groups * (base_slices + 1);
+    if (b < big) {
+      grp = b / (base_slices + 1);
+      sl = b % (base_slices + 1);
+      stride = base_slices + 1;
+    } else {
+      grp = extra_groups + (b - big) / base_slices;
+      sl = (b - big) % base_slices;
+      stride = base_slices;
+    }
+  }
+  const int kvh = grp / n_head_chunks, g0 = (grp % n_head_chunks) * kProxyHeads;
   const int gc = min(kProxyHeads, G - g0);            // heads of this CTA
-  const int stride = gridDim.x;
-  const int n_my_tiles = static_cast<int>(blockIdx.x) < d.nb ? (d.nb - 1 - static_cast<int>(blockIdx.x)) / stride + 1 : 0;
+  const int n_my_tiles = sl < d.nb ? (d.nb - 1 - sl) / stride + 1 : 0;
   constexpr int kIssuerWarp = 4 * kProxyHeads;
 
   if (tid == 0) {
@@ -133,7 +149,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
       prefetch_tmap(&tmap_q);
       prefetch_tmap(&tmap_k);
       auto load_k = [&](int n) {
-        const int J = blockIdx.x + n * stride, kb = n & 1;
+        const int J = sl + n * stride, kb = n & 1;
         mbar_arrive_expect_tx(&s.bar_k_full[kb], 32768);
         tma_load_3d(s.k[kb][0], &tmap_k, &s.bar_k_full[kb], 0, kvh, J * kBlock);
         tma_load_3d(s.k[kb][1], &tmap_k, &s.bar_k_full[kb], 64, kvh, J * kBlock);
@@ -196,7 +212,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     // running maximum and sum of this row over the CTA's tiles
     float run_m = -INFINITY, run_l = 0.f;
     for (int n = 0; n < n_my_tiles && ok; ++n) {
-      const int J = blockIdx.x + n * stride;
+      const int J = sl + n * stride;
       const int qoff = d.nfull - 1 - J;
       const bool vis_up = qoff - 1 >= 0, vis_lo = qoff >= 0;  // "hi" (q + 1 >= 0) is visible whenever it is non-empty
       const int js = min(max(d.w_sink - J * kBlock, 0), kBlock);         // anchor: local key < js
@@ -342,7 +358,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
     }
     // this CTA's share of the row statistics
     {
-      const size_t o = (static_cast<size_t>(h) * w.n_slices + blockIdx.x) * kBlock + i;
+      const size_t o = (static_cast<size_t>(h) * w.n_slices + sl) * kBlock + i;
       w.cm[o] = run_m;
       w.cl[o] = run_l;
     }
@@ -352,7 +368,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   __syncthreads();
   if (tid == 0) {
     if (s.abort_flag) atomicExch(status, CRISP_ERR_DEVICE_TIMEOUT);
-    s.is_last = atomicAdd(&w.group_done[blockIdx.y], 1) == static_cast<int>(gridDim.x) - 1;
+    s.is_last = atomicAdd(&w.group_done[grp], 1) == stride - 1;
   }
   if (warp == kIssuerWarp) tmem_dealloc(tm, 512);
   __syncthreads();
@@ -363,7 +379,7 @@ proxy_partials_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_c
   for (int item = tid; item < gc * kBlock; item += blockDim.x) {
     const int h = kvh * G + g0 + item / kBlock, i = item % kBlock;
     float M = -INFINITY, L = 0.f;
-    for (int c = 0; c < static_cast<int>(gridDim.x); ++c) {
+    for (int c = 0; c < stride; ++c) {
       const size_t o = (static_cast<size_t>(h) * w.n_slices + c) * kBlock + i;
       const float m = __ldcg(w.cm + o), l = __ldcg(w.cl + o);
       const float nm = fmaxf(M, m);
@@ -464,15 +480,22 @@ __global__ void __launch_bounds__(128) tile_sums_kernel(const Dims d, const Rout
 // How the proxy kernel's grid is laid out: one CTA per SM; the (KV head, chunk of four query heads) groups share
 // the SMs evenly, each group's CTAs split its key tiles.
 struct ProxyGrid {
-  int n_head_chunks, groups, slices;
+  int n_head_chunks, groups, slices, extra;  // `extra` groups have slices + 1 CTAs
 };
 ProxyGrid proxy_grid(const Dims& d, int n_sm) {
   ProxyGrid g;
   g.n_head_chunks = (d.group + kProxyHeads - 1) / kProxyHeads;
   g.groups = d.hkv * g.n_head_chunks;
   g.slices = n_sm / g.groups;
-  if (g.slices < 1) g.slices = 1;
-  if (g.slices > d.nb) g.slices = d.nb;
+  g.extra = n_sm % g.groups;  // the SMs the even split leaves over go to the first groups
+  if (g.slices < 1) {
+    g.slices = 1;
+    g.extra = 0;
+  }
+  if (g.slices >= d.nb) {
+    g.slices = d.nb;
+    g.extra = 0;
+  }
   return g;
 }
 // The workspace is sized without knowing the device: room for the CTAs of a 160-SM part; a larger device simply
@@ -535,8 +558,13 @@ int launch_route(const Dims& d, const void* q, const void* k, void* ws, float* c
   CRISP_CUDA_TRY(cudaGetDevice(&dev), "route: current device");
   CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "route: SM count");
   ProxyGrid g = proxy_grid(d, n_sm);
-  if (g.slices > w.n_slices) g.slices = w.n_slices;
-  CRISP_KERNEL("proxy", stream, launch_pdl(proxy, dim3(g.slices, g.groups), dim3(kProxyThreads), smem, stream, tq, tk, d, w, status, g.n_head_chunks));
+  if (g.slices + (g.extra > 0 ? 1 : 0) > w.n_slices) {
+    g.slices = std::min(g.slices, w.n_slices);
+    g.extra = 0;
+  }
+  CRISP_KERNEL("proxy", stream,
+               launch_pdl(proxy, dim3(g.slices * g.groups + g.extra), dim3(kProxyThreads), smem, stream, tq, tk, d, w,
+                          status, g.n_head_chunks, g.slices, g.extra));
   CRISP_KERNEL("tile_sums", stream, launch_pdl(tile_sums_kernel, dim3(w.n_chunks, d.hq), dim3(128), 0, stream, d, w, p_v, p_s, c_struct, pattern));
   CRISP_CUDA_TRY(cudaGetLastError(), "route: launch");
   return CRISP_OK;
