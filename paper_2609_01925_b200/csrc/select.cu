@@ -76,6 +76,7 @@ struct SelectPtrs {
   int* take;        // [hq][nb] ties of row m that are selected
   int* local_off;   // [hq][nb] exclusive prefix sum of the row lengths inside the head
   long long* head_total;  // [hq] entries of the head's lists
+  int* pe_list;     // [hq + 1] the PE heads in ascending order, then (at index hq) how many there are
   int words;
 };
 
@@ -297,6 +298,17 @@ prepare_kernel(const Dims d, const __nv_bfloat16* __restrict__ q, const __nv_bfl
   }
   // ---------------- VS head: both directions, then the lengths of its lists
   const int h = blockIdx.x, nb = d.nb;
+  if (h == 0 && tid < 32) {
+    // the PE heads in ascending order, for the pooled-logits kernel's work items
+    int n = 0;
+    for (int h0 = 0; h0 < d.hq; h0 += 32) {
+      const bool pe = h0 + tid < d.hq && pattern[h0 + tid] == CRISP_PATTERN_PE;
+      const uint32_t mask = __ballot_sync(0xffffffffu, pe);
+      if (pe) w.pe_list[n + __popc(mask & ((1u << tid) - 1u))] = h0 + tid;
+      n += __popc(mask);
+    }
+    if (tid == 0) w.pe_list[d.hq] = n;
+  }
   if (pattern[h] != CRISP_PATTERN_VS) return;
   double* sorted = reinterpret_cast<double*>(sm_raw);  // [nb] values in descending order (gamma rule)
   float* p = reinterpret_cast<float*>(sorted + nb);    // [nb]
@@ -342,12 +354,15 @@ prepare_kernel(const Dims d, const __nv_bfloat16* __restrict__ q, const __nv_bfl
 //
 // Persistent CTAs.  A work item is one PE head and one strip of 128 query blocks (rows m); the strip's three
 // operand terms stay in shared memory while the CTA walks over the strip's key tiles jt = 0 .. mt.  The K-side
-// operands arrive in two halves of 64 dims (two 48 KB slots): while the MMAs of one half run, the other slot is
-// refilled for the next tile.  Two TMEM accumulators and two groups of four epilogue warps (one thread per row;
-// group 0 drains the even tiles of an item, group 1 the odd ones) keep the MMAs of tile t + 1 running while tile
-// t is drained.  A strip holds complete rows, so the epilogue threads carry the running maximum and sum of their
-// row across their tiles and leave the row's softmax normalisers at the end of the item; the normalised map
-// itself is never written.
+// operands arrive in two halves of 64 dims (two 48 KB slots), loaded by a thread of their own: a slot is refilled
+// the moment the MMAs that read it have completed, while the other half's MMAs run (with the loads issued by the
+// MMA thread, which sits in the tensor pipe's queue while it issues, every half arrived ~1700 cycles late).
+// Two TMEM accumulators and two groups of four epilogue warps (one thread per row; group 0 drains the even tiles
+// of an item, group 1 the odd ones) keep the MMAs of tile t + 1 running while tile t is drained.  A strip holds
+// complete rows, so the epilogue threads carry the running maximum and sum of their row across their tiles and
+// leave the row's softmax normalisers at the end of the item; the normalised map itself is never written.  The
+// logits go to global memory through a 32 x 32 staging tile per warp, so that a store writes whole 128-byte
+// lines of four rows instead of 16 bytes of 32 rows.
 struct LogitsMaps {
   CUtensorMap q[3], k[3];
 };
@@ -361,7 +376,9 @@ struct LogitsSmem {
   int abort_flag;
   int n_pe;
   float2 row_state[kBlock];  // (running maximum, running sum) of the rows' odd tiles, handed to the even tiles' threads
-  int pe_heads[1024];
+  // per epilogue warp: 32 rows x 32 columns of a tile on their way to global memory; the 16-byte chunk q of row r
+  // sits at chunk position q ^ (r % 8)
+  alignas(16) float stage[8][32 * 32];
 };
 
 // Item `idx` of CTA `cta`: positions of the size-sorted order (long strips first) are dealt out in rounds of
@@ -376,7 +393,7 @@ __device__ __forceinline__ bool logits_item(int round, int cta, int n_cta, int n
   return true;
 }
 
-__global__ void __launch_bounds__(288, 1)
+__global__ void __launch_bounds__(320, 1)
 pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const int32_t* __restrict__ pattern,
                  const SelectPtrs w, int* status) {
   pdl_enter();
@@ -385,10 +402,7 @@ pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const in
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     s.abort_flag = 0;
-    int n = 0;
-    for (int h = 0; h < d.hq && n < 1024; ++h)
-      if (pattern[h] == CRISP_PATTERN_PE) s.pe_heads[n++] = h;
-    s.n_pe = n;
+    s.n_pe = w.pe_list[d.hq];
     mbar_init(&s.bar_a_full, 1);
     mbar_init(&s.bar_a_free, 1);
     for (int i = 0; i < 2; ++i) {
@@ -413,13 +427,43 @@ pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const in
   const int nt = (d.nb + kBlock - 1) / kBlock;
   const int n_items = nt * n_pe, n_cta = gridDim.x, cta = blockIdx.x;
 
-  if (warp == 8) {
+  if (warp == 9) {
     if (lane == 0) {
-      // ---- TMA producer and MMA issuer
+      // ---- TMA producer: the strip's operands once per item, the K-side operands half by half.  It runs in a
+      // thread of its own so that a slot is refilled the moment the MMAs that read it have completed, while the
+      // issuing thread sits in the tensor pipe's queue.
       for (int pl = 0; pl < 3; ++pl) {
         prefetch_tmap(&maps.q[pl]);
         prefetch_tmap(&maps.k[pl]);
       }
+      bool ok = true;
+      uint32_t T = 0;  // tiles loaded so far by this CTA
+      for (int round = 0; ok; ++round) {
+        int hs, mt;
+        if (!logits_item(round, cta, n_cta, n_items, n_pe, nt, &hs, &mt)) break;
+        const int h = w.pe_list[hs], kvh = h / d.group;
+        // the strip's operands may be replaced once every MMA of the previous item has read them
+        if (round > 0) ok = mbar_wait(&s.bar_a_free, (round - 1) & 1, &s.abort_flag);
+        if (!ok) break;
+        mbar_arrive_expect_tx(&s.bar_a_full, 6u * 16384u);
+        for (int pl = 0; pl < 3; ++pl)
+          for (int hf = 0; hf < 2; ++hf) tma_load_3d(s.a[pl][hf], &maps.q[pl], &s.bar_a_full, hf * 64, h, mt * kBlock);
+        for (int jt = 0; jt <= mt && ok; ++jt, ++T) {
+          for (int hf = 0; hf < 2 && ok; ++hf) {
+            // slot hf is free once the previous tile's MMAs on it have completed
+            if (T > 0) ok = mbar_wait(&s.bar_b_free[hf], (T - 1) & 1, &s.abort_flag);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&s.bar_b_full[hf], 3u * 16384u);
+            for (int pl = 0; pl < 3; ++pl)
+              tma_load_3d(s.b[hf][pl], &maps.k[pl], &s.bar_b_full[hf], hf * 64, kvh, jt * kBlock);
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 8) {
+    if (lane == 0) {
+      // ---- MMA issuer
       constexpr uint32_t idesc = umma_idesc_bf16(128, 128, false, false);
       // (term of Q, term of K), smallest products first
       const int pa[6] = {2, 0, 1, 1, 0, 0}, pb[6] = {0, 2, 1, 0, 1, 0};
@@ -428,27 +472,9 @@ pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const in
       bool ok = true;
       uint32_t T = 0;               // tiles issued so far by this CTA
       uint32_t acc_uses[2] = {0, 0};  // tiles that went into each accumulator
-      auto load_b = [&](int hf, int kvh, int jt) {
-        mbar_arrive_expect_tx(&s.bar_b_full[hf], 3u * 16384u);
-        for (int pl = 0; pl < 3; ++pl) tma_load_3d(s.b[hf][pl], &maps.k[pl], &s.bar_b_full[hf], hf * 64, kvh, jt * kBlock);
-      };
       for (int round = 0; ok; ++round) {
         int hs, mt;
         if (!logits_item(round, cta, n_cta, n_items, n_pe, nt, &hs, &mt)) break;
-        const int h = s.pe_heads[hs], kvh = h / d.group;
-        // the strip's operands may be replaced once every MMA of the previous item has read them
-        if (round > 0) ok = mbar_wait(&s.bar_a_free, (round - 1) & 1, &s.abort_flag);
-        if (!ok) break;
-        mbar_arrive_expect_tx(&s.bar_a_full, 6u * 16384u);
-        for (int pl = 0; pl < 3; ++pl)
-          for (int hf = 0; hf < 2; ++hf) tma_load_3d(s.a[pl][hf], &maps.q[pl], &s.bar_a_full, hf * 64, h, mt * kBlock);
-        // first tile of the item: both halves of the K-side operands (the slots are free: see the loop's end)
-        if (T > 0) {
-          ok = mbar_wait(&s.bar_b_free[0], (T - 1) & 1, &s.abort_flag) && mbar_wait(&s.bar_b_free[1], (T - 1) & 1, &s.abort_flag);
-          if (!ok) break;
-        }
-        load_b(0, kvh, 0);
-        load_b(1, kvh, 0);
         ok = mbar_wait(&s.bar_a_full, round & 1, &s.abort_flag);
         for (int jt = 0; jt <= mt && ok; ++jt, ++T) {
           // even tiles of an item accumulate in buffer 0 (drained by epilogue group 0), odd ones in buffer 1
@@ -469,22 +495,9 @@ pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const in
                 umma_ss(tm + acc * 128, ad, bd, idesc, (hf > 0 || t > 0 || k4 > 0) ? 1u : 0u);
               }
             umma_commit(&s.bar_b_free[hf]);
-            if (hf == 0) {
-              // Slot 1 of this tile: free once the previous tile's second half has been multiplied, which the
-              // pipe does before it starts on the MMAs just issued; the load then has their time to arrive.
-              // (The first tile of an item had both slots filled in the item's prologue.)
-              if (jt > 0) {
-                ok = mbar_wait(&s.bar_b_free[1], (T - 1) & 1, &s.abort_flag);
-                if (ok) load_b(1, kvh, jt);
-              }
-            } else {
+            if (hf == 1) {
               umma_commit(&s.bar_acc_full[acc]);
               if (jt == mt) umma_commit(&s.bar_a_free);
-              // slot 0 for the next tile: free once this tile's first half is done, i.e. while its second runs
-              if (jt < mt) {
-                ok = mbar_wait(&s.bar_b_free[0], T & 1, &s.abort_flag);
-                if (ok) load_b(0, kvh, jt + 1);
-              }
             }
           }
         }
@@ -501,10 +514,9 @@ pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const in
     for (int round = 0; ok; ++round) {
       int hs, mt;
       if (!logits_item(round, cta, n_cta, n_items, n_pe, nt, &hs, &mt)) break;
-      const int h = s.pe_heads[hs];
+      const int h = w.pe_list[hs];
       const int m = mt * kBlock + r_;
       const bool row_ok = m < d.nb;
-      float* zrow = w.amat + (static_cast<size_t>(h) * d.nb + (row_ok ? m : 0)) * d.nb;
       float M = -INFINITY, S = 0.f;
       for (int jt = gr; jt <= mt && ok; jt += 2, ++uses) {
         ok = mbar_wait_warp(&s.bar_acc_full[gr], uses & 1, &s.abort_flag);
@@ -517,41 +529,91 @@ pe_logits_kernel(const __grid_constant__ LogitsMaps maps, const Dims d, const in
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&s.bar_acc_free[gr]);
-        if (!row_ok) continue;
         const int J0 = jt * kBlock;
-        const int n_valid = min(kBlock, m - J0 + 1);  // columns J <= m of this tile (128 except on the diagonal tile)
+        // Tiles left of the strip's diagonal tile are causal in full for every row of the strip; only the
+        // diagonal tile (jt == mt) needs per-row column counts.
+        const bool full = jt < mt && vec_ok;
+        const int n_valid = full ? kBlock : min(kBlock, m - J0 + 1);  // columns J <= m of this tile
         float tmax = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float z = __uint_as_float(r[c][i]) * d.scale_log2;
-            r[c][i] = __float_as_uint(z);
-            if (c * 32 + i < n_valid) tmax = fmaxf(tmax, z);
-          }
-        float tsum = 0.f;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c * 32 + i < n_valid) tsum += ex2(__uint_as_float(r[c][i]) - tmax);
-        const float nm = fmaxf(M, tmax);
-        S = S * ex2(M - nm) + tsum * ex2(tmax - nm);
-        M = nm;
-        if (vec_ok && n_valid == kBlock) {
-          float4* dst = reinterpret_cast<float4*>(zrow + J0);
+        if (full) {
+          float t0 = -INFINITY, t1 = -INFINITY, t2 = -INFINITY, t3 = -INFINITY;
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              dst[c * 8 + (i >> 2)] = make_float4(__uint_as_float(r[c][i]), __uint_as_float(r[c][i + 1]),
-                                                  __uint_as_float(r[c][i + 2]), __uint_as_float(r[c][i + 3]));
+            for (int i = 0; i < 32; i += 4) {
+              const float z0 = __uint_as_float(r[c][i]) * d.scale_log2, z1 = __uint_as_float(r[c][i + 1]) * d.scale_log2;
+              const float z2 = __uint_as_float(r[c][i + 2]) * d.scale_log2, z3 = __uint_as_float(r[c][i + 3]) * d.scale_log2;
+              r[c][i] = __float_as_uint(z0); r[c][i + 1] = __float_as_uint(z1);
+              r[c][i + 2] = __float_as_uint(z2); r[c][i + 3] = __float_as_uint(z3);
+              t0 = fmaxf(t0, z0); t1 = fmaxf(t1, z1); t2 = fmaxf(t2, z2); t3 = fmaxf(t3, z3);
+            }
+          tmax = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
         } else {
 #pragma unroll
           for (int c = 0; c < 4; ++c)
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c * 32 + i < n_valid) zrow[J0 + c * 32 + i] = __uint_as_float(r[c][i]);
+            for (int i = 0; i < 32; ++i) {
+              const float z = __uint_as_float(r[c][i]) * d.scale_log2;
+              r[c][i] = __float_as_uint(z);
+              if (c * 32 + i < n_valid) tmax = fmaxf(tmax, z);
+            }
+        }
+        if (row_ok) {
+          // (the order of the additions is the same in both branches: the sums must not depend on the path)
+          float tsum = 0.f;
+          if (full) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+              for (int i = 0; i < 32; ++i) tsum += ex2(__uint_as_float(r[c][i]) - tmax);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (c * 32 + i < n_valid) tsum += ex2(__uint_as_float(r[c][i]) - tmax);
+          }
+          const float nm = fmaxf(M, tmax);
+          S = S * ex2(M - nm) + tsum * ex2(tmax - nm);
+          M = nm;
+        }
+        // The thread holds 128 columns of ONE row; stored from here, a warp's store would touch 32 rows (32 lines
+        // of 16 bytes each).  The warp passes 32 x 32 chunks through shared memory instead, so that every store
+        // writes four rows of 128 contiguous bytes.
+        float* stg = s.stage[warp];
+        const int m_warp = mt * kBlock + (warp & 3) * 32;  // first row of this warp
+        const int rr0 = lane >> 3, qq = lane & 7;          // this lane stores chunk qq of rows rr0, rr0 + 4, ...
+        float* dst0 = w.amat + (static_cast<size_t>(h) * d.nb + m_warp + rr0) * d.nb + J0 + 4 * qq;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+#pragma unroll
+          for (int q4 = 0; q4 < 8; ++q4)
+            *reinterpret_cast<uint4*>(stg + lane * 32 + ((q4 ^ (lane & 7)) << 2)) =
+                make_uint4(r[c][4 * q4], r[c][4 * q4 + 1], r[c][4 * q4 + 2], r[c][4 * q4 + 3]);
+          __syncwarp();
+#pragma unroll
+          for (int kk = 0; kk < 8; ++kk) {
+            const int rr = 4 * kk + rr0;
+            const float4 vv = *reinterpret_cast<const float4*>(stg + rr * 32 + ((qq ^ (rr & 7)) << 2));
+            const int m_rr = m_warp + rr;
+            float* dst = dst0 + static_cast<size_t>(4 * kk) * d.nb + c * 32;
+            if (full) {
+              if (m_rr < d.nb) *reinterpret_cast<float4*>(dst) = vv;
+            } else {
+              const int cnt = min(kBlock, m_rr - J0 + 1) - (c * 32 + 4 * qq);  // how many of the four columns are causal
+              if (m_rr < d.nb && cnt > 0) {
+                if (vec_ok && cnt >= 4) {
+                  *reinterpret_cast<float4*>(dst) = vv;
+                } else {
+                  dst[0] = vv.x;
+                  if (cnt > 1) dst[1] = vv.y;
+                  if (cnt > 2) dst[2] = vv.z;
+                  if (cnt > 3) dst[3] = vv.w;
+                }
+              }
+            }
+          }
+          __syncwarp();
         }
       }
       // the odd tiles' statistics join the even tiles' (every row has an even tile: tile 0)
@@ -1141,6 +1203,7 @@ SelectPtrs carve(const Dims& d, void* ws, size_t* total) {
   w.take = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
   w.local_off = static_cast<int*>(take(sizeof(int) * d.hq * d.nb));
   w.head_total = static_cast<long long*>(take(sizeof(long long) * d.hq));
+  w.pe_list = static_cast<int*>(take(sizeof(int) * (d.hq + 1)));
   *total = off;
   return w;
 }
@@ -1198,7 +1261,7 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
                    "select: smem attribute");
     const int nt = (d.nb + kBlock - 1) / kBlock;
     const int grid = min(n_sm, nt * d.hq);
-    CRISP_KERNEL("pe_logits", stream, launch_pdl(pe_logits_kernel, dim3(grid), dim3(288), smem, stream, maps, d, pattern, w, status));
+    CRISP_KERNEL("pe_logits", stream, launch_pdl(pe_logits_kernel, dim3(grid), dim3(320), smem, stream, maps, d, pattern, w, status));
   }
   // up to four CTAs per SM if every head is PE (two when half of them are); a warp takes a row at a time
   // ... and never more than 2^18 entries of a head per CTA (the 32-bit mass words of pe_hist_kernel)
