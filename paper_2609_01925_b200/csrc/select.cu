@@ -834,6 +834,63 @@ __device__ __forceinline__ void hist_group(const float (&z)[4], int J, int m, fl
     }
 }
 
+// Level 0 (bins = exponents) of one group of 128 consecutive entries, four per lane.  An entry is at most the
+// row's largest value, 1 / (row sum N_b), so its exponent is e_top - k with k >= 0, and most entries have k < 4.
+// Each lane keeps one packed 64-bit accumulator per k in registers - low-significand sum in bits 0-19,
+// high-significand sum in bits 20-39, count from bit 40 - and the warp adds them up once per flush
+// (hist0_flush), so such an entry costs a handful of integer instructions and no shared-memory traffic.  A group
+// in which any lane holds another kind of entry (k >= 4, or a value below 2^-37) takes the general path.
+template <bool kMasked>
+__device__ __forceinline__ void hist0_group(const float (&z)[4], int J, int m, float M, float inv, int e_top,
+                                            unsigned long long (&acc)[4], unsigned int* cnt, unsigned int* slo,
+                                            unsigned int* shi, const SelectPtrs& w, int h, int lane) {
+  unsigned int key[4];
+  bool fast = true;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    key[e] = __float_as_uint(pe_value(z[e], M, inv));
+    const bool valid = !kMasked || J + e <= m;
+    const int ex = static_cast<int>(key[e] >> 23);
+    fast = fast && (!valid || (e_top - ex < 4 && ex >= kMinFastExp));
+  }
+  if (!__all_sync(0xffffffffu, fast)) {
+    int gt = 0, in = 0;
+    hist_group<0, kMasked>(z, J, m, M, inv, 0u, cnt, slo, shi, w, h, lane, gt, in);
+    return;
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const bool valid = !kMasked || J + e <= m;
+    const int k = e_top - static_cast<int>(key[e] >> 23);
+    const unsigned long long packed = static_cast<unsigned long long>(key[e] & 0xFFFu) |
+                                      (static_cast<unsigned long long>(((key[e] >> 12) & 0x7FFu) | 0x800u) << 20) |
+                                      (1ull << 40);
+#pragma unroll
+    for (int b = 0; b < 4; ++b)
+      if (valid && k == b) acc[b] += packed;
+  }
+}
+// Adds the lanes' accumulators into the CTA's shared-memory bins e_top .. e_top - 3 and clears them.  A lane may
+// hold at most 255 entries per accumulator between two flushes (the 20-bit fields).
+__device__ __forceinline__ void hist0_flush(unsigned long long (&acc)[4], int e_top, unsigned int* cnt,
+                                            unsigned int* slo, unsigned int* shi, int lane) {
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    const unsigned int n = static_cast<unsigned int>(acc[b] >> 40);
+    if (__any_sync(0xffffffffu, n != 0u)) {
+      const unsigned int ns = __reduce_add_sync(0xffffffffu, n);
+      const unsigned int lo = __reduce_add_sync(0xffffffffu, static_cast<unsigned int>(acc[b] & 0xFFFFFu));
+      const unsigned int hi = __reduce_add_sync(0xffffffffu, static_cast<unsigned int>((acc[b] >> 20) & 0xFFFFFu));
+      if (lane == 0) {
+        atomicAdd(&cnt[e_top - b], ns);
+        atomicAdd(&slo[e_top - b], lo);
+        atomicAdd(&shi[e_top - b], hi);
+      }
+    }
+    acc[b] = 0ull;
+  }
+}
+
 // Four consecutive logits of a row.  With kVec the row's storage is read as one float4 (columns beyond m but
 // inside the row's N_b slots hold unspecified values, which the callers mask); otherwise element by element.
 template <bool kVec>
@@ -849,18 +906,24 @@ __device__ __forceinline__ void load_z4(const float* __restrict__ row, int J, in
 
 // One histogram level of one head per CTA column (blockIdx.y = head).  A warp takes one row at a time (rows dealt
 // round robin from the longest down), reads its logits as float4 - 512 entries in flight per warp - recomputes
-// the normalised values and bins the ones whose upper bits match the prefix found so far.  Entries that share a
-// bin with the first pending entry of the warp are added across the warp and cost one set of adds (three such
-// rounds at level 0, where a row's values share two or three exponents; one at the lower levels, whose entries
-// are spread over thousands of bins unless the map is flat); what is left goes in lane by lane.  Level 2 also
+// the normalised values and bins the ones whose upper bits match the prefix found so far.  At level 0 the lanes
+// keep the bins of the row's top four exponents in registers (hist0_group).  Elsewhere entries that share a
+// bin with the first pending entry of the warp are added across the warp and cost one set of adds (one such round
+// at the lower levels, whose entries are spread over thousands of bins unless the map is flat; three in level 0's
+// general path); what is left goes in lane by lane.  Level 2 also
 // counts, per row, the entries above and inside the cut's last bin.  The last CTA of a head to finish locates
 // the cut in the head's finished histogram.
 template <int kLevel, bool kVec>
 __global__ void __launch_bounds__(kHistThreads)
-pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w, int resident_ctas, int min_ctas) {
   pdl_enter();
   const int h = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (pattern[h] != CRISP_PATTERN_PE) return;
+  // The grid has room for every head being a PE head; how many there are is known only on the device.  The PE
+  // heads share the CTAs that fit on the GPU at once evenly, so that the launch is one full wave rather than
+  // one and a bit; the CTAs beyond a head's share leave at once.  (min_ctas keeps a CTA's bin sums in 32 bits.)
+  const int n_ctas = min(static_cast<int>(gridDim.x), max(min_ctas, resident_ctas / max(1, w.pe_list[d.hq])));
+  if (static_cast<int>(blockIdx.x) >= n_ctas) return;
   extern __shared__ uint8_t hist_raw[];
   constexpr int nbins = level_bins(kLevel);
   unsigned int* cnt = reinterpret_cast<unsigned int*>(hist_raw);  // [nbins] each
@@ -878,27 +941,42 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
     const float* am = w.amat + static_cast<size_t>(h) * d.nb * d.nb;
     const float* rm = w.row_m + static_cast<size_t>(h) * d.nb;
     const float* ri = w.row_inv + static_cast<size_t>(h) * d.nb;
-    const int n_warps = gridDim.x * (kHistThreads / 32), gw = blockIdx.x * (kHistThreads / 32) + warp;
+    const int n_warps = n_ctas * (kHistThreads / 32), gw = blockIdx.x * (kHistThreads / 32) + warp;
     for (int m = d.nb - 1 - gw; m >= 0; m -= n_warps) {
       const float* row = am + static_cast<size_t>(m) * d.nb;
       const float M = rm[m], inv = ri[m];
       int gt = 0, in = 0;
       int J0 = 0;
+      // level 0: the row's largest value is inv itself (its exponent bounds every entry's), see hist0_group
+      const int e_top = static_cast<int>(__float_as_uint(inv) >> 23);
+      unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
       // whole steps of 512 entries: the four loads of a lane are issued before any of them is binned
       for (; J0 + 511 <= m; J0 += 512) {
         float z[4][4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) load_z4<kVec>(row, J0 + 128 * u + 4 * lane, m, z[u]);
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
-          hist_group<kLevel, false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
+        for (int u = 0; u < 4; ++u) {
+          if (kLevel == 0) {
+            hist0_group<false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, e_top, acc, cnt, slo, shi, w, h, lane);
+          } else {
+            hist_group<kLevel, false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
+          }
+        }
+        // 16 entries per lane and step: flush well before a 20-bit field can overflow
+        if (kLevel == 0 && (J0 & (512 * 8 - 1)) == 512 * 7) hist0_flush(acc, e_top, cnt, slo, shi, lane);
       }
       // the rest of the row, 128 entries at a time
       for (; J0 <= m; J0 += 128) {
         float z[4];
         load_z4<kVec>(row, J0 + 4 * lane, m, z);
-        hist_group<kLevel, true>(z, J0 + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
+        if (kLevel == 0) {
+          hist0_group<true>(z, J0 + 4 * lane, m, M, inv, e_top, acc, cnt, slo, shi, w, h, lane);
+        } else {
+          hist_group<kLevel, true>(z, J0 + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
+        }
       }
+      if (kLevel == 0) hist0_flush(acc, e_top, cnt, slo, shi, lane);
       if (kLevel == 2) {
         gt = warp_sum_i(gt);
         in = warp_sum_i(in);
@@ -923,7 +1001,7 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   // the last CTA of this head to get here locates the cut in the finished histogram
   __threadfence();
   __syncthreads();
-  if (tid == 0) is_last = atomicAdd(&w.hist_done[kLevel * d.hq + h], 1) == static_cast<int>(gridDim.x) - 1;
+  if (tid == 0) is_last = atomicAdd(&w.hist_done[kLevel * d.hq + h], 1) == n_ctas - 1;
   __syncthreads();
   if (!is_last) return;
   __threadfence();
@@ -1263,11 +1341,13 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
     const int grid = min(n_sm, nt * d.hq);
     CRISP_KERNEL("pe_logits", stream, launch_pdl(pe_logits_kernel, dim3(grid), dim3(320), smem, stream, maps, d, pattern, w, status));
   }
-  // up to four CTAs per SM if every head is PE (two when half of them are); a warp takes a row at a time
-  // ... and never more than 2^18 entries of a head per CTA (the 32-bit mass words of pe_hist_kernel)
+  // histogram passes: a warp takes a row at a time; the grid is sized for a single PE head, the kernel uses as many
+  // CTAs per head as make one full wave over the PE heads there are
   const long long causal = static_cast<long long>(d.nb) * (d.nb + 1) / 2;
-  int hist_ctas = max(1, min((d.nb + 15) / 16, (4 * n_sm + d.hq - 1) / d.hq));
-  hist_ctas = max(hist_ctas, static_cast<int>((causal + (1 << 18) - 1) >> 18));
+  // two CTAs of kHistThreads fit on an SM; a CTA must see fewer than 2^19 entries of a head (its 32-bit bin sums)
+  const int resident_ctas = 2 * n_sm;
+  const int min_ctas = static_cast<int>((causal + (1 << 19) - 1) >> 19);
+  const int hist_ctas = max(min_ctas, max(1, min((d.nb + 15) / 16, 64)));
   auto hist_smem = [](int level) { return static_cast<size_t>(level_bins(level)) * 12; };
   const bool vec = (d.nb & 3) == 0;  // rows start on 16-byte boundaries
   auto* hist0 = vec ? pe_hist_kernel<0, true> : pe_hist_kernel<0, false>;
@@ -1275,9 +1355,9 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   auto* hist2 = vec ? pe_hist_kernel<2, true> : pe_hist_kernel<2, false>;
   CRISP_CUDA_TRY(cudaFuncSetAttribute(hist1, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(hist_smem(1))),
                  "select: smem attribute");
-  CRISP_KERNEL("pe_hist0", stream, launch_pdl(hist0, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(0), stream, d, pattern, w));
-  CRISP_KERNEL("pe_hist1", stream, launch_pdl(hist1, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(1), stream, d, pattern, w));
-  CRISP_KERNEL("pe_hist2", stream, launch_pdl(hist2, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(2), stream, d, pattern, w));
+  CRISP_KERNEL("pe_hist0", stream, launch_pdl(hist0, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(0), stream, d, pattern, w, resident_ctas, min_ctas));
+  CRISP_KERNEL("pe_hist1", stream, launch_pdl(hist1, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(1), stream, d, pattern, w, resident_ctas, min_ctas));
+  CRISP_KERNEL("pe_hist2", stream, launch_pdl(hist2, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(2), stream, d, pattern, w, resident_ctas, min_ctas));
   const int rows_ctas = max(1, min((d.nb + 31) / 32, 8));
   CRISP_KERNEL("pe_rows", stream, launch_pdl(pe_rows_kernel, dim3(rows_ctas, d.hq), dim3(1024), 0, stream, d, pattern, w));
   CRISP_KERNEL("fill", stream, launch_pdl(fill_kernel, dim3((d.nb + 7) / 8, d.hq), dim3(256), 0, stream, 
