@@ -27,7 +27,7 @@ def pytest_collection_modifyitems(config, items):
 
 
 # Lines the parity tests want shown even under `-q` (sample sizes, excused counts, worst errors): they are
-# printed in the terminal summary and, on a GPU machine, appended to gpurun_out/parity_summary.txt.
+# printed in the terminal summary and, when CRISP_PARITY_SUMMARY names a file, appended to it.
 _PARITY_LINES = []
 
 
@@ -42,10 +42,12 @@ def pytest_terminal_summary(terminalreporter):
     terminalreporter.section("parity summary")
     for line in _PARITY_LINES:
         terminalreporter.write_line(line)
+    path = os.environ.get("CRISP_PARITY_SUMMARY")
+    if not path:
+        return
     try:
-        out = os.path.join(ROOT, "gpurun_out")
-        os.makedirs(out, exist_ok=True)
-        with open(os.path.join(out, "parity_summary.txt"), "a") as f:
+        os.makedirs(os.path.dirname(os.path.abspath(path)), exist_ok=True)
+        with open(path, "a") as f:
             f.write("\n".join(_PARITY_LINES) + "\n")
     except OSError:  # pragma: no cover
         pass
