@@ -705,7 +705,8 @@ __device__ void locate_cut(const Dims& d, const SelectPtrs& w, int h, int level,
   unsigned int hit_count = 0u;
 #pragma unroll
   for (int i = 0; i < kPer; ++i) {
-    if (my_hit == 0x7fffffff && cc[i] != 0u && before + mm[i] >= gamma) {
+    // (a bin is non-empty if it has a count or a mass: only the last level keeps counts on every path)
+    if (my_hit == 0x7fffffff && (cc[i] != 0u || mm[i] != 0ull) && before + mm[i] >= gamma) {
       my_hit = kPer * tid + i;
       hit_above = before;
       hit_count = cc[i];
@@ -815,11 +816,12 @@ __device__ __forceinline__ void hist_group(const float (&z)[4], int J, int m, fl
         hi += ((key[e] >> 12) & 0x7FFu) | 0x800u;
         bin[e] = -1;
       }
-    n = __reduce_add_sync(0xffffffffu, n);
+    // (counts matter at the last level only: above it a bin that received an entry has a non-zero mass)
+    if (kLevel == 2) n = __reduce_add_sync(0xffffffffu, n);
     lo = __reduce_add_sync(0xffffffffu, lo);
     hi = __reduce_add_sync(0xffffffffu, hi);
     if (lane == 0) {
-      atomicAdd(&cnt[ref], n);
+      if (kLevel == 2) atomicAdd(&cnt[ref], n);
       atomicAdd(&slo[ref], lo);
       atomicAdd(&shi[ref], hi);
     }
@@ -828,7 +830,7 @@ __device__ __forceinline__ void hist_group(const float (&z)[4], int J, int m, fl
 #pragma unroll
   for (int e = 0; e < 4; ++e)
     if (bin[e] >= 0) {
-      atomicAdd(&cnt[bin[e]], 1u);
+      if (kLevel == 2) atomicAdd(&cnt[bin[e]], 1u);
       atomicAdd(&slo[bin[e]], key[e] & 0xFFFu);
       atomicAdd(&shi[bin[e]], ((key[e] >> 12) & 0x7FFu) | 0x800u);
     }
@@ -990,7 +992,7 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
     unsigned int* gc = w.hcount + static_cast<size_t>(h) * kHistStride + level_offset(kLevel);
     unsigned long long* gm = w.hmass + static_cast<size_t>(h) * kHistStride + level_offset(kLevel);
     for (int i = tid; i < nbins; i += kHistThreads)
-      if (cnt[i]) {
+      if (cnt[i] | slo[i] | shi[i]) {
         // the bin's exponent: its own index at level 0, the cut's exponent below
         const int e = kLevel == 0 ? i : static_cast<int>(prefix >> kL0Shift);
         const unsigned long long sig = (static_cast<unsigned long long>(shi[i]) << 12) + slo[i];
