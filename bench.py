@@ -497,7 +497,7 @@ def main():
                      "peak": peak, "unit": "TFLOP/s", "frac": sparse_tflops / peak,
                      "peak_source": f"{peaks['source']} ({'sustained' if peak == peaks['bf16_sustained'] else 'burst'})",
                      "traffic": None,
-                     "traffic_note": "not captured in this run; ncu DRAM bytes of the kernel at L128k (4.66 GB per launch "
+                     "traffic_note": "not captured in this run; ncu DRAM bytes of the kernel at L128k (4.67 GB per launch "
                                      "for 2.68 GB algorithmic) are in profiles/dram_traffic_L128k_ncu.md",
                      "algorithmic_flop_per_launch": nnz * FLOP_PER_BLOCK},
         "stages_hbm": stages_hbm, "kernels": kernels, "near_threshold_excused": near,
