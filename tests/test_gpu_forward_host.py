@@ -40,6 +40,20 @@ def test_forward_host_equals_forward_for_every_chunking(gpc):
     assert rc == B.OK and torch.equal(oh2, o_ref)
 
 
+def test_forward_host_ragged_length_and_group_of_seven():
+    """A length that is not a multiple of the block and the Qwen-like group size (7 query heads per KV head)."""
+    n, hq, hkv = 1536 + 37, 14, 2
+    q, k, v = synth.random_qkv(n, hq, hkv, seed=9, device="cuda")
+    p = crisp.make_params(n, hq, hkv, sink_tokens=4, tau=0.05, k_min_blocks=2)
+    o_ref, pat_ref, nnz_ref = _whole_layer(p, q, k, v)
+    oh = torch.zeros_like(o_ref).pin_memory()
+    pat = torch.full((hq,), -1, dtype=torch.int32)
+    stage = torch.empty(B.crisp_forward_host_stage_bytes(p, 1), dtype=torch.uint8, device="cuda")
+    rc, nnz = B.crisp_forward_host(p, q.cpu().pin_memory(), k.cpu().pin_memory(), v.cpu().pin_memory(), oh, 1, stage,
+                                   pattern_host=pat)
+    assert rc == B.OK and torch.equal(oh, o_ref) and torch.equal(pat, pat_ref) and nnz == nnz_ref
+
+
 def test_forward_host_argument_checks():
     p = crisp.make_params(1024, 4, 2, sink_tokens=4, k_min_blocks=2)
     assert B.crisp_forward_host_stage_bytes(p, 3) == 0          # not a divisor of H_kv
