@@ -496,9 +496,15 @@ def main():
         "roofline": {"bound": "tensor", "kernel": "prefill_kernel<sparse>", "achieved": sparse_tflops,
                      "peak": peak, "unit": "TFLOP/s", "frac": sparse_tflops / peak,
                      "peak_source": f"{peaks['source']} ({'sustained' if peak == peaks['bf16_sustained'] else 'burst'})",
-                     "traffic": None,
-                     "traffic_note": "not captured in this run; ncu DRAM bytes of the kernel at L128k (4.67 GB per launch "
-                                     "for 2.68 GB algorithmic) are in profiles/dram_traffic_L128k_ncu.md",
+                     # ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel: constants
+                     # copied from the committed captures (nothing is parsed at run time); other workloads: null
+                     "traffic": {"L512k": 123_110_000_000, "L128k": 4_671_830_272}.get(wl.name) if wl.n_q_heads == w.n_q_heads else None,
+                     "traffic_source": {"L512k": "profiles/dram_traffic_L128k_ncu.md, section 'Earlier capture at L512k' "
+                                                 "(118.8 GB read + 4.31 GB written per launch; the attention kernel is "
+                                                 "unchanged since); algorithmic 10.7 GB: K/V are re-streamed per item "
+                                                 "and shared through L2",
+                                        "L128k": "profiles/dram_traffic_L128k_ncu.md (3.63 GB read + 1.04 GB written per "
+                                                 "launch for 2.68 GB algorithmic)"}.get(wl.name, "not captured for this workload"),
                      "algorithmic_flop_per_launch": nnz * FLOP_PER_BLOCK},
         "stages_hbm": stages_hbm, "kernels": kernels, "near_threshold_excused": near,
         "cpu_baseline": cpu_baseline, "e2e": e2e,
