@@ -228,7 +228,7 @@ def kernel_bytes(name, w, n_pe, n_kv_pe, nnz):
         "pe_logits": (n_pe + n_kv_pe) * nb * 768 + n_pe * causal * 4,           # bf16 terms read, logits written
         "pe_hist0": n_pe * causal * 4, "pe_hist1": n_pe * causal * 4, "pe_hist2": n_pe * causal * 4,
         "fill": n_pe * causal * 4 + nnz * 4 + 8 * hq * (nb + 1),
-        "merge_lists": nnz * 4,                                      # lists read (the union lists written on top)
+        "check_lists": nnz * 4,                                      # lists read once (validated before use)
     }
     return table.get(name)
 
@@ -498,12 +498,12 @@ def main():
                      "peak_source": f"{peaks['source']} ({'sustained' if peak == peaks['bf16_sustained'] else 'burst'})",
                      # ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel: constants
                      # copied from the committed captures (nothing is parsed at run time); other workloads: null
-                     "traffic": {"L512k": 123_110_000_000, "L128k": 4_671_830_272}.get(wl.name) if wl.n_q_heads == w.n_q_heads else None,
+                     "traffic": {"L512k": 123_110_000_000, "L128k": 4_711_334_912}.get(wl.name) if wl.n_q_heads == w.n_q_heads else None,
                      "traffic_source": {"L512k": "profiles/dram_traffic_L128k_ncu.md, section 'Earlier capture at L512k' "
-                                                 "(118.8 GB read + 4.31 GB written per launch; the attention kernel is "
+                                                 "(118.8 GB read + 4.31 GB written per launch; its tensor-core loop is "
                                                  "unchanged since); algorithmic 10.7 GB: K/V are re-streamed per item "
                                                  "and shared through L2",
-                                        "L128k": "profiles/dram_traffic_L128k_ncu.md (3.63 GB read + 1.04 GB written per "
+                                        "L128k": "profiles/dram_traffic_L128k_ncu.md (3.67 GB read + 1.04 GB written per "
                                                  "launch for 2.68 GB algorithmic)"}.get(wl.name, "not captured for this workload"),
                      "algorithmic_flop_per_launch": nnz * FLOP_PER_BLOCK},
         "stages_hbm": stages_hbm, "kernels": kernels, "near_threshold_excused": near,

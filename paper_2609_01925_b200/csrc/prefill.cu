@@ -3,7 +3,9 @@
 // One CTA processes work items; an item is one query head and a PAIR of adjacent query blocks
 // (two 128-row tiles).  Both tiles share every K/V block that TMA brings into shared memory, which
 // halves the L2 -> shared-memory traffic per flop.  The key blocks of the pair are the sorted union
-// of the two blocks' lists; each entry carries two flags saying which tile uses it.  (When the pairs of a problem
+// of the two blocks' lists, each with two flags saying which tile uses it; the union is never stored: the
+// producer and the issuers form it on the fly by a two-way merge of the two lists (EntryStream), and a tile's
+// softmax warps walk that tile's own list (TileReader).  (When the pairs of a problem
 // do not even fill the SMs, an item is a single query block instead: tile 1 stays idle, the CTAs are twice as many
 // and a block alone steps faster than a pair.)
 //
@@ -47,9 +49,8 @@ constexpr float kRescaleThreshold = 8.0f;  // log2 units
 constexpr int kStages = 5;                 // K/V ring slots of 32 KB
 
 struct PrefillArgs {
-  const int32_t* merged;   // per item: union list, entry = key block | flags (sparse only)
+  const int32_t* col_idx;  // the heads' lists (sparse only)
   const int64_t* row_ptr;  // [hq][nb+1]
-  const int* item_len;     // [hq][n_pairs] number of union entries (sparse only)
   const int* order;        // [n_items] item ids sorted by decreasing cost (sparse only)
   __nv_bfloat16* o;        // [n][hq][128]
   float* lse;              // [hq][n] or null
@@ -80,8 +81,9 @@ struct PrefillSmem {
 struct Item {
   int h, kvh, m0, m1;
   bool tile1;
-  int n_entries;
-  long long base;  // offset of the item's union list
+  int n_entries;    // dense: key blocks of the item; sparse: unused (the union's length is found by walking it)
+  int n0, n1;       // sparse: lengths of the two query blocks' lists (n1 = 0 without a second tile)
+  long long base0;  // sparse: offset of block m0's list in col_idx; block m1's follows it
 };
 
 template <bool kDense>
@@ -108,37 +110,40 @@ __device__ __forceinline__ Item decode_item(int pos, const Dims& d, const Prefil
   it.tile1 = a.rows_per_item == 2 && it.m1 < d.nb;
   if (kDense) {
     it.n_entries = it.tile1 ? it.m1 + 1 : it.m0 + 1;
-    it.base = 0;
+    it.n0 = it.n1 = 0;
+    it.base0 = 0;
   } else {
-    it.n_entries = a.item_len[it.h * a.n_pairs + u];
-    it.base = a.row_ptr[static_cast<size_t>(it.h) * (d.nb + 1) + it.m0];
+    const int64_t* rp = a.row_ptr + static_cast<size_t>(it.h) * (d.nb + 1) + it.m0;
+    it.n_entries = 0;
+    it.base0 = rp[0];
+    it.n0 = static_cast<int>(rp[1] - rp[0]);
+    it.n1 = it.tile1 ? static_cast<int>(rp[2] - rp[1]) : 0;
   }
   return it;
 }
 
-// Entry e of an item: key block and per-tile flags.  Sparse lists are fetched 32 entries at a time,
-// one per lane, and broadcast with a shuffle; all 32 lanes of the warp must call this together.
+// The key blocks of ONE tile of an item, in order (what its softmax warps walk: they need neither the other
+// tile's blocks nor the position of a block in the K/V stream).  Sparse lists are fetched 32 entries at a time,
+// one per lane, and broadcast with a shuffle; all 32 lanes of the warp must call get together.
 template <bool kDense>
-struct EntryReader {
+struct TileReader {
   const int32_t* list;
   uint32_t chunk;
-  int m0;
-  bool tile1;
-  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& a) {
-    list = kDense ? nullptr : a.merged + it.base;
-    m0 = it.m0;
-    tile1 = it.tile1;
+  int n;  // blocks of the tile
+  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& a, int t) {
+    if (kDense) {
+      list = nullptr;
+      n = (t == 0 ? it.m0 : it.m1) + 1;
+    } else {
+      list = a.col_idx + it.base0 + (t == 0 ? 0 : it.n0);
+      n = t == 0 ? it.n0 : it.n1;
+    }
     chunk = 0;
   }
-  __device__ __forceinline__ uint32_t get(int e, int n_entries, int lane) {
-    if (kDense) {
-      uint32_t x = static_cast<uint32_t>(e);
-      if (e <= m0) x |= kFlag0;
-      if (tile1) x |= kFlag1;
-      return x;
-    }
-    if ((e & 31) == 0) chunk = (e + lane < n_entries) ? static_cast<uint32_t>(list[e + lane]) : 0u;
-    return __shfl_sync(0xffffffffu, chunk, e & 31);
+  __device__ __forceinline__ int get(int i, int lane) {
+    if (kDense) return i;
+    if ((i & 31) == 0) chunk = (i + lane < n) ? static_cast<uint32_t>(list[i + lane]) : 0u;
+    return static_cast<int>(__shfl_sync(0xffffffffu, chunk, i & 31));
   }
 };
 
@@ -276,31 +281,63 @@ __device__ __forceinline__ float exp_pack(const uint32_t (&x)[2][32], int r, int
   return (s0 + s1) + (s2 + s3);
 }
 
-// Entry stream for a role run by a single thread: the next entry is fetched one iteration early, so the
-// global-load latency hides behind the current step.
+// The K/V blocks of an item in the order they are loaded - the sorted union of the two query blocks' lists, each
+// entry with two flags saying which tile uses it - for a role run by a single thread (producer, issuers).  The
+// union is formed on the fly by a two-way merge of the lists; each list's next element is fetched one call early,
+// so the global-load latency hides behind the current step.
 template <bool kDense>
 struct EntryStream {
-  const int32_t* list;
-  uint32_t next;
-  int m0, n_entries;
+  static constexpr int kEnd = 0x3fffffff;  // larger than any key block, below the flag bits
+  const int32_t *l0, *l1;
+  int n0, n1, i0, i1;
+  int a, b, a_nx, b_nx;  // heads of the two lists and their successors (kEnd: exhausted)
+  int e, m0, n_entries;  // dense
   bool tile1;
-  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& a) {
-    list = kDense ? nullptr : a.merged + it.base;
+  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& args) {
     m0 = it.m0;
     tile1 = it.tile1;
     n_entries = it.n_entries;
-    next = (!kDense && n_entries > 0) ? static_cast<uint32_t>(__ldg(list)) : 0u;
+    e = 0;
+    if (!kDense) {
+      l0 = args.col_idx + it.base0;
+      l1 = l0 + it.n0;
+      n0 = it.n0;
+      n1 = it.n1;
+      i0 = i1 = 0;
+      a = n0 > 0 ? __ldg(l0) : kEnd;
+      a_nx = n0 > 1 ? __ldg(l0 + 1) : kEnd;
+      b = n1 > 0 ? __ldg(l1) : kEnd;
+      b_nx = n1 > 1 ? __ldg(l1 + 1) : kEnd;
+    }
   }
-  __device__ __forceinline__ uint32_t get(int e) {
+  // the next entry of the stream; false when there is none
+  __device__ __forceinline__ bool next(uint32_t* ent) {
     if (kDense) {
+      if (e >= n_entries) return false;
       uint32_t x = static_cast<uint32_t>(e);
       if (e <= m0) x |= kFlag0;
       if (tile1) x |= kFlag1;
-      return x;
+      ++e;
+      *ent = x;
+      return true;
     }
-    const uint32_t cur = next;
-    if (e + 1 < n_entries) next = static_cast<uint32_t>(__ldg(list + e + 1));
-    return cur;
+    const int J = min(a, b);
+    if (J == kEnd) return false;
+    uint32_t x = static_cast<uint32_t>(J);
+    if (a == J) {
+      x |= kFlag0;
+      ++i0;
+      a = a_nx;
+      a_nx = i0 + 1 < n0 ? __ldg(l0 + i0 + 1) : kEnd;
+    }
+    if (b == J) {
+      x |= kFlag1;
+      ++i1;
+      b = b_nx;
+      b_nx = i1 + 1 < n1 ? __ldg(l1 + i1 + 1) : kEnd;
+    }
+    *ent = x;
+    return true;
   }
 };
 
@@ -382,8 +419,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           tma_load_3d(s.q[1][0], &tmap_q, &s.q_full, 0, it.h, it.m1 * kBlock);
           tma_load_3d(s.q[1][1], &tmap_q, &s.q_full, 64, it.h, it.m1 * kBlock);
         }
-        for (int e = 0; e < it.n_entries && ok; ++e, ++ecount) {
-          const uint32_t ent = rd.get(e);
+        uint32_t ent;
+        for (; ok && rd.next(&ent); ++ecount) {
           const int J = static_cast<int>(ent & kColMask);
           // loads 2*ecount (K) and 2*ecount + 1 (V) go to consecutive ring slots
 #pragma unroll
@@ -487,21 +524,21 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         const Item it = decode_item<kDense>(idx, d, a);
         ok = mbar_wait(&s.q_full, it_count & 1, abort_flag);
         if (!ok) break;
-        const uint32_t item_loads_end = 2u * (ecount_base + it.n_entries);
         if (t == 1 && !it.tile1) {
-          // an item without a second tile: see its loads through and release Q
-          skip_to(item_loads_end);
+          // an item without a second tile: see its loads through (the K/V stream is block m0's list) and release Q
+          const uint32_t n_stream = kDense ? it.n_entries : it.n0;
+          skip_to(2u * (ecount_base + n_stream));
           if (ok) mbar_arrive(&s.q_free);
-          ecount_base += it.n_entries;
+          ecount_base += n_stream;
           continue;
         }
         EntryStream<kDense> rd;
         rd.init(it, a);
-        int e = 0;
-        // next step of this tile: walks the union list (flags only, never waits)
+        uint32_t e = 0;  // entries of the item's K/V stream walked so far
+        // next step of this tile: walks the stream (flags only, never waits)
         auto find_next = [&](Step& st) {
-          while (e < it.n_entries) {
-            const uint32_t ent = rd.get(e);
+          uint32_t ent;
+          while (rd.next(&ent)) {
             ++e;
             if (ent & flag_t) {
               st.ec = ecount_base + e - 1;
@@ -563,8 +600,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
           cur = nx;
           have = have_nx;
         }
-        skip_to(item_loads_end);  // blocks after this tile's diagonal belong to the other tile
-        ecount_base += it.n_entries;
+        // blocks after this tile's diagonal belong to the other tile: walk the stream to its end and see them through
+        {
+          Step rest;
+          while (find_next(rest)) {}
+        }
+        skip_to(2u * (ecount_base + e));
+        ecount_base += e;
       }
     }
     __syncwarp();
@@ -600,15 +642,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       if (idx < 0) break;
       const Item it = decode_item<kDense>(idx, d, a);
       if (t == 1 && !it.tile1) continue;
-      EntryReader<kDense> rd;
-      rd.init(it, a);
+      TileReader<kDense> rd;
+      rd.init(it, a, t);
       const int m_t = t == 0 ? it.m0 : it.m1;
       float m_used = 0.f, l_run = 0.f;
       bool first = true;
-      for (int e = 0; e < it.n_entries && ok; ++e) {
-        const uint32_t ent = rd.get(e, it.n_entries, lane);
-        if (!(ent & (t == 0 ? kFlag0 : kFlag1))) continue;
-        const int J = static_cast<int>(ent & kColMask);
+      for (int i = 0; i < rd.n && ok; ++i) {
+        const int J = rd.get(i, lane);
         const bool diag = (J == m_t);
         const uint32_t ph = step_count & 1;
         // Each 64-key half is one step of the online softmax.  The rescale decision is taken per warp
@@ -710,105 +750,61 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
   if (warp == 8) tmem_dealloc(tm, 512);
 }
 
-// Union of the lists of query blocks (2u, 2u+1) of one head, with per-tile flags.  One warp per pair;
-// the two lists become bitmaps in shared memory, the union is emitted in ascending order.
-__device__ __forceinline__ void merge_pair(const Dims& d, const int64_t* __restrict__ row_ptr,
-                                           const int32_t* __restrict__ col_idx, int32_t* __restrict__ merged,
-                                           int* __restrict__ item_len, int* __restrict__ cost_hist, int n_pairs,
-                                           int n_cost, int group_kv, int* __restrict__ status,
-                                           long long merged_capacity, uint32_t* b0, uint32_t* b1, int words, int u,
-                                           int h, int lane, int rows_per_item) {
+// The lists of one item (query blocks m0 and, if the item is a pair, m0 + 1 of one head), checked before the
+// attention kernel walks them.  The lists may come from the caller, so nothing about them is trusted: a row of
+// query block m must hold between 1 and m + 1 entries inside the range `capacity` bounds, strictly ascending,
+// none above m, the last one m itself (the diagonal block, which the attention kernel's Q hand-over relies on).
+// Anything else marks the launch CRISP_ERR_BAD_LIST, and the attention kernel, which reads the status word,
+// does no work at all.  One warp per item; it also enters the item into the histogram of the schedule's sort
+// keys.
+__global__ void __launch_bounds__(128)
+check_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
+                   int* __restrict__ cost_hist, int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate,
+                   int* __restrict__ status, long long capacity, int rows_per_item) {
+  pdl_enter();
+  if (gate != nullptr && *gate != 0) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
+  if (u >= n_pairs) return;
   const int m0 = rows_per_item * u, m1 = m0 + 1;
-  for (int i = lane; i < 2 * words; i += 32) b0[i] = 0u;
-  __syncwarp();
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int64_t s0 = rp[m0], e0 = rp[m0 + 1];
   const bool has1 = rows_per_item == 2 && m1 < d.nb;
   const int64_t e1 = has1 ? rp[m1 + 1] : e0;
-  // The lists may come from the caller, so nothing about them is trusted: a row of query block m must hold
-  // between 1 and m + 1 entries inside the workspace's range, strictly ascending, none above m, the last
-  // one m itself (the diagonal block, which the attention kernel's Q hand-over relies on).  Anything else
-  // marks the launch CRISP_ERR_BAD_LIST; nothing derived from a bad row is written and the attention
-  // kernel, which reads the status word, does no work at all.
-  bool bad = s0 < 0 || e0 - s0 < 1 || e0 - s0 > m0 + 1 || e1 > merged_capacity ||
-             (has1 && (e1 - e0 < 1 || e1 - e0 > m1 + 1));
-  // four loads per lane in flight before the bitmap updates
-  auto mark = [&](uint32_t* bits, int64_t from, int64_t to, int m) {
-    int prev_last = -1;  // last entry of the previous group of 32
-    for (int64_t i0 = from; i0 < to; i0 += 128) {
-      int c[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int64_t i = i0 + 32 * u + lane;
-        c[u] = i < to ? col_idx[i] : -1;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int64_t i = i0 + 32 * u + lane;
-        const bool live = i < to;
-        int before = __shfl_up_sync(0xffffffffu, c[u], 1);
-        if (lane == 0) before = prev_last;
-        const bool okc = !live || (c[u] >= 0 && c[u] <= m && c[u] > before && (i + 1 < to || c[u] == m));
-        bad = bad || !okc;
-        prev_last = __shfl_sync(0xffffffffu, c[u], 31);
-        // the entries ascend, so the 32 of a load fall into one or two words (more in a thin list): lanes with the
-        // same word combine their bits and one of them updates the bitmap
-        const int wd = (live && okc) ? (c[u] >> 5) : -1;
-        const unsigned int peers = __match_any_sync(0xffffffffu, wd);
-        const uint32_t mine = wd >= 0 ? (1u << (c[u] & 31)) : 0u;
-        const uint32_t all = __reduce_or_sync(peers, mine);
-        if (wd >= 0 && lane == __ffs(peers) - 1) atomicOr(&bits[wd], all);
-      }
-    }
-  };
+  bool bad = s0 < 0 || e0 - s0 < 1 || e0 - s0 > m0 + 1 || e1 > capacity || (has1 && (e1 - e0 < 1 || e1 - e0 > m1 + 1));
   if (!bad) {
-    mark(b0, s0, e0, m0);
-    if (has1) mark(b1, e0, e1, m1);
+    // four loads per lane in flight; an entry is compared with the one before it (the lane below, or the last
+    // entry of the previous group of 32)
+    auto check = [&](int64_t from, int64_t to, int m) {
+      int prev_last = -1;
+      for (int64_t i0 = from; i0 < to; i0 += 128) {
+        int c[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const int64_t i = i0 + 32 * v + lane;
+          c[v] = i < to ? col_idx[i] : 0x7fffffff;
+        }
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+          const int64_t i = i0 + 32 * v + lane;
+          const bool live = i < to;
+          int before = __shfl_up_sync(0xffffffffu, c[v], 1);
+          if (lane == 0) before = prev_last;
+          bad = bad || (live && !(c[v] >= 0 && c[v] <= m && c[v] > before && (i + 1 < to || c[v] == m)));
+          prev_last = __shfl_sync(0xffffffffu, c[v], 31);
+        }
+      }
+    };
+    check(s0, e0, m0);
+    if (has1) check(e0, e1, m1);
   }
   if (__any_sync(0xffffffffu, bad)) {
     if (lane == 0) atomicExch(status, CRISP_ERR_BAD_LIST);
     return;
   }
-  __syncwarp();
-  int32_t* out = merged + s0;
-  int written = 0;
-  // one 32-block word per step, lane b owning bit b: the entries of a word go out as one contiguous store
-  const int last_word = min(words - 1, (has1 ? m1 : m0) >> 5);
-  for (int wd = 0; wd <= last_word; ++wd) {
-    const uint32_t x0 = b0[wd], x1 = b1[wd];  // broadcast reads
-    const uint32_t un = x0 | x1;
-    if (un == 0u) continue;
-    if ((un >> lane) & 1u) {
-      uint32_t ent = static_cast<uint32_t>(wd * 32 + lane);
-      if ((x0 >> lane) & 1u) ent |= kFlag0;
-      if ((x1 >> lane) & 1u) ent |= kFlag1;
-      out[written + __popc(un & ((1u << lane) - 1u))] = static_cast<int32_t>(ent);
-    }
-    written += __popc(un);
-  }
-  if (lane == 0) {
-    item_len[h * n_pairs + u] = written;
-    // sort key: KV head first, then decreasing cost (= tile steps = len(m0) + len(m1))
+  // sort key: KV head first, then decreasing cost (= tile steps = len(m0) + len(m1))
+  if (lane == 0)
     atomicAdd(&cost_hist[(group_kv ? h / d.group : 0) * n_cost + (n_cost - 1 - static_cast<int>(e1 - s0))], 1);
-  }
-}
-
-// One warp per pair of query blocks; each also enters its pair into the histogram of the schedule's sort keys.
-__global__ void __launch_bounds__(128)
-merge_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
-                   int32_t* __restrict__ merged, int* __restrict__ item_len, int* __restrict__ cost_hist,
-                   int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate, int* __restrict__ status,
-                   long long merged_capacity, int rows_per_item) {
-  pdl_enter();
-  extern __shared__ uint32_t bm[];
-  if (gate != nullptr && *gate != 0) return;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
-  const int words = (d.nb + 31) / 32;
-  uint32_t* b0 = bm + static_cast<size_t>(warp) * 2 * words;
-  if (u < n_pairs)
-    merge_pair(d, row_ptr, col_idx, merged, item_len, cost_hist, n_pairs, n_cost, group_kv, status, merged_capacity,
-               b0, b0 + words, words, u, h, lane, rows_per_item);
 }
 
 // Counting sort of the items by (KV head, decreasing cost).  Grouping by KV head keeps the CTAs that
@@ -850,14 +846,12 @@ sched_scatter_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const in
 }
 
 struct PrefillWs {
-  int* item_len;
   int* order;
   int* cost_hist;
   int* cursor;  // per sort key: items placed so far
   int n_cost;  // distinct cost values (0 .. 2 N_b + 1)
   int n_bins;  // n_cost per KV head
   size_t zero_bytes;  // header + histogram
-  int32_t* merged;
 };
 
 PrefillWs carve(const Dims& d, void* ws, size_t* total) {
@@ -873,12 +867,8 @@ PrefillWs carve(const Dims& d, void* ws, size_t* total) {
   w.cursor = reinterpret_cast<int*>(base + off);
   off += align_up(sizeof(int) * static_cast<size_t>(w.n_bins), 256);
   w.zero_bytes = off;
-  w.item_len = reinterpret_cast<int*>(base + off);
-  off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
   w.order = reinterpret_cast<int*>(base + off);
   off += align_up(sizeof(int) * static_cast<size_t>(d.hq) * n_pairs, 256);
-  w.merged = reinterpret_cast<int32_t*>(base + off);
-  off += align_up(sizeof(int32_t) * static_cast<size_t>(d.hq) * d.nb * (static_cast<size_t>(d.nb) + 1) / 2, 256);
   *total = off;
   return w;
 }
@@ -913,9 +903,8 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   a.rows_per_item = ((d.nb + 1) / 2) * d.hq < n_sm ? 1 : 2;
   a.n_pairs = (d.nb + a.rows_per_item - 1) / a.rows_per_item;
   a.n_items = a.n_pairs * d.hq;
-  a.merged = w.merged;
+  a.col_idx = col_idx;
   a.row_ptr = row_ptr;
-  a.item_len = w.item_len;
   a.order = w.order;
   a.o = static_cast<__nv_bfloat16*>(o);
   a.lse = lse;
@@ -936,10 +925,11 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
                    "prefill: smem attribute");
     CRISP_KERNEL("prefill_dense", stream, launch_pdl(prefill_kernel<true>, dim3(grid), dim3(384), smem, stream, tq, tk, tv, d, a));
   } else {
-    const int words = (d.nb + 31) / 32;
-    CRISP_KERNEL("merge_lists", stream, launch_pdl(merge_lists_kernel, dim3((a.n_pairs + 3) / 4, d.hq), dim3(128), sizeof(uint32_t) * 8 * words, stream, 
-        d, row_ptr, col_idx, w.merged, w.item_len, w.cost_hist, a.n_pairs, w.n_cost, a.group_kv, gate, a.status,
-        static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2, a.rows_per_item));
+    // the lists are checked (and the items entered into the schedule's histogram) before anything walks them
+    const long long capacity = static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2;
+    CRISP_KERNEL("check_lists", stream,
+                 launch_pdl(check_lists_kernel, dim3((a.n_pairs + 3) / 4, d.hq), dim3(128), 0, stream, d, row_ptr, col_idx, w.cost_hist,
+                            a.n_pairs, w.n_cost, a.group_kv, gate, a.status, capacity, a.rows_per_item));
     const size_t scatter_smem = sizeof(int) * static_cast<size_t>(w.n_cost);
     if (scatter_smem > 48 * 1024)
       CRISP_CUDA_TRY(cudaFuncSetAttribute(sched_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
