@@ -226,6 +226,7 @@ def kernel_bytes(name, w, n_pe, n_kv_pe, nnz):
         "tile_sums": partial + 2 * 4 * nb * hq,                     # partials read, p_v and p_s written
         "prepare": (n_pe + n_kv_pe) * n * 256 + (n_pe + n_kv_pe) * nb * 1280,   # Q of PE heads, K; pooled means
         "pe_logits": (n_pe + n_kv_pe) * nb * 768 + n_pe * causal * 4,           # bf16 terms read, logits written
+        "pe_small": (n_pe + n_kv_pe) * nb * 512 + n_pe * causal * 4,   # short prompts: block means read, logits written
         "pe_hist0": n_pe * causal * 4, "pe_hist1": n_pe * causal * 4, "pe_hist2": n_pe * causal * 4,
         "fill": n_pe * causal * 4 + nnz * 4 + 8 * hq * (nb + 1),
         "check_lists": nnz * 4,                                      # lists read once (validated before use)

@@ -1010,6 +1010,211 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   locate_cut(d, w, h, kLevel, warp_tot, &first_hit);
 }
 
+// ------------------------------------------------------------------------------------------------
+// PE heads of short prompts (N_b <= kSmallNb, i.e. up to 8064 tokens): pooled logits, row statistics and the
+// gamma cut in one CTA
+// ------------------------------------------------------------------------------------------------
+// With at most 2016 causal entries per head the tensor-core kernel and the three histogram launches are all
+// fixed cost (~70 us together at 4096 tokens).  One CTA per PE head does the same work out of shared memory:
+// fp32 dot products of the block means, the rows' maxima and sums, a bitonic sort of the values and a prefix sum
+// of their masses in sorted order, which gives the cut directly.  It leaves exactly what pe_logits_kernel and the histogram levels
+// leave (the logits, the rows' normalisers, the cut state, and per row the number of entries above the cut's key
+// and equal to it), so pe_rows_kernel and fill_kernel follow unchanged.
+constexpr int kSmallNb = 63;  // 2016 entries: the sort network stays at 2048 keys
+constexpr int kSmallPitch = 132;  // floats per block mean in shared memory: 16-byte aligned rows, no bank conflicts
+struct SmallSmem {
+  float q[kSmallNb * kSmallPitch];
+  float k[kSmallNb * kSmallPitch];
+  float z[kSmallNb * (kSmallNb + 1) / 2];
+  unsigned int key[2048];  // the entries' values as bit patterns, sorted in descending order (zero-padded)
+  float row_m[kSmallNb], row_inv[kSmallNb];
+  long long scratch[33];
+  int first, run_start, run_len;
+  unsigned long long above;
+  CutState cut;
+};
+__global__ void __launch_bounds__(1024)
+pe_small_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs w) {
+  pdl_enter();
+  const int h = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (pattern[h] != CRISP_PATTERN_PE) return;
+  extern __shared__ uint8_t small_raw[];
+  SmallSmem& s = *reinterpret_cast<SmallSmem*>(small_raw);
+  const int nb = d.nb, n_entries = nb * (nb + 1) / 2, kvh = h / d.group;
+  // ---- block means of Q (this head) and K (its KV head)
+  const float* qb = w.qbar + static_cast<size_t>(h) * nb * kHeadDim;
+  const float* kb = w.kbar + static_cast<size_t>(kvh) * nb * kHeadDim;
+  for (int i = tid; i < nb * (kHeadDim / 4); i += 1024) {
+    const int r = i / (kHeadDim / 4), c4 = i % (kHeadDim / 4);
+    *reinterpret_cast<float4*>(&s.q[r * kSmallPitch + 4 * c4]) = reinterpret_cast<const float4*>(qb)[i];
+    *reinterpret_cast<float4*>(&s.k[r * kSmallPitch + 4 * c4]) = reinterpret_cast<const float4*>(kb)[i];
+  }
+  __syncthreads();
+  // ---- pooled logits in base-2 units, entry e = (m, J) in row-major order of the causal triangle
+  float* am = w.amat + static_cast<size_t>(h) * nb * nb;
+  for (int e = tid; e < n_entries; e += 1024) {
+    int m = static_cast<int>((sqrtf(8.0f * static_cast<float>(e) + 1.0f) - 1.0f) * 0.5f);
+    while (m * (m + 1) / 2 > e) --m;
+    while ((m + 1) * (m + 2) / 2 <= e) ++m;
+    const int J = e - m * (m + 1) / 2;
+    const float4* qv = reinterpret_cast<const float4*>(&s.q[m * kSmallPitch]);
+    const float4* kv = reinterpret_cast<const float4*>(&s.k[J * kSmallPitch]);
+    float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < kHeadDim / 4; ++c) {
+      const float4 a = qv[c], b = kv[c];
+      acc0 = fmaf(a.x, b.x, acc0);
+      acc1 = fmaf(a.y, b.y, acc1);
+      acc2 = fmaf(a.z, b.z, acc2);
+      acc3 = fmaf(a.w, b.w, acc3);
+    }
+    const float z = ((acc0 + acc1) + (acc2 + acc3)) * d.scale_log2;
+    s.z[e] = z;
+    am[static_cast<size_t>(m) * nb + J] = z;
+  }
+  __syncthreads();
+  // ---- rows: maximum and 1 / (sum N_b), one warp per row
+  for (int m = warp; m < nb; m += 32) {
+    const float* zr = &s.z[m * (m + 1) / 2];
+    float mx = -INFINITY;
+    for (int J = lane; J <= m; J += 32) mx = fmaxf(mx, zr[J]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.f;
+    for (int J = lane; J <= m; J += 32) sum += ex2(zr[J] - mx);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) {
+      const float inv = 1.0f / (sum * static_cast<float>(nb));
+      s.row_m[m] = mx;
+      s.row_inv[m] = inv;
+      w.row_m[static_cast<size_t>(h) * nb + m] = mx;
+      w.row_inv[static_cast<size_t>(h) * nb + m] = inv;
+    }
+  }
+  __syncthreads();
+  // ---- the entries' keys (bit patterns of the values), padded with zeros to a power of two and sorted in
+  // descending order (bitonic network in shared memory)
+  int padded = 1024;
+  while (padded < n_entries) padded <<= 1;
+  for (int e = tid; e < padded; e += 1024) {
+    unsigned int key = 0u;
+    if (e < n_entries) {
+      int m = static_cast<int>((sqrtf(8.0f * static_cast<float>(e) + 1.0f) - 1.0f) * 0.5f);
+      while (m * (m + 1) / 2 > e) --m;
+      while ((m + 1) * (m + 2) / 2 <= e) ++m;
+      key = __float_as_uint(pe_value(s.z[e], s.row_m[m], s.row_inv[m]));
+    }
+    s.key[e] = key;
+  }
+  if (tid == 0) {
+    s.first = 0x7fffffff;
+    s.run_start = 0;
+    s.run_len = 0;
+    s.above = 0ull;
+  }
+  __syncthreads();
+  for (int size = 2; size <= padded; size <<= 1)
+    for (int stride = size >> 1; stride > 0; stride >>= 1) {
+      for (int t = tid; t < (padded >> 1); t += 1024) {
+        const int lo = ((t & ~(stride - 1)) << 1) | (t & (stride - 1)), hi = lo + stride;  // (stride is a power of two)
+        const bool descending = (lo & size) == 0;
+        const unsigned int a = s.key[lo], b = s.key[hi];
+        if ((a < b) == descending) {
+          s.key[lo] = b;
+          s.key[hi] = a;
+        }
+      }
+      __syncthreads();
+    }
+  // ---- the cut: the first position of the sorted order at which the running mass reaches gamma
+  const double gd = static_cast<double>(d.gamma) * static_cast<double>(kMassScale);
+  const unsigned long long gamma = gd >= 1.8e19 ? 0xffffffffffffffffull : static_cast<unsigned long long>(gd);
+  const int per = padded >> 10;  // consecutive positions per thread
+  unsigned long long mass[2];
+  unsigned long long local = 0ull;
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    mass[i] = i < per ? __float2ull_rn(__uint_as_float(s.key[tid * per + i]) * kMassScale) : 0ull;
+    local += mass[i];
+  }
+  long long total_ll;
+  unsigned long long before = static_cast<unsigned long long>(
+      block_exclusive_scan_1024(static_cast<long long>(local), s.scratch, &total_ll));  // (the total is below 2^61)
+  {
+    unsigned long long run = before;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+      if (i < per) {
+        if (run < gamma && run + mass[i] >= gamma) s.first = tid * per + i;  // exactly one position qualifies
+        run += mass[i];
+      }
+  }
+  __syncthreads();
+  CutState c;
+  c.prefix = 0u;
+  c.cutkey = 0u;
+  c.mass_above = 0ull;
+  c.take = -1;  // the target exceeds the total mass (gamma >= 1 or rounding): keep every causal entry
+  if (s.first != 0x7fffffff && s.first < n_entries) {
+    const unsigned int cutkey = s.key[s.first];
+    // the run of entries equal to the cut's key: where it starts (the mass before it is the mass above the cut)
+    // and how long it is
+    {
+      unsigned long long run = before;
+      int mine = 0;
+#pragma unroll
+      for (int i = 0; i < 2; ++i)
+        if (i < per) {
+          const int pos = tid * per + i;
+          if (s.key[pos] == cutkey && pos < n_entries) {
+            ++mine;
+            if (pos == 0 || s.key[pos - 1] != cutkey) {
+              s.run_start = pos;
+              s.above = run;
+            }
+          }
+          run += mass[i];
+        }
+      if (mine) atomicAdd(&s.run_len, mine);
+    }
+    __syncthreads();
+    // all entries at the cut are equal; t = the smallest count whose mass reaches gamma
+    const unsigned long long v = __float2ull_rn(__uint_as_float(cutkey) * kMassScale);
+    long long t = 1;
+    if (v > 0ull) t = static_cast<long long>((gamma - s.above + v - 1ull) / v);
+    if (t < 1) t = 1;
+    if (t > s.run_len) t = s.run_len;
+    c.prefix = cutkey;
+    c.cutkey = cutkey;
+    c.mass_above = s.above;
+    c.take = t;
+  }
+  if (tid == 0) {
+    s.cut = c;
+    w.cut[h] = c;
+  }
+  if (c.take == -1) return;
+
+  // ---- per row: entries above the cut's key and equal to it
+  for (int m = warp; m < nb; m += 32) {
+    const float* zr = &s.z[m * (m + 1) / 2];
+    const float M = s.row_m[m], inv = s.row_inv[m];
+    int gt = 0, eq = 0;
+    for (int J = lane; J <= m; J += 32) {
+      const unsigned int kk = __float_as_uint(pe_value(zr[J], M, inv));
+      gt += kk > c.cutkey;
+      eq += kk == c.cutkey;
+    }
+    gt = warp_sum_i(gt);
+    eq = warp_sum_i(eq);
+    if (lane == 0) {
+      w.n_gt[static_cast<size_t>(h) * nb + m] = gt;
+      w.n_eq[static_cast<size_t>(h) * nb + m] = eq;
+    }
+  }
+}
+
 // Per PE head: exact per-row counts of the entries above and tied with the cut, the ties taken per row (in
 // row-major order: row m takes clamp(T - ties in rows < m, 0, ties_m)), the row lengths and their prefix sum.
 // Only rows with an entry inside the cut's last bin (2048 adjacent fp32 values) are read again; the last CTA of a head to finish
@@ -1327,39 +1532,47 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   int dev = 0, n_sm = 0;
   CRISP_CUDA_TRY(cudaGetDevice(&dev), "select: device");
   CRISP_CUDA_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev), "select: SM count");
-  {
-    LogitsMaps maps;
-    for (int pl = 0; pl < 3; ++pl) {
-      rc = make_tmap_bf16_nhd(&maps.q[pl], w.qsplit + static_cast<size_t>(pl) * d.nb * d.hq * kHeadDim, d.nb, d.hq);
-      if (rc != CRISP_OK) return rc;
-      rc = make_tmap_bf16_nhd(&maps.k[pl], w.ksplit + static_cast<size_t>(pl) * d.nb * d.hkv * kHeadDim, d.nb, d.hkv);
-      if (rc != CRISP_OK) return rc;
-    }
-    const size_t smem = sizeof(LogitsSmem) + 1024;
-    CRISP_CUDA_TRY(cudaFuncSetAttribute(pe_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        static_cast<int>(smem)),
+  if (d.nb <= kSmallNb) {
+    // short prompt: logits, row statistics and the cut of a PE head in one CTA
+    CRISP_CUDA_TRY(cudaFuncSetAttribute(pe_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(sizeof(SmallSmem))),
                    "select: smem attribute");
-    const int nt = (d.nb + kBlock - 1) / kBlock;
-    const int grid = min(n_sm, nt * d.hq);
-    CRISP_KERNEL("pe_logits", stream, launch_pdl(pe_logits_kernel, dim3(grid), dim3(320), smem, stream, maps, d, pattern, w, status));
+    CRISP_KERNEL("pe_small", stream, launch_pdl(pe_small_kernel, dim3(d.hq), dim3(1024), sizeof(SmallSmem), stream, d, pattern, w));
+  } else {
+    {
+      LogitsMaps maps;
+      for (int pl = 0; pl < 3; ++pl) {
+        rc = make_tmap_bf16_nhd(&maps.q[pl], w.qsplit + static_cast<size_t>(pl) * d.nb * d.hq * kHeadDim, d.nb, d.hq);
+        if (rc != CRISP_OK) return rc;
+        rc = make_tmap_bf16_nhd(&maps.k[pl], w.ksplit + static_cast<size_t>(pl) * d.nb * d.hkv * kHeadDim, d.nb, d.hkv);
+        if (rc != CRISP_OK) return rc;
+      }
+      const size_t smem = sizeof(LogitsSmem) + 1024;
+      CRISP_CUDA_TRY(cudaFuncSetAttribute(pe_logits_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(smem)),
+                     "select: smem attribute");
+      const int nt = (d.nb + kBlock - 1) / kBlock;
+      const int grid = min(n_sm, nt * d.hq);
+      CRISP_KERNEL("pe_logits", stream, launch_pdl(pe_logits_kernel, dim3(grid), dim3(320), smem, stream, maps, d, pattern, w, status));
+    }
+    // histogram passes: a warp takes a row at a time; the grid is sized for a single PE head, the kernel uses as many
+    // CTAs per head as make one full wave over the PE heads there are
+    const long long causal = static_cast<long long>(d.nb) * (d.nb + 1) / 2;
+    // two CTAs of kHistThreads fit on an SM; a CTA must see fewer than 2^19 entries of a head (its 32-bit bin sums)
+    const int resident_ctas = 2 * n_sm;
+    const int min_ctas = static_cast<int>((causal + (1 << 19) - 1) >> 19);
+    const int hist_ctas = max(min_ctas, max(1, min((d.nb + 15) / 16, 64)));
+    auto hist_smem = [](int level) { return static_cast<size_t>(level_bins(level)) * 12; };
+    const bool vec = (d.nb & 3) == 0;  // rows start on 16-byte boundaries
+    auto* hist0 = vec ? pe_hist_kernel<0, true> : pe_hist_kernel<0, false>;
+    auto* hist1 = vec ? pe_hist_kernel<1, true> : pe_hist_kernel<1, false>;
+    auto* hist2 = vec ? pe_hist_kernel<2, true> : pe_hist_kernel<2, false>;
+    CRISP_CUDA_TRY(cudaFuncSetAttribute(hist1, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(hist_smem(1))),
+                   "select: smem attribute");
+    CRISP_KERNEL("pe_hist0", stream, launch_pdl(hist0, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(0), stream, d, pattern, w, resident_ctas, min_ctas));
+    CRISP_KERNEL("pe_hist1", stream, launch_pdl(hist1, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(1), stream, d, pattern, w, resident_ctas, min_ctas));
+    CRISP_KERNEL("pe_hist2", stream, launch_pdl(hist2, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(2), stream, d, pattern, w, resident_ctas, min_ctas));
   }
-  // histogram passes: a warp takes a row at a time; the grid is sized for a single PE head, the kernel uses as many
-  // CTAs per head as make one full wave over the PE heads there are
-  const long long causal = static_cast<long long>(d.nb) * (d.nb + 1) / 2;
-  // two CTAs of kHistThreads fit on an SM; a CTA must see fewer than 2^19 entries of a head (its 32-bit bin sums)
-  const int resident_ctas = 2 * n_sm;
-  const int min_ctas = static_cast<int>((causal + (1 << 19) - 1) >> 19);
-  const int hist_ctas = max(min_ctas, max(1, min((d.nb + 15) / 16, 64)));
-  auto hist_smem = [](int level) { return static_cast<size_t>(level_bins(level)) * 12; };
-  const bool vec = (d.nb & 3) == 0;  // rows start on 16-byte boundaries
-  auto* hist0 = vec ? pe_hist_kernel<0, true> : pe_hist_kernel<0, false>;
-  auto* hist1 = vec ? pe_hist_kernel<1, true> : pe_hist_kernel<1, false>;
-  auto* hist2 = vec ? pe_hist_kernel<2, true> : pe_hist_kernel<2, false>;
-  CRISP_CUDA_TRY(cudaFuncSetAttribute(hist1, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(hist_smem(1))),
-                 "select: smem attribute");
-  CRISP_KERNEL("pe_hist0", stream, launch_pdl(hist0, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(0), stream, d, pattern, w, resident_ctas, min_ctas));
-  CRISP_KERNEL("pe_hist1", stream, launch_pdl(hist1, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(1), stream, d, pattern, w, resident_ctas, min_ctas));
-  CRISP_KERNEL("pe_hist2", stream, launch_pdl(hist2, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(2), stream, d, pattern, w, resident_ctas, min_ctas));
   const int rows_ctas = max(1, min((d.nb + 31) / 32, 8));
   CRISP_KERNEL("pe_rows", stream, launch_pdl(pe_rows_kernel, dim3(rows_ctas, d.hq), dim3(1024), 0, stream, d, pattern, w));
   CRISP_KERNEL("fill", stream, launch_pdl(fill_kernel, dim3((d.nb + 7) / 8, d.hq), dim3(256), 0, stream, 
