@@ -1297,81 +1297,51 @@ pe_rows_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
 // ------------------------------------------------------------------------------------------------
 // Global offsets and the lists
 // ------------------------------------------------------------------------------------------------
-// The kept columns of one group of 128 consecutive entries of a PE row (four per lane) go, in ascending order,
-// to stage[base ...]; returns how many there were.  kEdge: the group may reach beyond the row's end.
+// The kept columns of one PE row, in ascending order, straight to the list.  A warp takes the row 32 consecutive
+// entries at a time (lane l holds column J0 + 32 u + l), so the kept entries of a group are the set bits of one
+// ballot, their places in the list the bit counts below each lane, and the group leaves as one store to
+// consecutive addresses - no scan, no staging.  Sixteen groups' loads are in flight per lane.
 template <bool kEdge>
-__device__ __forceinline__ int fill_group(const float (&z)[4], int J, int m, float M, float inv, unsigned int cutkey,
-                                          bool all, int take, int& ties_seen, int* stage, int base, int lane) {
-  bool keep[4], eq[4];
-  int n_eq_lane = 0;
+__device__ __forceinline__ void fill_step(const float* __restrict__ row, int J0, int m, float M, float inv,
+                                          unsigned int cutkey, bool all, int take, int& ties_seen, int& written,
+                                          int32_t* __restrict__ out, int lane) {
+  constexpr int kGroups = 16;
+  const unsigned int below = (1u << lane) - 1u;
+  float z[kGroups];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const unsigned int key = __float_as_uint(pe_value(z[e], M, inv));
-    const bool valid = !kEdge || J + e <= m;
-    keep[e] = valid && (all || key > cutkey || J + e == 0 || J + e == m);
-    eq[e] = valid && !all && key == cutkey;
-    n_eq_lane += eq[e] ? 1 : 0;
+  for (int u = 0; u < kGroups; ++u) {
+    const int J = J0 + 32 * u + lane;
+    z[u] = (!kEdge || J <= m) ? __ldcs(row + J) : 0.f;
   }
-  // ties are rare: their ranks in the row are worked out only in groups that hold one
-  if (__any_sync(0xffffffffu, n_eq_lane > 0)) {
-    int incl = n_eq_lane;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += t;
+  for (int u = 0; u < kGroups; ++u) {
+    const int J = J0 + 32 * u + lane;
+    if (kEdge && J0 + 32 * u > m) break;  // warp-uniform
+    const bool valid = !kEdge || J <= m;
+    const unsigned int key = __float_as_uint(pe_value(z[u], M, inv));
+    bool keep = valid && (all || key > cutkey || J == 0 || J == m);
+    const bool eq = valid && !all && key == cutkey;
+    // ties are rare: the first `take` of a row's ties, in column order, are kept
+    const unsigned int eq_bits = __ballot_sync(0xffffffffu, eq);
+    if (eq_bits != 0u) {
+      if (eq && ties_seen + __popc(eq_bits & below) < take) keep = true;
+      ties_seen += __popc(eq_bits);
     }
-    int rank = ties_seen + incl - n_eq_lane;
-#pragma unroll
-    for (int e = 0; e < 4; ++e)
-      if (eq[e]) {
-        keep[e] = keep[e] || rank < take;
-        ++rank;
-      }
-    ties_seen += __shfl_sync(0xffffffffu, incl, 31);
+    const unsigned int keep_bits = __ballot_sync(0xffffffffu, keep);
+    if (keep) out[written + __popc(keep_bits & below)] = J;
+    written += __popc(keep_bits);
   }
-  const int n_keep = (keep[0] ? 1 : 0) + (keep[1] ? 1 : 0) + (keep[2] ? 1 : 0) + (keep[3] ? 1 : 0);
-  int incl = n_keep;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(0xffffffffu, incl, o);
-    if (lane >= o) incl += t;
-  }
-  int pos = base + incl - n_keep;
-#pragma unroll
-  for (int e = 0; e < 4; ++e)
-    if (keep[e]) stage[pos++] = J + e;
-  return __shfl_sync(0xffffffffu, incl, 31);
 }
 
-template <bool kVec>
 __device__ __forceinline__ void fill_pe_row(const float* __restrict__ row, int m, float M, float inv, unsigned int cutkey,
-                                            bool all, int take, int32_t* __restrict__ out, int* stage, int lane) {
+                                            bool all, int take, int32_t* __restrict__ out, int lane) {
   int written = 0, ties_seen = 0;
-  // Steps of 512 columns (four loads per lane in flight); the kept columns of a step are gathered in shared
-  // memory and leave as contiguous 128-byte stores.
   for (int J0 = 0; J0 <= m; J0 += 512) {
-    const bool whole = J0 + 511 < m;  // the step lies inside the row and does not hold the diagonal
-    float z[4][4];
-    int n = 0;
-    if (whole) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) load_z4<kVec>(row, J0 + 128 * u + 4 * lane, m, z[u]);
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        n += fill_group<false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, cutkey, all, take, ties_seen, stage, n, lane);
+    if (J0 + 511 < m) {  // the step lies inside the row and does not hold the diagonal
+      fill_step<false>(row, J0, m, M, inv, cutkey, all, take, ties_seen, written, out, lane);
     } else {
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (J0 + 128 * u <= m) load_z4<kVec>(row, J0 + 128 * u + 4 * lane, m, z[u]);
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (J0 + 128 * u <= m)
-          n += fill_group<true>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, cutkey, all, take, ties_seen, stage, n, lane);
+      fill_step<true>(row, J0, m, M, inv, cutkey, all, take, ties_seen, written, out, lane);
     }
-    __syncwarp();
-    for (int i = lane; i < n; i += 32) out[written + i] = stage[i];
-    written += n;
-    __syncwarp();
   }
 }
 
@@ -1380,10 +1350,12 @@ fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs 
             int32_t* __restrict__ col_idx, int64_t capacity, int64_t* __restrict__ nnz_needed, int* status) {
   pdl_enter();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.y;
+  // CTAs that start together hold the same rows of different heads, so the cheap rows of the VS heads run under
+  // the memory traffic of the PE heads' rows
+  const int h = blockIdx.x;
   // offsets of the heads: every CTA adds the (few) head totals itself
   __shared__ long long s_base, s_total;
-  __shared__ int stage_all[8][512];
+  __shared__ int stage_all[8][1024];  // VS rows: the entries of 32 bitmap words
   if (threadIdx.x < 32) {
     long long before = 0, all = 0;
     for (int hh = lane; hh < d.hq; hh += 32) {
@@ -1408,7 +1380,7 @@ fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs 
     if (total > capacity) atomicExch(status, CRISP_ERR_CAPACITY);
   }
   // long rows first, so that the tail of the launch is made of short ones
-  const int m = d.nb - 1 - (blockIdx.x * 8 + warp);
+  const int m = d.nb - 1 - (blockIdx.y * 8 + warp);
   if (m < 0) return;
   const size_t rbase = static_cast<size_t>(h) * d.nb;
   const long long start = head_base + w.local_off[rbase + m];
@@ -1423,6 +1395,7 @@ fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs 
     const uint32_t* selv = w.selv + static_cast<size_t>(h) * w.words;
     const uint32_t* selsr = w.selsr + static_cast<size_t>(h) * (w.words + 2);
     const int nwords = (m >> 5) + 1;
+    int* stage = stage_all[warp];
     for (int w0 = 0; w0 < nwords; w0 += 32) {
       const int wd = w0 + lane;
       uint32_t bits = wd < nwords ? vs_keep_word(selv, selsr, d.nb, m, wd) : 0u;
@@ -1433,26 +1406,25 @@ fill_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPtrs 
         const int t = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += t;
       }
-      // emit word by word, lane b owning bit b: the entries of a word go out as one contiguous store
-      const int nw = min(32, nwords - w0);
-      for (int k = 0; k < nw; ++k) {
-        const uint32_t wbits = __shfl_sync(0xffffffffu, bits, k);
-        if (wbits == 0u) continue;
-        const int base = written + __shfl_sync(0xffffffffu, incl - c, k);
-        if ((wbits >> lane) & 1u) out[base + __popc(wbits & ((1u << lane) - 1u))] = (w0 + k) * 32 + lane;
+      // every lane unpacks its own word into the warp's staging area (a word holds a handful of entries, so this
+      // takes as many rounds as the fullest word has bits), then the chunk leaves as contiguous 128-byte stores
+      const int n_chunk = __shfl_sync(0xffffffffu, incl, 31);
+      int pos = incl - c;
+      while (bits != 0u) {
+        stage[pos++] = wd * 32 + __ffs(bits) - 1;
+        bits &= bits - 1u;
       }
-      written += __shfl_sync(0xffffffffu, incl, 31);
+      __syncwarp();
+      for (int i = lane; i < n_chunk; i += 32) out[written + i] = stage[i];
+      __syncwarp();
+      written += n_chunk;
     }
   } else {
     const CutState c = w.cut[h];
     const float* row = w.amat + (rbase + m) * d.nb;
     const float M = w.row_m[rbase + m], inv = w.row_inv[rbase + m];
     const int take = w.take[rbase + m];
-    if ((d.nb & 3) == 0) {
-      fill_pe_row<true>(row, m, M, inv, c.cutkey, c.take == -1, take, out, stage_all[warp], lane);
-    } else {
-      fill_pe_row<false>(row, m, M, inv, c.cutkey, c.take == -1, take, out, stage_all[warp], lane);
-    }
+    fill_pe_row(row, m, M, inv, c.cutkey, c.take == -1, take, out, lane);
   }
 }
 
@@ -1575,7 +1547,7 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
   }
   const int rows_ctas = max(1, min((d.nb + 31) / 32, 8));
   CRISP_KERNEL("pe_rows", stream, launch_pdl(pe_rows_kernel, dim3(rows_ctas, d.hq), dim3(1024), 0, stream, d, pattern, w));
-  CRISP_KERNEL("fill", stream, launch_pdl(fill_kernel, dim3((d.nb + 7) / 8, d.hq), dim3(256), 0, stream, 
+  CRISP_KERNEL("fill", stream, launch_pdl(fill_kernel, dim3(d.hq, (d.nb + 7) / 8), dim3(256), 0, stream, 
                                    d, pattern, w, row_ptr, col_idx, capacity, nnz_needed, status));
   CRISP_CUDA_TRY(cudaGetLastError(), "select: launch");
   return CRISP_OK;
