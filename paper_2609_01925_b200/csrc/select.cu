@@ -836,6 +836,77 @@ __device__ __forceinline__ void hist_group(const float (&z)[4], int J, int m, fl
     }
 }
 
+// Level 1 of one group of 128 consecutive entries, four per lane.  Every entry the level sees has the cut's
+// exponent, and its bin is the upper twelve bits of its mantissa, so a bin's sum of significands is its count
+// times a constant plus the sum of the entries' lower eleven bits: count (bits 21-31) and sum (bits 0-20) share
+// one 32-bit word `pk` and an entry costs ONE shared-memory add.  The fields hold 1024 entries; the add returns
+// the word's old value, and a thread that finds 256 or more entries in it moves the word's content to the
+// bin's wide counters (cnt, slo) before its next add, so with 512 threads, each with at most one add between two
+// checks, a word never holds more than 256 + 512 entries.  Entries that share the bin of the warp's first pending
+// entry are summed across the warp first and go to the wide counters directly (a flat map puts every entry there).
+constexpr unsigned int kPkShift = 21, kPkDrain = 256;
+template <bool kMasked>
+__device__ __forceinline__ void hist1_group(const float (&z)[4], int J, int m, float M, float inv, unsigned int prefix,
+                                            unsigned int* cnt, unsigned int* slo, unsigned int* pk, const SelectPtrs& w,
+                                            int h, int lane) {
+  unsigned int key[4];
+  int bin[4];
+  bool any = false;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    key[e] = __float_as_uint(pe_value(z[e], M, inv));
+    const bool ins = (!kMasked || J + e <= m) && (key[e] >> kL0Shift) == (prefix >> kL0Shift);
+    bin[e] = ins ? static_cast<int>((key[e] >> kL1Shift) & (kL1Bins - 1)) : -1;
+    any = any || ins;
+  }
+  if (!__any_sync(0xffffffffu, any)) return;  // nothing of this group lies in the cut's bin
+  if ((prefix >> 23) < kMinFastExp) {          // values below 2^-37: straight to the global histogram
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (bin[e] >= 0) hist_slow_add(w, h, 1, bin[e], __uint_as_float(key[e]));
+    return;
+  }
+  {
+    const bool left = (bin[0] & bin[1] & bin[2] & bin[3]) >= 0;  // some bin is not -1
+    const uint32_t have = __ballot_sync(0xffffffffu, left);
+    const int first = bin[0] >= 0 ? bin[0] : (bin[1] >= 0 ? bin[1] : (bin[2] >= 0 ? bin[2] : bin[3]));
+    const int ref = __shfl_sync(0xffffffffu, first, __ffs(have) - 1);
+    unsigned int n = 0u, lo = 0u;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+      if (bin[e] == ref && bin[e] >= 0) ++n;
+    // worth a warp-wide sum only when the bin is crowded
+    if (__reduce_add_sync(0xffffffffu, n) > 8u) {
+      n = 0u;
+#pragma unroll
+      for (int e = 0; e < 4; ++e)
+        if (bin[e] == ref) {
+          ++n;
+          lo += key[e] & 0x7FFu;
+          bin[e] = -1;
+        }
+      n = __reduce_add_sync(0xffffffffu, n);
+      lo = __reduce_add_sync(0xffffffffu, lo);
+      if (lane == 0) {
+        atomicAdd(&cnt[ref], n);
+        atomicAdd(&slo[ref], lo);
+      }
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    if (bin[e] >= 0) {
+      const unsigned int old = atomicAdd(&pk[bin[e]], (1u << kPkShift) | (key[e] & 0x7FFu));
+      if ((old >> kPkShift) >= kPkDrain) {
+        const unsigned int t = atomicExch(&pk[bin[e]], 0u);
+        atomicAdd(&cnt[bin[e]], t >> kPkShift);
+        atomicAdd(&slo[bin[e]], t & ((1u << kPkShift) - 1u));
+      }
+    }
+    asm volatile("" ::: "memory");  // one add per thread between two checks
+  }
+}
+
 // Level 0 (bins = exponents) of one group of 128 consecutive entries, four per lane.  An entry is at most the
 // row's largest value, 1 / (row sum N_b), so its exponent is e_top - k with k >= 0, and most entries have k < 4.
 // Each lane keeps one packed 64-bit accumulator per k in registers - low-significand sum in bits 0-19,
@@ -961,6 +1032,8 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
         for (int u = 0; u < 4; ++u) {
           if (kLevel == 0) {
             hist0_group<false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, e_top, acc, cnt, slo, shi, w, h, lane);
+          } else if (kLevel == 1) {
+            hist1_group<false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane);
           } else {
             hist_group<kLevel, false>(z[u], J0 + 128 * u + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
           }
@@ -974,6 +1047,8 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
         load_z4<kVec>(row, J0 + 4 * lane, m, z);
         if (kLevel == 0) {
           hist0_group<true>(z, J0 + 4 * lane, m, M, inv, e_top, acc, cnt, slo, shi, w, h, lane);
+        } else if (kLevel == 1) {
+          hist1_group<true>(z, J0 + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane);
         } else {
           hist_group<kLevel, true>(z, J0 + 4 * lane, m, M, inv, prefix, cnt, slo, shi, w, h, lane, gt, in);
         }
@@ -995,8 +1070,15 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
       if (cnt[i] | slo[i] | shi[i]) {
         // the bin's exponent: its own index at level 0, the cut's exponent below
         const int e = kLevel == 0 ? i : static_cast<int>(prefix >> kL0Shift);
-        const unsigned long long sig = (static_cast<unsigned long long>(shi[i]) << 12) + slo[i];
-        atomicAdd(&gc[i], cnt[i]);
+        unsigned long long sig = (static_cast<unsigned long long>(shi[i]) << 12) + slo[i];
+        unsigned int n = cnt[i];
+        if (kLevel == 1) {
+          // shi is the packed word of hist1_group: count | sum of the lower eleven mantissa bits
+          n += shi[i] >> kPkShift;
+          sig = static_cast<unsigned long long>(n) * (0x800000ull | (static_cast<unsigned long long>(i) << kL1Shift)) +
+                slo[i] + (shi[i] & ((1u << kPkShift) - 1u));
+        }
+        atomicAdd(&gc[i], n);
         atomicAdd(&gm[i], sig << (e - kMinFastExp));
       }
   }
