@@ -1001,7 +1001,7 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   constexpr int nbins = level_bins(kLevel);
   unsigned int* cnt = reinterpret_cast<unsigned int*>(hist_raw);  // [nbins] each
   unsigned int* slo = cnt + nbins;
-  unsigned int* shi = slo + nbins;
+  unsigned int* shi = slo + nbins;  // at level 1: the packed count | sum words of hist1_group
   __shared__ unsigned long long warp_tot[17];
   __shared__ int first_hit;
   __shared__ int is_last;
