@@ -807,8 +807,9 @@ check_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   pdl_enter();
   if (gate != nullptr && *gate != 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int u = blockIdx.x * 4 + warp, h = blockIdx.y;
-  if (u >= n_pairs) return;
+  // long lists first (the late query blocks), so that the launch ends on the short ones
+  const int u = n_pairs - 1 - (blockIdx.x * 4 + warp), h = blockIdx.y;
+  if (u < 0) return;
   const int m0 = rows_per_item * u, m1 = m0 + 1;
   const int64_t* rp = row_ptr + static_cast<size_t>(h) * (d.nb + 1);
   const int64_t s0 = rp[m0], e0 = rp[m0 + 1];
@@ -816,19 +817,20 @@ check_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   const int64_t e1 = has1 ? rp[m1 + 1] : e0;
   bool bad = s0 < 0 || e0 - s0 < 1 || e0 - s0 > m0 + 1 || e1 > capacity || (has1 && (e1 - e0 < 1 || e1 - e0 > m1 + 1));
   if (!bad) {
-    // four loads per lane in flight; an entry is compared with the one before it (the lane below, or the last
+    // eight loads per lane in flight; an entry is compared with the one before it (the lane below, or the last
     // entry of the previous group of 32)
+    constexpr int kInFlight = 8;
     auto check = [&](int64_t from, int64_t to, int m) {
       int prev_last = -1;
-      for (int64_t i0 = from; i0 < to; i0 += 128) {
-        int c[4];
+      for (int64_t i0 = from; i0 < to; i0 += 32 * kInFlight) {
+        int c[kInFlight];
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
+        for (int v = 0; v < kInFlight; ++v) {
           const int64_t i = i0 + 32 * v + lane;
-          c[v] = i < to ? col_idx[i] : 0x7fffffff;
+          c[v] = i < to ? __ldcs(col_idx + i) : 0x7fffffff;
         }
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
+        for (int v = 0; v < kInFlight; ++v) {
           const int64_t i = i0 + 32 * v + lane;
           const bool live = i < to;
           int before = __shfl_up_sync(0xffffffffu, c[v], 1);
