@@ -909,8 +909,8 @@ __device__ __forceinline__ void hist1_group(const float (&z)[4], int J, int m, f
 
 // Level 0 (bins = exponents) of one group of 128 consecutive entries, four per lane.  An entry is at most the
 // row's largest value, 1 / (row sum N_b), so its exponent is e_top - k with k >= 0, and most entries have k < 4.
-// Each lane keeps one packed 64-bit accumulator per k in registers - low-significand sum in bits 0-19,
-// high-significand sum in bits 20-39, count from bit 40 - and the warp adds them up once per flush
+// Each lane keeps one packed 64-bit accumulator per k in registers - the sum of the 24-bit significands in the
+// low word, the count in the high word - and the warp adds them up once per flush
 // (hist0_flush), so such an entry costs a handful of integer instructions and no shared-memory traffic.  A group
 // in which any lane holds another kind of entry (k >= 4, or a value below 2^-37) takes the general path.
 template <bool kMasked>
@@ -935,25 +935,25 @@ __device__ __forceinline__ void hist0_group(const float (&z)[4], int J, int m, f
   for (int e = 0; e < 4; ++e) {
     const bool valid = !kMasked || J + e <= m;
     const int k = e_top - static_cast<int>(key[e] >> 23);
-    const unsigned long long packed = static_cast<unsigned long long>(key[e] & 0xFFFu) |
-                                      (static_cast<unsigned long long>(((key[e] >> 12) & 0x7FFu) | 0x800u) << 20) |
-                                      (1ull << 40);
+    // whole 24-bit significand in the low word (255 entries fit in 32 bits), count in the high word
+    const unsigned long long packed = static_cast<unsigned long long>((key[e] & 0x7FFFFFu) | 0x800000u) | (1ull << 32);
 #pragma unroll
     for (int b = 0; b < 4; ++b)
       if (valid && k == b) acc[b] += packed;
   }
 }
 // Adds the lanes' accumulators into the CTA's shared-memory bins e_top .. e_top - 3 and clears them.  A lane may
-// hold at most 255 entries per accumulator between two flushes (the 20-bit fields).
+// hold at most 255 entries per accumulator between two flushes (255 significands fit in 32 bits).
 __device__ __forceinline__ void hist0_flush(unsigned long long (&acc)[4], int e_top, unsigned int* cnt,
                                             unsigned int* slo, unsigned int* shi, int lane) {
 #pragma unroll
   for (int b = 0; b < 4; ++b) {
-    const unsigned int n = static_cast<unsigned int>(acc[b] >> 40);
+    const unsigned int n = static_cast<unsigned int>(acc[b] >> 32);
     if (__any_sync(0xffffffffu, n != 0u)) {
+      // the lanes' significand sums in two halves: the low twelve bits and the rest (below 2^20 per lane)
       const unsigned int ns = __reduce_add_sync(0xffffffffu, n);
-      const unsigned int lo = __reduce_add_sync(0xffffffffu, static_cast<unsigned int>(acc[b] & 0xFFFFFu));
-      const unsigned int hi = __reduce_add_sync(0xffffffffu, static_cast<unsigned int>((acc[b] >> 20) & 0xFFFFFu));
+      const unsigned int lo = __reduce_add_sync(0xffffffffu, static_cast<unsigned int>(acc[b]) & 0xFFFu);
+      const unsigned int hi = __reduce_add_sync(0xffffffffu, static_cast<unsigned int>(acc[b]) >> 12);
       if (lane == 0) {
         atomicAdd(&cnt[e_top - b], ns);
         atomicAdd(&slo[e_top - b], lo);
