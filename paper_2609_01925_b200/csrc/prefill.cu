@@ -803,7 +803,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 __global__ void __launch_bounds__(128)
 check_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                    int* __restrict__ cost_hist, int n_pairs, int n_cost, int group_kv, const int* __restrict__ gate,
-                   int* __restrict__ status, long long capacity, int rows_per_item) {
+                   int* __restrict__ status, long long capacity, int rows_per_item, int* __restrict__ plain_order) {
   pdl_enter();
   if (gate != nullptr && *gate != 0) return;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -845,6 +845,11 @@ check_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   }
   if (__any_sync(0xffffffffu, bad)) {
     if (lane == 0) atomicExch(status, CRISP_ERR_BAD_LIST);
+    return;
+  }
+  if (plain_order != nullptr) {
+    // every CTA of the attention kernel gets one item at most: any order will do, and no sort follows
+    if (lane == 0) plain_order[h * n_pairs + u] = (n_pairs - 1 - u) * d.hq + h;
     return;
   }
   // sort key: KV head first, then decreasing cost (= tile steps = len(m0) + len(m1))
@@ -972,17 +977,22 @@ int launch_prefill(const Dims& d, const void* q, const void* k, const void* v, c
   } else {
     // the lists are checked (and the items entered into the schedule's histogram) before anything walks them
     const long long capacity = static_cast<long long>(d.hq) * d.nb * (static_cast<long long>(d.nb) + 1) / 2;
+    // with an SM for every item the schedule needs no sort: check_lists writes the order itself
+    const bool one_item_per_cta = a.n_items <= n_sm;
     CRISP_KERNEL("check_lists", stream,
                  launch_pdl(check_lists_kernel, dim3((a.n_pairs + 3) / 4, d.hq), dim3(128), 0, stream, d, row_ptr, col_idx, w.cost_hist,
-                            a.n_pairs, w.n_cost, a.group_kv, gate, a.status, capacity, a.rows_per_item));
-    const size_t scatter_smem = sizeof(int) * static_cast<size_t>(w.n_cost);
-    if (scatter_smem > 48 * 1024)
-      CRISP_CUDA_TRY(cudaFuncSetAttribute(sched_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(scatter_smem)),
-                     "prefill: scatter smem attribute");
-    CRISP_KERNEL("sched_scatter", stream,
-                 launch_pdl(sched_scatter_kernel, dim3((a.n_pairs + 255) / 256, d.hq), dim3(256), scatter_smem, stream, 
-                     d, row_ptr, w.cost_hist, w.cursor, w.order, a.n_pairs, w.n_cost, a.group_kv, gate, a.status, a.rows_per_item));
+                            a.n_pairs, w.n_cost, a.group_kv, gate, a.status, capacity, a.rows_per_item,
+                            one_item_per_cta ? w.order : nullptr));
+    if (!one_item_per_cta) {
+      const size_t scatter_smem = sizeof(int) * static_cast<size_t>(w.n_cost);
+      if (scatter_smem > 48 * 1024)
+        CRISP_CUDA_TRY(cudaFuncSetAttribute(sched_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            static_cast<int>(scatter_smem)),
+                       "prefill: scatter smem attribute");
+      CRISP_KERNEL("sched_scatter", stream,
+                   launch_pdl(sched_scatter_kernel, dim3((a.n_pairs + 255) / 256, d.hq), dim3(256), scatter_smem, stream,
+                       d, row_ptr, w.cost_hist, w.cursor, w.order, a.n_pairs, w.n_cost, a.group_kv, gate, a.status, a.rows_per_item));
+    }
     CRISP_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         static_cast<int>(smem)),
                    "prefill: smem attribute");
