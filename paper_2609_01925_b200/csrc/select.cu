@@ -1092,6 +1092,52 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   locate_cut(d, w, h, kLevel, warp_tot, &first_hit);
 }
 
+// The head-wide part of a PE head's row bookkeeping, run by one CTA of 1024 threads once the per-row counts of the
+// entries above the cut's key (n_gt) and equal to it (n_eq) are final: the ties taken per row (in row-major order),
+// the forced entries, the row lengths and their scan.
+__device__ void pe_rows_finish(const Dims& d, const SelectPtrs& w, int h, const CutState& c, long long* scratch) {
+  const int tid = threadIdx.x;
+  const size_t base = static_cast<size_t>(h) * d.nb;
+  const float* am = w.amat + base * d.nb;
+  const int seg = (d.nb + 1023) / 1024;
+  const int b0 = min(tid * seg, d.nb), b1 = min(b0 + seg, d.nb);
+  long long local = 0;
+  if (c.take != -1)
+    for (int m = b0; m < b1; ++m) local += __ldcg(&w.n_eq[base + m]);
+  long long before = block_exclusive_scan_1024(local, scratch, nullptr);
+  long long len_local = 0;
+  for (int m = b0; m < b1; ++m) {
+    int count, take;
+    if (c.take == -1) {
+      take = 0;
+      count = m + 1;  // every causal entry
+    } else {
+      const int eq = __ldcg(&w.n_eq[base + m]);
+      const long long left = c.take - before;
+      take = static_cast<int>(left <= 0 ? 0 : (left >= eq ? eq : left));
+      before += eq;
+      // the forced entries (column 0 and the diagonal): selected already, or to be added
+      const float M = w.row_m[base + m], inv = w.row_inv[base + m];
+      const float* row = am + static_cast<size_t>(m) * d.nb;
+      const unsigned int k0 = __float_as_uint(pe_value(row[0], M, inv)), km = __float_as_uint(pe_value(row[m], M, inv));
+      const bool sel0 = k0 > c.cutkey || (k0 == c.cutkey && take >= 1);   // column 0 is the row's first tie
+      const bool selm = km > c.cutkey || (km == c.cutkey && take >= eq);  // the diagonal is its last
+      count = __ldcg(&w.n_gt[base + m]) + take + (sel0 ? 0 : 1);
+      if (m > 0) count += selm ? 0 : 1;
+    }
+    w.take[base + m] = take;
+    w.counts[base + m] = count;
+    len_local += count;
+  }
+  long long total;
+  long long run = block_exclusive_scan_1024(len_local, scratch, &total);
+  for (int m = b0; m < b1; ++m) {
+    w.local_off[base + m] = static_cast<int>(run);
+    run += w.counts[base + m];
+  }
+  if (tid == 0) w.head_total[h] = total;
+}
+
 // ------------------------------------------------------------------------------------------------
 // PE heads of short prompts (N_b <= kSmallNb, i.e. up to 8064 tokens): pooled logits, row statistics and the
 // gamma cut in one CTA
@@ -1101,7 +1147,7 @@ pe_hist_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
 // fp32 dot products of the block means, the rows' maxima and sums, a bitonic sort of the values and a prefix sum
 // of their masses in sorted order, which gives the cut directly.  It leaves exactly what pe_logits_kernel and the histogram levels
 // leave (the logits, the rows' normalisers, the cut state, and per row the number of entries above the cut's key
-// and equal to it), so pe_rows_kernel and fill_kernel follow unchanged.
+// and equal to it) and ends with the head-wide step of pe_rows_kernel, so fill_kernel follows unchanged.
 constexpr int kSmallNb = 63;  // 2016 entries: the sort network stays at 2048 keys
 constexpr int kSmallPitch = 132;  // floats per block mean in shared memory: 16-byte aligned rows, no bank conflicts
 struct SmallSmem {
@@ -1276,9 +1322,8 @@ pe_small_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectP
     s.cut = c;
     w.cut[h] = c;
   }
-  if (c.take == -1) return;
-
   // ---- per row: entries above the cut's key and equal to it
+  if (c.take != -1)
   for (int m = warp; m < nb; m += 32) {
     const float* zr = &s.z[m * (m + 1) / 2];
     const float M = s.row_m[m], inv = s.row_inv[m];
@@ -1295,6 +1340,9 @@ pe_small_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectP
       w.n_eq[static_cast<size_t>(h) * nb + m] = eq;
     }
   }
+  // ---- ties per row, row lengths, their scan (what pe_rows_kernel does for the long prompts)
+  __syncthreads();
+  pe_rows_finish(d, w, h, c, s.scratch);
 }
 
 // Per PE head: exact per-row counts of the entries above and tied with the cut, the ties taken per row (in
@@ -1337,43 +1385,7 @@ pe_rows_kernel(const Dims d, const int32_t* __restrict__ pattern, const SelectPt
   __syncthreads();
   if (!is_last) return;
   __threadfence();
-  const int seg = (d.nb + 1023) / 1024;
-  const int b0 = min(tid * seg, d.nb), b1 = min(b0 + seg, d.nb);
-  long long local = 0;
-  if (c.take != -1)
-    for (int m = b0; m < b1; ++m) local += __ldcg(&w.n_eq[base + m]);
-  long long before = block_exclusive_scan_1024(local, scratch, nullptr);
-  long long len_local = 0;
-  for (int m = b0; m < b1; ++m) {
-    int count, take;
-    if (c.take == -1) {
-      take = 0;
-      count = m + 1;  // every causal entry
-    } else {
-      const int eq = __ldcg(&w.n_eq[base + m]);
-      const long long left = c.take - before;
-      take = static_cast<int>(left <= 0 ? 0 : (left >= eq ? eq : left));
-      before += eq;
-      // the forced entries (column 0 and the diagonal): selected already, or to be added
-      const float M = w.row_m[base + m], inv = w.row_inv[base + m];
-      const float* row = am + static_cast<size_t>(m) * d.nb;
-      const unsigned int k0 = __float_as_uint(pe_value(row[0], M, inv)), km = __float_as_uint(pe_value(row[m], M, inv));
-      const bool sel0 = k0 > c.cutkey || (k0 == c.cutkey && take >= 1);   // column 0 is the row's first tie
-      const bool selm = km > c.cutkey || (km == c.cutkey && take >= eq);  // the diagonal is its last
-      count = __ldcg(&w.n_gt[base + m]) + take + (sel0 ? 0 : 1);
-      if (m > 0) count += selm ? 0 : 1;
-    }
-    w.take[base + m] = take;
-    w.counts[base + m] = count;
-    len_local += count;
-  }
-  long long total;
-  long long run = block_exclusive_scan_1024(len_local, scratch, &total);
-  for (int m = b0; m < b1; ++m) {
-    w.local_off[base + m] = static_cast<int>(run);
-    run += w.counts[base + m];
-  }
-  if (tid == 0) w.head_total[h] = total;
+  pe_rows_finish(d, w, h, c, scratch);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1627,8 +1639,10 @@ int launch_select(const Dims& d, const void* q, const void* k, const int32_t* pa
     CRISP_KERNEL("pe_hist1", stream, launch_pdl(hist1, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(1), stream, d, pattern, w, resident_ctas, min_ctas));
     CRISP_KERNEL("pe_hist2", stream, launch_pdl(hist2, dim3(hist_ctas, d.hq), dim3(kHistThreads), hist_smem(2), stream, d, pattern, w, resident_ctas, min_ctas));
   }
-  const int rows_ctas = max(1, min((d.nb + 31) / 32, 8));
-  CRISP_KERNEL("pe_rows", stream, launch_pdl(pe_rows_kernel, dim3(rows_ctas, d.hq), dim3(1024), 0, stream, d, pattern, w));
+  if (d.nb > kSmallNb) {  // (pe_small_kernel ends with the same step)
+    const int rows_ctas = max(1, min((d.nb + 31) / 32, 8));
+    CRISP_KERNEL("pe_rows", stream, launch_pdl(pe_rows_kernel, dim3(rows_ctas, d.hq), dim3(1024), 0, stream, d, pattern, w));
+  }
   CRISP_KERNEL("fill", stream, launch_pdl(fill_kernel, dim3(d.hq, (d.nb + 7) / 8), dim3(256), 0, stream, 
                                    d, pattern, w, row_ptr, col_idx, capacity, nnz_needed, status));
   CRISP_CUDA_TRY(cudaGetLastError(), "select: launch");

@@ -109,8 +109,8 @@ def test_per_kernel_profile_records():
     names = [n for n, _ in recs]
     assert names[:2] == ["proxy", "tile_sums"] and names[-1] == "prefill_sparse" and "fill" in names
     # 2048 tokens take the short-prompt selection kernel and, with an SM for every attention item, no schedule
-    # sort (8 launches); more than 64 blocks take 12
-    assert len(names) == 8 and "pe_small" in names and "sched_scatter" not in names
+    # sort (7 launches); more than 64 blocks take 12
+    assert len(names) == 7 and "pe_small" in names and "sched_scatter" not in names and "pe_rows" not in names
     assert all(ms > 0 for _, ms in recs)
     layer.route(q, k)
     assert B.crisp_profile_read() == []
