@@ -818,27 +818,30 @@ check_lists_kernel(const Dims d, const int64_t* __restrict__ row_ptr, const int3
   bool bad = s0 < 0 || e0 - s0 < 1 || e0 - s0 > m0 + 1 || e1 > capacity || (has1 && (e1 - e0 < 1 || e1 - e0 > m1 + 1));
   if (!bad) {
     // eight loads per lane in flight; an entry is compared with the one before it (the lane below, or the last
-    // entry of the previous group of 32)
+    // entry of the previous group of 32).  In range and strictly ascending; the last entry is the diagonal.
     constexpr int kInFlight = 8;
     auto check = [&](int64_t from, int64_t to, int m) {
+      const int32_t* lst = col_idx + from;
+      const int len = static_cast<int>(to - from);
       int prev_last = -1;
-      for (int64_t i0 = from; i0 < to; i0 += 32 * kInFlight) {
+      for (int i0 = 0; i0 < len; i0 += 32 * kInFlight) {
         int c[kInFlight];
 #pragma unroll
         for (int v = 0; v < kInFlight; ++v) {
-          const int64_t i = i0 + 32 * v + lane;
-          c[v] = i < to ? __ldcs(col_idx + i) : 0x7fffffff;
+          const int i = i0 + 32 * v + lane;
+          c[v] = i < len ? __ldcs(lst + i) : 0x7fffffff;  // the padding passes the ascent test, not the range test
         }
 #pragma unroll
         for (int v = 0; v < kInFlight; ++v) {
-          const int64_t i = i0 + 32 * v + lane;
-          const bool live = i < to;
+          const int i = i0 + 32 * v + lane;
           int before = __shfl_up_sync(0xffffffffu, c[v], 1);
           if (lane == 0) before = prev_last;
-          bad = bad || (live && !(c[v] >= 0 && c[v] <= m && c[v] > before && (i + 1 < to || c[v] == m)));
+          bad = bad || (i < len && (static_cast<unsigned int>(c[v]) > static_cast<unsigned int>(m) || c[v] <= before));
           prev_last = __shfl_sync(0xffffffffu, c[v], 31);
         }
       }
+      // (lists are not empty here: their lengths were checked above)
+      if (lane == 0) bad = bad || __ldg(lst + len - 1) != m;
     };
     check(s0, e0, m0);
     if (has1) check(e0, e1, m1);
