@@ -125,25 +125,32 @@ __device__ __forceinline__ Item decode_item(int pos, const Dims& d, const Prefil
 
 // The key blocks of ONE tile of an item, in order (what its softmax warps walk: they need neither the other
 // tile's blocks nor the position of a block in the K/V stream).  Sparse lists are fetched 32 entries at a time,
-// one per lane, and broadcast with a shuffle; all 32 lanes of the warp must call get together.
+// one per lane, and broadcast with a shuffle; all 32 lanes of the warp must call get together.  The fetch runs
+// one group of 32 ahead, so that its latency (the lists of a long prompt come from DRAM) never stalls the
+// softmax, which is the critical path of a step.
 template <bool kDense>
 struct TileReader {
   const int32_t* list;
-  uint32_t chunk;
+  uint32_t chunk, chunk_next;
   int n;  // blocks of the tile
-  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& a, int t) {
+  __device__ __forceinline__ void init(const Item& it, const PrefillArgs& a, int t, int lane) {
     if (kDense) {
       list = nullptr;
       n = (t == 0 ? it.m0 : it.m1) + 1;
+      chunk = chunk_next = 0;
     } else {
       list = a.col_idx + it.base0 + (t == 0 ? 0 : it.n0);
       n = t == 0 ? it.n0 : it.n1;
+      chunk = lane < n ? static_cast<uint32_t>(__ldg(list + lane)) : 0u;
+      chunk_next = 32 + lane < n ? static_cast<uint32_t>(__ldg(list + 32 + lane)) : 0u;
     }
-    chunk = 0;
   }
   __device__ __forceinline__ int get(int i, int lane) {
     if (kDense) return i;
-    if ((i & 31) == 0) chunk = (i + lane < n) ? static_cast<uint32_t>(list[i + lane]) : 0u;
+    if ((i & 31) == 0 && i > 0) {
+      chunk = chunk_next;
+      chunk_next = (i + 32 + lane < n) ? static_cast<uint32_t>(__ldg(list + i + 32 + lane)) : 0u;
+    }
     return static_cast<int>(__shfl_sync(0xffffffffu, chunk, i & 31));
   }
 };
@@ -680,13 +687,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const Item it = decode_item<kDense>(idx, d, a);
       if (t == 1 && !it.tile1) continue;
       TileReader<kDense> rd;
-      rd.init(it, a, t);
+      rd.init(it, a, t, lane);
       const int m_t = t == 0 ? it.m0 : it.m1;
       float m_used = 0.f, l_run = 0.f;
       bool first = true;
       for (int i = 0; i < rd.n && ok; ++i) {
-        const int J = rd.get(i, lane);
-        const bool diag = (J == m_t);
         const uint32_t ph = step_count & 1;
         // Each 64-key half is one step of the online softmax.  The rescale decision is taken per warp
         // (the TMEM accesses are warp-collective): if any row of the warp outgrew its reference maximum by
@@ -695,6 +700,8 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         ok = mbar_wait_warp(&s.s_full[t][0], ph, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
+        const int J = rd.get(i, lane);  // (behind the wait: an item's first fetch overlaps it)
+        const bool diag = (J == m_t);
         uint32_t x[2][32];
         tmem_ld_x32(s_addr, x[0]);
         tmem_ld_x32(s_addr + 32, x[1]);
