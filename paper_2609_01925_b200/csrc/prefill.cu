@@ -691,8 +691,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       const int m_t = t == 0 ? it.m0 : it.m1;
       float m_used = 0.f, l_run = 0.f;
       bool first = true;
+      // the key block of a step is looked up during the step before it (an item's first one here: the wait for its
+      // first S covers the fetch), so the shuffle never sits between the arrival of S and the work on it
+      int J_next = rd.get(0, lane);
       for (int i = 0; i < rd.n && ok; ++i) {
         const uint32_t ph = step_count & 1;
+        const int J = J_next;
+        const bool diag = (J == m_t);
         // Each 64-key half is one step of the online softmax.  The rescale decision is taken per warp
         // (the TMEM accesses are warp-collective): if any row of the warp outgrew its reference maximum by
         // more than the threshold, every row of the warp moves to its own current maximum.
@@ -700,11 +705,10 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
         ok = mbar_wait_warp(&s.s_full[t][0], ph, abort_flag);
         if (!ok) break;
         tc_fence_after_sync();
-        const int J = rd.get(i, lane);  // (behind the wait: an item's first fetch overlaps it)
-        const bool diag = (J == m_t);
         uint32_t x[2][32];
         tmem_ld_x32(s_addr, x[0]);
         tmem_ld_x32(s_addr + 32, x[1]);
+        if (i + 1 < rd.n) J_next = rd.get(i + 1, lane);  // under the TMEM loads
         tmem_ld_wait();
         float mx = (diag ? row_max<true>(x, r, 0) : row_max<false>(x, r, 0)) * d.scale_log2;
         if (first) {
