@@ -374,7 +374,7 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
     for (int i = 0; i < 4; ++i) {
       mbar_init(&s.itm_full[i], 1);
-      mbar_init(&s.itm_empty[i], 10);  // two issuers and eight softmax warps
+      mbar_init(&s.itm_empty[i], 11);  // two issuers, eight softmax warps and the list prefetcher
     }
     for (int i = 0; i < 2; ++i)
       for (int h = 0; h < 2; ++h) {
@@ -796,7 +796,28 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
     }
   }
   else {
-    reg_dealloc<kRegsOther>();  // idle warps of the third warpgroup
+    // =============================================================== warp 11: pulls an item's lists into L2
+    // The lists of a long prompt come from DRAM, and producer, issuers and softmax warps all walk them with
+    // little look-ahead.  This warp touches every 128-byte line of an item's lists when the item starts (hints
+    // only: nobody waits for them), so all but the first few entries are in L2 when they are asked for.
+    reg_dealloc<kRegsOther>();
+    bool ok = true;
+    for (int it_count = 0; ok; ++it_count) {
+      const int qslot = it_count & 3;
+      ok = mbar_wait_warp(&s.itm_full[qslot], (it_count >> 2) & 1, abort_flag);
+      if (!ok) break;
+      const int idx = *reinterpret_cast<volatile int*>(&s.item_q[qslot]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s.itm_empty[qslot]);
+      if (idx < 0) break;
+      if (!kDense) {
+        const Item it = decode_item<kDense>(idx, d, a);
+        const char* lists = reinterpret_cast<const char*>(a.col_idx + it.base0);
+        const long long bytes = static_cast<long long>(it.n0 + it.n1) * 4;
+        for (long long off = static_cast<long long>(lane) * 128; off < bytes; off += 32 * 128)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(lists + off));
+      }
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
