@@ -499,7 +499,7 @@ def main():
                      "peak_source": f"{peaks['source']} ({'sustained' if peak == peaks['bf16_sustained'] else 'burst'})",
                      # ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel: constants
                      # copied from the committed captures (nothing is parsed at run time); other workloads: null
-                     "traffic": {"L512k": 123_110_000_000, "L128k": 4_713_770_240}.get(wl.name) if wl.n_q_heads == w.n_q_heads else None,
+                     "traffic": {"L512k": 123_110_000_000, "L128k": 4_682_425_856}.get(wl.name) if wl.n_q_heads == w.n_q_heads else None,
                      "traffic_source": {"L512k": "profiles/dram_traffic_L128k_ncu.md, section 'Earlier capture at L512k' "
                                                  "(118.8 GB read + 4.31 GB written per launch; its tensor-core loop is "
                                                  "unchanged since); algorithmic 10.7 GB: K/V are re-streamed per item "
