@@ -14,6 +14,7 @@
 //   warps 4-7   softmax of tile 1
 //   warp  8     TMA producer (one thread): Q once per item, K and V blocks through one five-slot ring
 //   warps 9,10  MMA issuers, one thread per tile: S_t = Q_t K^T (SS) and O_t += P_t V (P read from TMEM)
+//   warp  11    pulls the lines of an item's lists into L2 when the item starts (sparse kernel; hints only)
 // TMEM (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each.  Every key block is worked on in two
 // halves of 64 keys (A, B): S_A and S_B are separate MMAs (N = 64) into the two halves of S_t, and P_t (bf16)
 // is written over the columns of S_B.  The columns of S_A are therefore free as soon as the softmax has read
@@ -26,7 +27,8 @@
 // Each half is one step of the online softmax, which rescales O lazily, only when the running maximum
 // grows by more than 2^8, and does it in place in TMEM.
 // Both issuers see every load of the K/V ring in order and release every slot once, so the ring never runs
-// ahead of either tile; apart from that the two tiles run free of each other.
+// ahead of either tile; apart from that the two tiles run free of each other, except that tile 0's softmax warps
+// trail tile 1's by part of a run of exponentials (see the pacing in the softmax branch).
 // Work items are handed out dynamically: the producer takes the next position of the cost-sorted order from
 // a device counter and passes it to the other roles through a four-slot queue, which balances the load and
 // keeps the CTAs that run at the same time on the same K/V blocks (they share them through L2).
