@@ -467,6 +467,11 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
 
       // Operand descriptors are built once; inside the loops only the 14-bit start-address field moves
       // (a compile-time offset per K step), so issuing an MMA costs two integer adds.
+      // (an offset moves only the 14-bit start-address field in the descriptor's low word and cannot carry out
+      // of it: a 32-bit add on the low word, not a 64-bit one - the issuing threads are on the critical path)
+      auto desc_add = [](uint64_t desc, uint32_t off) {
+        return (desc & 0xffffffff00000000ull) | static_cast<uint64_t>(static_cast<uint32_t>(desc) + off);
+      };
       const uint64_t q_desc = umma_desc_sw128(smem_u32(s.q[t][0]), 0, 1024);
       // slot s of the ring starts 32 KB after slot s - 1: +2048 in the descriptor's address field
       const uint64_t k_desc0 = umma_desc_sw128(smem_u32(s.kv[0][0]), 0, 1024);      // K block: K-major B operand
@@ -499,13 +504,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       auto mma_qk_half = [&](const Step& st, int h) {
         const int slot = (2u * st.ec) % kStages;
         // key rows 64-127 of the block start 64 x 128 B further into each 64-dim half
-        const uint64_t bd0 = k_desc0 + static_cast<uint64_t>(slot) * 2048u + static_cast<uint64_t>(h) * (8192u >> 4);
+        const uint64_t bd0 = desc_add(k_desc0, static_cast<uint32_t>(slot) * 2048u + static_cast<uint32_t>(h) * (8192u >> 4));
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
           // K step kk: 64-column half kk / 4 (16 KB apart), 32 bytes per step inside the swizzle atom
           constexpr uint32_t kHalf = 16384 >> 4, kStep = 32 >> 4;
-          const uint64_t off = static_cast<uint64_t>((kk >> 2) * kHalf + (kk & 3) * kStep);
-          umma_ss(s_tm + h * 64, q_desc + off, bd0 + off, idesc_qk, kk > 0);
+          const uint32_t off = (kk >> 2) * kHalf + (kk & 3) * kStep;
+          umma_ss(s_tm + h * 64, desc_add(q_desc, off), desc_add(bd0, off), idesc_qk, kk > 0);
         }
         umma_commit(&s.s_full[t][h]);
         if (h == 1) {
@@ -516,13 +521,13 @@ prefill_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant
       // O_t += P_h V_h: four steps of 16 keys; P_h (bf16) sits in columns 64 + 32 h .. of the tile's S region
       auto mma_pv_half = [&](const Step& st, int h, bool first) {
         const int slot = (2u * st.ec + 1u) % kStages;
-        const uint64_t bd0 = v_desc0 + static_cast<uint64_t>(slot) * 2048u;
+        const uint64_t bd0 = desc_add(v_desc0, static_cast<uint32_t>(slot) * 2048u);
 #pragma unroll
         for (int k4 = 0; k4 < 4; ++k4) {
           const int kk = h * 4 + k4;
           // V block as the MN-major B operand: 16 keys per step = two groups of 8 key rows = 2048 B
-          const uint64_t off = static_cast<uint64_t>(kk * (2048 >> 4));
-          umma_ts(o_tm, s_tm + 64 + kk * 8, bd0 + off, idesc_pv, (kk > 0 || !first) ? 1u : 0u);
+          const uint32_t off = kk * (2048 >> 4);
+          umma_ts(o_tm, s_tm + 64 + kk * 8, desc_add(bd0, off), idesc_pv, (kk > 0 || !first) ? 1u : 0u);
         }
         umma_commit(&s.o_done[t][h]);
         if (h == 1) umma_commit(&s.kv_empty[slot]);
